@@ -1,0 +1,21 @@
+"""CPU oracle for the VC-Attention hot path -- TEST INFRASTRUCTURE, not product code.
+
+A plain, slow NumPy restatement of what the path computes, written from the paper:
+
+* ``codecs``     number formats (E4M3, E2M1, bf16) and the ExpCast-FP8 map (Eq. 7)
+* ``prep``       the preprocessing chain (Sec. 3.4 "Fused preprocessing", App. B)
+* ``attention``  exact fp64 attention and the emulated low-bit recurrence
+                 (Eq. 1, Eq. 6, Eq. 7)
+
+Only the tests, ``__graft_entry__.smoke()`` and the ``cpu_baseline`` / ``--impl reference``
+legs of ``bench.py`` may import this package.  It shares no code with the CUDA path and
+never imports it.
+
+Pins (tests/test_oracle_*.py): the codecs are pinned exhaustively and against an
+independent library cast; Hadamard, K smoothing, permutation, block demeaning and mean
+restoration are pinned by the identities the paper states for them; ExpCast-FP8 by the
+paper's worked example and printed constants; the recurrence by brute-force attention
+with quantization switched off.  The *end-to-end quantized* output has no printed value
+in the paper: "parity unpinned" for the granularity of the Q/K scales, the NVFP4
+second-level scales and the RoPE channel split, which are readings fixed by this build.
+"""
