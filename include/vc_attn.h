@@ -1,0 +1,152 @@
+/*
+ * vc_attn.h -- C ABI of the VC-Attention hot path on NVIDIA B200 (sm_100a).
+ *
+ * The library computes low-bit attention for video-diffusion transformers in two stages:
+ *
+ *   vc_prep      the fused preprocessing pass (paper Sec. 3.4 "Fused preprocessing",
+ *                App. B): RoPE, Q/K Hadamard rotation, K channel-mean smoothing, V
+ *                per-128-token block-mean smoothing (Eq. 4), gather by the token-group
+ *                permutation pi (Eq. 3), padding, quantization to the 8-bit (FP8 E4M3) or
+ *                4-bit (NVFP4: E2M1 under a per-16 E4M3 microscale) formats with scales.
+ *   vc_attn_fwd  the quantized attention forward: low-bit Q K^T, the online softmax of
+ *                Eq. 1 whose exponent is written directly as an E4M3 probability code
+ *                (ExpCast-FP8, Eq. 7), low-bit P V, and the block means added back inside
+ *                the recurrence (Eq. 6); epilogue O = s_V * A / l.
+ *   vc_attn      vc_prep followed by vc_attn_fwd.
+ *
+ * Conventions
+ *   - Every pointer is a DEVICE pointer unless the name says host; all must be 16-byte
+ *     aligned.  The caller owns every buffer; the library allocates no device memory.
+ *   - All work is enqueued on `stream` (a cudaStream_t passed as void*; NULL = the legacy
+ *     default stream).  No entry point synchronizes except vc_poll_status and
+ *     vc_attn_host.
+ *   - Errors are return codes only.  Argument errors are detected on the host before any
+ *     launch.  A device-side wait that exceeds its spin limit writes a code to the status
+ *     word at the start of the workspace and the kernel exits normally; vc_poll_status
+ *     reads it back as VC_ERR_TIMEOUT.
+ *   - Q, K, V are [B, H, N, d] bf16 with d contiguous; strides are given in elements
+ *     (0 = packed).  N tokens form a T x Hg x Wg grid in row-major (t, y, x) order.
+ *     O is [B, H, N, d] bf16, packed, in the original query order.
+ */
+#ifndef VC_ATTN_H_
+#define VC_ATTN_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  VC_OK = 0,
+  VC_ERR_INVALID_ARG = 1,   /* null pointer, bad size, misaligned pointer            */
+  VC_ERR_UNSUPPORTED = 2,   /* a combination this build does not implement           */
+  VC_ERR_WORKSPACE = 3,     /* reserved                                              */
+  VC_ERR_CUDA = 4,          /* a CUDA runtime/driver call failed                     */
+  VC_ERR_TIMEOUT = 5        /* a bounded device-side wait gave up                    */
+} vc_status;
+
+/* probability formats of the softmax stage (Sec. 3.3, App. A "Scope of ExpCast-FP8") */
+enum {
+  VC_P_DEFAULT = 0,         /* ExpCast-FP8 at 8 bits, NVFP4 at 4 bits                */
+  VC_P_EXPCAST_E4M3 = 1,    /* Eq. 7: one FMA, the byte viewed as E4M3               */
+  VC_P_EXP_E4M3 = 2,        /* exponentiate, then cast to E4M3 (Fig. 4a upper box)   */
+  VC_P_NVFP4 = 3            /* E2M1 under a per-16-key E4M3 microscale               */
+};
+
+/* stages of the chain that can be switched off (all on = the paper's method) */
+enum {
+  VC_FLAG_ROPE = 1,
+  VC_FLAG_HADAMARD = 2,
+  VC_FLAG_K_SMOOTH = 4,
+  VC_FLAG_V_SMOOTH = 8,
+  VC_FLAG_ALL = 15
+};
+
+typedef struct {
+  int32_t B, H, N, d;               /* d in {64, 128}; N >= 1                           */
+  int32_t grid_t, grid_h, grid_w;   /* grid_t * grid_h * grid_w == N                    */
+  int32_t bits;                     /* 8 or 4                                           */
+  int32_t p_format;                 /* VC_P_*                                           */
+  int32_t flags;                    /* VC_FLAG_*                                        */
+  float softmax_scale;              /* 0 => 1/sqrt(d)                                   */
+  float beta;                       /* ExpCast offset of Eq. 7; 0 => -0.35              */
+  int32_t rope_dim_t, rope_dim_h, rope_dim_w; /* channels per axis, even, sum == d;
+                                       all 0 => (d - 4*(d/6), 2*(d/6), 2*(d/6))         */
+  float rope_theta;                 /* 0 => 10000                                       */
+  int64_t stride_b, stride_h, stride_n;       /* of Q, K and V, in elements; 0 => packed */
+  int32_t heads_per_pass;           /* heads preprocessed per launch group (L2 reuse of
+                                       the second read of K and V); 0 => library default */
+  int32_t reserved;
+} vc_params;
+
+/* Device pointers into the quantized bundle written by vc_prep (N_pad = 128*ceil(N/128),
+ * nb = N_pad/128, BH = B*H).  8 bits: codes are E4M3 bytes.  4 bits: codes are E2M1
+ * nibbles, two per byte, the even index in the low nibble; micro are unsigned E4M3 bytes.
+ *   q_codes [BH][N_pad][d]      (4 bits: [BH][N_pad][d/2])   rows in query order
+ *   k_codes [BH][N_pad][d]      (4 bits: [BH][N_pad][d/2])   rows in permuted order
+ *   v_codes [BH][d][N_pad]      (4 bits: [BH][d][N_pad/2])   residual, channel-major
+ *   q_scale [BH][nb] fp32       (4 bits: [BH], the outer NVFP4 scale g_Q)
+ *   k_scale [BH][nb] fp32       (4 bits: [BH], g_K)
+ *   v_scale [BH][d]  fp32       (4 bits: all ones)
+ *   v_means [BH][nb][d] bf16    block means / v_scale (4 bits: unscaled), App. B
+ *   k_mean  [BH][d]  fp32       post-RoPE channel mean of K
+ *   q_micro [BH][N_pad][d/16], k_micro [BH][N_pad][d/16], v_micro [BH][d][N_pad/16]  (4 bits)
+ */
+typedef struct {
+  void *q_codes, *k_codes, *v_codes;
+  float *q_scale, *k_scale, *v_scale;
+  void *v_means;
+  float *k_mean;
+  void *q_micro, *k_micro, *v_micro;
+  size_t q_codes_bytes, k_codes_bytes, v_codes_bytes, q_scale_bytes, k_scale_bytes,
+         v_scale_bytes, v_means_bytes, k_mean_bytes, q_micro_bytes, k_micro_bytes,
+         v_micro_bytes;
+} vc_quant_ptrs;
+
+/* Sizes (bytes) of the caller-allocated quantized bundle and workspace; 0 on bad params. */
+size_t vc_quant_bytes(const vc_params *p);
+size_t vc_workspace_bytes(const vc_params *p);
+
+/* Preprocessing pass (Sec. 3.4, App. B).  perm: int32 [B][H][N], row t of the permuted
+ * K/V is row perm[t] of the input (Eq. 3), or NULL for the identity; it must be a
+ * permutation of [0, N) per (b, h) (not checked).  Writes `quant`; uses `workspace`
+ * (contents on entry irrelevant; the first 4 bytes become the status word). */
+vc_status vc_prep(const vc_params *p, const void *q, const void *k, const void *v,
+                  const int32_t *perm, void *quant, void *workspace, void *stream);
+
+/* Quantized attention forward (Eq. 1, Eq. 6, Eq. 7) from a bundle in vc_prep's layout.
+ * o: [B][H][N][d] bf16.  workspace as above. */
+vc_status vc_attn_fwd(const vc_params *p, const void *quant, void *o, void *workspace,
+                      void *stream);
+
+/* vc_prep followed by vc_attn_fwd on the same stream. */
+vc_status vc_attn(const vc_params *p, const void *q, const void *k, const void *v,
+                  const int32_t *perm, void *o, void *quant, void *workspace, void *stream);
+
+/* The same with HOST input/output buffers (pinned memory recommended): copies q, k, v
+ * (packed [B][H][N][d] bf16) and perm (or NULL) to the device staging buffers q_dev,
+ * k_dev, v_dev, perm_dev, runs vc_attn, copies o_dev to o_host and synchronizes the
+ * stream.  The staging buffers are caller-allocated device memory of the same sizes. */
+vc_status vc_attn_host(const vc_params *p, const void *q_host, const void *k_host,
+                       const void *v_host, const int32_t *perm_host, void *o_host,
+                       void *q_dev, void *k_dev, void *v_dev, int32_t *perm_dev, void *o_dev,
+                       void *quant, void *workspace, void *stream);
+
+/* Device pointers of the bundle's sections (for tests and for feeding a bundle in). */
+vc_status vc_quant_view(const vc_params *p, const void *quant, vc_quant_ptrs *out);
+
+/* Synchronizes `stream` and returns VC_ERR_TIMEOUT if a kernel recorded a timed-out wait,
+ * VC_ERR_CUDA on a CUDA error, VC_OK otherwise.  Clears the status word. */
+vc_status vc_poll_status(void *workspace, void *stream);
+
+/* Number of kernels this library has launched in this process (diagnostics). */
+uint64_t vc_launch_count(void);
+
+const char *vc_status_string(vc_status s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* VC_ATTN_H_ */

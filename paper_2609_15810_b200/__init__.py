@@ -1,0 +1,12 @@
+"""VC-Attention hot path for NVIDIA B200 (sm_100a): thin Python binding over libvc.so.
+
+Every step of the path runs in the library's CUDA kernels; this package only marshals
+arguments (PyTorch supplies device memory and streams).  Importing the binding raises if
+the library has not been built (``python -m paper_2609_15810_b200.build``): there is no
+CPU fallback.
+"""
+from .binding import (VcError, Params, QuantView, load_library, vc_attn, vc_attn_fwd,  # noqa: F401
+                      vc_attn_host, vc_launch_count, vc_poll_status, vc_prep, vc_quant_bytes,
+                      vc_quant_view, vc_status_string, vc_workspace_bytes,
+                      VC_FLAG_ALL, VC_FLAG_HADAMARD, VC_FLAG_K_SMOOTH, VC_FLAG_ROPE, VC_FLAG_V_SMOOTH,
+                      VC_P_DEFAULT, VC_P_EXPCAST_E4M3, VC_P_EXP_E4M3, VC_P_NVFP4)

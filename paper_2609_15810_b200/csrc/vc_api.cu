@@ -1,0 +1,257 @@
+// C-ABI entry points of libvc: argument validation, buffer layouts, launch sequencing.
+#include <atomic>
+#include <cstring>
+
+#include "vc_internal.h"
+
+namespace vc {
+
+static std::atomic<uint64_t> g_launches{0};
+void count_launches(int n) { g_launches.fetch_add((uint64_t)n, std::memory_order_relaxed); }
+
+static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+vc_status resolve(const vc_params* p, Problem* out) {
+  if (!p || !out) return VC_ERR_INVALID_ARG;
+  Problem pr{};
+  pr.B = p->B; pr.H = p->H; pr.N = p->N; pr.d = p->d;
+  if (pr.B < 1 || pr.H < 1 || pr.N < 1) return VC_ERR_INVALID_ARG;
+  if ((int64_t)pr.B * pr.H > (1 << 20) || pr.N > (1 << 22)) return VC_ERR_INVALID_ARG;
+  if (pr.d != 64 && pr.d != 128) return VC_ERR_INVALID_ARG;
+  pr.BH = pr.B * pr.H;
+  pr.grid_t = p->grid_t; pr.grid_h = p->grid_h; pr.grid_w = p->grid_w;
+  if (pr.grid_t < 1 || pr.grid_h < 1 || pr.grid_w < 1) return VC_ERR_INVALID_ARG;
+  if ((int64_t)pr.grid_t * pr.grid_h * pr.grid_w != pr.N) return VC_ERR_INVALID_ARG;
+  pr.bits = p->bits;
+  if (pr.bits != 8 && pr.bits != 4) return VC_ERR_INVALID_ARG;
+  pr.p_format = p->p_format;
+  if (pr.p_format == VC_P_DEFAULT) pr.p_format = pr.bits == 8 ? VC_P_EXPCAST_E4M3 : VC_P_NVFP4;
+  if (pr.p_format < VC_P_EXPCAST_E4M3 || pr.p_format > VC_P_NVFP4) return VC_ERR_INVALID_ARG;
+  if (pr.bits == 8 && pr.p_format == VC_P_NVFP4) return VC_ERR_UNSUPPORTED;
+  if (pr.bits == 4 && pr.p_format != VC_P_NVFP4) return VC_ERR_UNSUPPORTED;
+  pr.flags = p->flags;
+  if (pr.flags & ~VC_FLAG_ALL) return VC_ERR_INVALID_ARG;
+  pr.softmax_scale = p->softmax_scale != 0.f ? p->softmax_scale : 1.0f / sqrtf((float)pr.d);
+  if (!(pr.softmax_scale > 0.f)) return VC_ERR_INVALID_ARG;
+  pr.beta = p->beta != 0.f ? p->beta : -0.35f;
+  pr.rope_theta = p->rope_theta != 0.f ? p->rope_theta : 10000.0f;
+  if (p->rope_dim_t == 0 && p->rope_dim_h == 0 && p->rope_dim_w == 0) {
+    int s = 2 * (pr.d / 6);
+    pr.rope_dim[0] = pr.d - 2 * s; pr.rope_dim[1] = s; pr.rope_dim[2] = s;
+  } else {
+    pr.rope_dim[0] = p->rope_dim_t; pr.rope_dim[1] = p->rope_dim_h; pr.rope_dim[2] = p->rope_dim_w;
+  }
+  int sum = 0;
+  for (int a = 0; a < 3; ++a) {
+    if (pr.rope_dim[a] < 0 || (pr.rope_dim[a] & 1)) return VC_ERR_INVALID_ARG;
+    sum += pr.rope_dim[a];
+  }
+  if (sum != pr.d) return VC_ERR_INVALID_ARG;
+  pr.stride_n = p->stride_n ? p->stride_n : pr.d;
+  pr.stride_h = p->stride_h ? p->stride_h : (int64_t)pr.N * pr.d;
+  pr.stride_b = p->stride_b ? p->stride_b : (int64_t)pr.H * pr.N * pr.d;
+  if (pr.stride_n < pr.d || (pr.stride_n % 8) || (pr.stride_h % 8) || (pr.stride_b % 8))
+    return VC_ERR_INVALID_ARG;   // rows are read with 16-byte vector loads
+  pr.n_pad = kBlock * ((pr.N + kBlock - 1) / kBlock);
+  pr.nb = pr.n_pad / kBlock;
+  pr.heads_per_pass = p->heads_per_pass > 0 ? p->heads_per_pass : 0;
+  *out = pr;
+  return VC_OK;
+}
+
+QuantLayout quant_layout(const Problem& pr) {
+  QuantLayout L{};
+  const size_t BH = pr.BH, np_ = pr.n_pad, d = pr.d, nb = pr.nb;
+  const bool four = pr.bits == 4;
+  L.q_codes_bytes = four ? BH * np_ * d / 2 : BH * np_ * d;
+  L.k_codes_bytes = L.q_codes_bytes;
+  L.v_codes_bytes = L.q_codes_bytes;
+  L.q_scale_bytes = four ? BH * 4 : BH * nb * 4;
+  L.k_scale_bytes = L.q_scale_bytes;
+  L.v_scale_bytes = BH * d * 4;
+  L.v_means_bytes = BH * nb * d * 2;
+  L.k_mean_bytes = BH * d * 4;
+  L.q_micro_bytes = four ? BH * np_ * d / 16 : 0;
+  L.k_micro_bytes = L.q_micro_bytes;
+  L.v_micro_bytes = L.q_micro_bytes;
+  size_t off = 0;
+  auto place = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 1024); return o; };
+  L.q_codes = place(L.q_codes_bytes);
+  L.k_codes = place(L.k_codes_bytes);
+  L.v_codes = place(L.v_codes_bytes);
+  L.q_scale = place(L.q_scale_bytes);
+  L.k_scale = place(L.k_scale_bytes);
+  L.v_scale = place(L.v_scale_bytes);
+  L.v_means = place(L.v_means_bytes);
+  L.k_mean = place(L.k_mean_bytes);
+  L.q_micro = place(L.q_micro_bytes);
+  L.k_micro = place(L.k_micro_bytes);
+  L.v_micro = place(L.v_micro_bytes);
+  L.total = off;
+  return L;
+}
+
+WorkLayout work_layout(const Problem& pr) {
+  WorkLayout W{};
+  const size_t BH = pr.BH, d = pr.d, nb = pr.nb;
+  const int len[3] = {pr.grid_t, pr.grid_h, pr.grid_w};
+  int e = 0;
+  for (int a = 0; a < 3; ++a) { W.rope_off[a] = e; e += len[a] * (pr.rope_dim[a] / 2); }
+  W.rope_entries = e;
+  size_t off = 0;
+  auto place = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 1024); return o; };
+  W.status = place(256);
+  W.rope = place((size_t)e * 8);
+  W.k_part = place(BH * nb * d * 4);
+  W.v_mu = place(BH * nb * d * 4);
+  W.amax_bytes = BH * d * 4 + 2 * BH * 4;
+  W.amax = place(W.amax_bytes);
+  W.total = off;
+  return W;
+}
+
+static bool misaligned(const void* p) { return ((uintptr_t)p & 15) != 0; }
+
+}  // namespace vc
+
+using namespace vc;
+
+extern "C" {
+
+size_t vc_quant_bytes(const vc_params* p) {
+  Problem pr;
+  if (resolve(p, &pr) != VC_OK) return 0;
+  return quant_layout(pr).total;
+}
+
+size_t vc_workspace_bytes(const vc_params* p) {
+  Problem pr;
+  if (resolve(p, &pr) != VC_OK) return 0;
+  return work_layout(pr).total;
+}
+
+vc_status vc_prep(const vc_params* p, const void* q, const void* k, const void* v,
+                  const int32_t* perm, void* quant, void* workspace, void* stream) {
+  Problem pr;
+  vc_status st = resolve(p, &pr);
+  if (st != VC_OK) return st;
+  if (!q || !k || !v || !quant || !workspace) return VC_ERR_INVALID_ARG;
+  if (misaligned(q) || misaligned(k) || misaligned(v) || misaligned(quant) ||
+      misaligned(workspace) || (perm && misaligned(perm)))
+    return VC_ERR_INVALID_ARG;
+  QuantLayout ql = quant_layout(pr);
+  WorkLayout wl = work_layout(pr);
+  cudaError_t e = launch_prep(pr, ql, wl, q, k, v, perm, (uint8_t*)quant, (uint8_t*)workspace,
+                              (cudaStream_t)stream);
+  return e == cudaSuccess ? VC_OK : VC_ERR_CUDA;
+}
+
+vc_status vc_attn_fwd(const vc_params* p, const void* quant, void* o, void* workspace,
+                      void* stream) {
+  Problem pr;
+  vc_status st = resolve(p, &pr);
+  if (st != VC_OK) return st;
+  if (!quant || !o || !workspace) return VC_ERR_INVALID_ARG;
+  if (misaligned(quant) || misaligned(o) || misaligned(workspace)) return VC_ERR_INVALID_ARG;
+  QuantLayout ql = quant_layout(pr);
+  WorkLayout wl = work_layout(pr);
+  cudaError_t e = launch_attn_fwd(pr, ql, wl, (const uint8_t*)quant, o, (uint8_t*)workspace,
+                                  (cudaStream_t)stream);
+  if (e == cudaErrorNotSupported) return VC_ERR_UNSUPPORTED;
+  return e == cudaSuccess ? VC_OK : VC_ERR_CUDA;
+}
+
+vc_status vc_attn(const vc_params* p, const void* q, const void* k, const void* v,
+                  const int32_t* perm, void* o, void* quant, void* workspace, void* stream) {
+  vc_status st = vc_prep(p, q, k, v, perm, quant, workspace, stream);
+  if (st != VC_OK) return st;
+  return vc_attn_fwd(p, quant, o, workspace, stream);
+}
+
+vc_status vc_attn_host(const vc_params* p, const void* q_host, const void* k_host,
+                       const void* v_host, const int32_t* perm_host, void* o_host,
+                       void* q_dev, void* k_dev, void* v_dev, int32_t* perm_dev, void* o_dev,
+                       void* quant, void* workspace, void* stream) {
+  Problem pr;
+  vc_status st = resolve(p, &pr);
+  if (st != VC_OK) return st;
+  if (!q_host || !k_host || !v_host || !o_host || !q_dev || !k_dev || !v_dev || !o_dev)
+    return VC_ERR_INVALID_ARG;
+  if (perm_host && !perm_dev) return VC_ERR_INVALID_ARG;
+  if (p->stride_b || p->stride_h || p->stride_n) {
+    if (pr.stride_n != pr.d || pr.stride_h != (int64_t)pr.N * pr.d ||
+        pr.stride_b != (int64_t)pr.H * pr.N * pr.d)
+      return VC_ERR_INVALID_ARG;   // host buffers are packed
+  }
+  cudaStream_t s = (cudaStream_t)stream;
+  const size_t bytes = (size_t)pr.BH * pr.N * pr.d * 2;
+  if (cudaMemcpyAsync(q_dev, q_host, bytes, cudaMemcpyHostToDevice, s) != cudaSuccess ||
+      cudaMemcpyAsync(k_dev, k_host, bytes, cudaMemcpyHostToDevice, s) != cudaSuccess ||
+      cudaMemcpyAsync(v_dev, v_host, bytes, cudaMemcpyHostToDevice, s) != cudaSuccess)
+    return VC_ERR_CUDA;
+  if (perm_host &&
+      cudaMemcpyAsync(perm_dev, perm_host, (size_t)pr.BH * pr.N * 4, cudaMemcpyHostToDevice, s) !=
+          cudaSuccess)
+    return VC_ERR_CUDA;
+  st = vc_attn(p, q_dev, k_dev, v_dev, perm_host ? perm_dev : nullptr, o_dev, quant, workspace,
+               stream);
+  if (st != VC_OK) return st;
+  if (cudaMemcpyAsync(o_host, o_dev, bytes, cudaMemcpyDeviceToHost, s) != cudaSuccess)
+    return VC_ERR_CUDA;
+  return cudaStreamSynchronize(s) == cudaSuccess ? VC_OK : VC_ERR_CUDA;
+}
+
+vc_status vc_quant_view(const vc_params* p, const void* quant, vc_quant_ptrs* out) {
+  Problem pr;
+  vc_status st = resolve(p, &pr);
+  if (st != VC_OK) return st;
+  if (!quant || !out) return VC_ERR_INVALID_ARG;
+  QuantLayout L = quant_layout(pr);
+  uint8_t* b = (uint8_t*)quant;
+  std::memset(out, 0, sizeof(*out));
+  out->q_codes = b + L.q_codes; out->k_codes = b + L.k_codes; out->v_codes = b + L.v_codes;
+  out->q_scale = (float*)(b + L.q_scale); out->k_scale = (float*)(b + L.k_scale);
+  out->v_scale = (float*)(b + L.v_scale);
+  out->v_means = b + L.v_means;
+  out->k_mean = (float*)(b + L.k_mean);
+  if (pr.bits == 4) {
+    out->q_micro = b + L.q_micro; out->k_micro = b + L.k_micro; out->v_micro = b + L.v_micro;
+  }
+  out->q_codes_bytes = L.q_codes_bytes; out->k_codes_bytes = L.k_codes_bytes;
+  out->v_codes_bytes = L.v_codes_bytes; out->q_scale_bytes = L.q_scale_bytes;
+  out->k_scale_bytes = L.k_scale_bytes; out->v_scale_bytes = L.v_scale_bytes;
+  out->v_means_bytes = L.v_means_bytes; out->k_mean_bytes = L.k_mean_bytes;
+  out->q_micro_bytes = L.q_micro_bytes; out->k_micro_bytes = L.k_micro_bytes;
+  out->v_micro_bytes = L.v_micro_bytes;
+  return VC_OK;
+}
+
+vc_status vc_poll_status(void* workspace, void* stream) {
+  if (!workspace) return VC_ERR_INVALID_ARG;
+  uint32_t word = 0;
+  cudaStream_t s = (cudaStream_t)stream;
+  if (cudaMemcpyAsync(&word, workspace, 4, cudaMemcpyDeviceToHost, s) != cudaSuccess) return VC_ERR_CUDA;
+  if (cudaStreamSynchronize(s) != cudaSuccess) return VC_ERR_CUDA;
+  if (word != 0) {
+    cudaMemsetAsync(workspace, 0, 4, s);
+    cudaStreamSynchronize(s);
+    return VC_ERR_TIMEOUT;
+  }
+  return VC_OK;
+}
+
+uint64_t vc_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+const char* vc_status_string(vc_status s) {
+  switch (s) {
+    case VC_OK: return "ok";
+    case VC_ERR_INVALID_ARG: return "invalid argument";
+    case VC_ERR_UNSUPPORTED: return "unsupported configuration";
+    case VC_ERR_WORKSPACE: return "workspace error";
+    case VC_ERR_CUDA: return "CUDA error";
+    case VC_ERR_TIMEOUT: return "device-side wait timed out";
+  }
+  return "unknown status";
+}
+
+}  // extern "C"

@@ -1,0 +1,60 @@
+// Internal declarations shared by the translation units of libvc (not part of the ABI).
+#pragma once
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "vc_attn.h"
+
+namespace vc {
+
+constexpr int kBlock = 128;   // B_v of Eq. 4 = row block of the Q/K scales = MMA tile
+
+// Resolved parameters: defaults filled in, derived sizes added.
+struct Problem {
+  int B, H, N, d, BH;
+  int grid_t, grid_h, grid_w;
+  int bits, p_format, flags;
+  float softmax_scale, beta, rope_theta;
+  int rope_dim[3];
+  int64_t stride_b, stride_h, stride_n;
+  int n_pad, nb;
+  int heads_per_pass;
+};
+
+// Byte offsets of the sections of the quantized bundle.
+struct QuantLayout {
+  size_t q_codes, k_codes, v_codes, q_scale, k_scale, v_scale, v_means, k_mean;
+  size_t q_micro, k_micro, v_micro;
+  size_t q_codes_bytes, k_codes_bytes, v_codes_bytes, q_scale_bytes, k_scale_bytes,
+      v_scale_bytes, v_means_bytes, k_mean_bytes, q_micro_bytes, k_micro_bytes, v_micro_bytes;
+  size_t total;
+};
+
+// Byte offsets of the sections of the workspace.
+struct WorkLayout {
+  size_t status;     // uint32 status word (+ padding)
+  size_t rope;       // float2 (cos, sin) compact per-axis tables
+  size_t k_part;     // fp32 [BH][nb][d] per-block column sums of RoPE(K)
+  size_t v_mu;       // fp32 [BH][nb][d] block means of the gathered V
+  size_t amax;       // uint32 [BH][d] residual amax bits (8-bit V) then [2][BH] Q/K head amax (4-bit)
+  size_t amax_bytes;
+  size_t total;
+  int rope_off[3];   // entry offset of each axis table
+  int rope_entries;
+};
+
+vc_status resolve(const vc_params* p, Problem* out);
+QuantLayout quant_layout(const Problem& pr);
+WorkLayout work_layout(const Problem& pr);
+
+// Launchers (each returns the CUDA error of its launches; all asynchronous on `stream`).
+cudaError_t launch_prep(const Problem& pr, const QuantLayout& ql, const WorkLayout& wl,
+                        const void* q, const void* k, const void* v, const int32_t* perm,
+                        uint8_t* quant, uint8_t* work, cudaStream_t stream);
+cudaError_t launch_attn_fwd(const Problem& pr, const QuantLayout& ql, const WorkLayout& wl,
+                            const uint8_t* quant, void* o, uint8_t* work, cudaStream_t stream);
+
+void count_launches(int n);
+
+}  // namespace vc

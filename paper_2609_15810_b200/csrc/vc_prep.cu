@@ -1,0 +1,581 @@
+// Fused preprocessing pass of VC-Attention for sm_100a (Sec. 3.4 "Fused preprocessing",
+// App. B): every operand is read as bf16 with 16-byte vector loads and leaves as low-bit
+// codes plus scales; no rotated / permuted / centered high-precision tensor reaches HBM.
+//
+//   Q : RoPE -> Hadamard (registers + warp shuffles) -> per-128-row scale -> codes
+//   K : RoPE -> column sums (stats launch) ... gather by pi -> RoPE at the source position
+//       -> subtract channel mean -> Hadamard -> scale -> codes
+//   V : gather by pi -> block mean (Eq. 4) and residual amax (stats launch) ...
+//       gather -> residual -> codes written channel-major, block means beside them
+//
+// The two global reductions (K channel mean over all tokens, per-channel amax of the V
+// residual over all tokens) force a statistics launch before the quantizing launch; heads
+// are processed in groups so that the second read of K and V can hit L2.
+#include <cuda_bf16.h>
+#include <cuda_fp4.h>
+#include <cuda_fp8.h>
+
+#include "vc_internal.h"
+
+namespace vc {
+namespace {
+
+constexpr int kThreads = 256;
+
+struct RopeDesc {
+  int pair_start[3];   // first channel pair of each axis
+  int pairs[3];        // channel pairs per axis
+  int off[3];          // entry offset of each axis table
+  int len[3];          // positions per axis
+  int entries;
+  int grid_h, grid_w;
+  unsigned long long mul_w, mul_h;   // ceil(2^40 / divisor)
+};
+
+struct PrepArgs {
+  const __nv_bfloat16 *q, *k, *v;
+  const int32_t* perm;
+  int64_t stride_b, stride_h, stride_n;
+  int H, N, n_pad, nb, bh0, flags, rope_in_smem;
+  uint8_t *q_codes, *k_codes, *v_codes, *q_micro, *k_micro, *v_micro;
+  float *q_scale, *k_scale, *v_scale, *k_mean;
+  __nv_bfloat16* v_means;
+  const float2* rope;
+  float *k_part, *v_mu;
+  unsigned int *v_amax, *qk_amax;   // qk_amax: [2][BH]
+  int BH;
+  RopeDesc rd;
+};
+
+__device__ __forceinline__ unsigned int div40(unsigned int x, unsigned long long mul) {
+  return (unsigned int)(((unsigned long long)x * mul) >> 40);
+}
+
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+  for (int s = 16; s > 0; s >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, s));
+  return v;
+}
+
+__device__ __forceinline__ float e4m3_to_float(unsigned int code) {
+  __half_raw h = __nv_cvt_fp8_to_halfraw((__nv_fp8_storage_t)code, __NV_E4M3);
+  return __half2float(__half(h));
+}
+
+// ---------------------------------------------------------------------------------------
+// RoPE tables: per axis a, entry [pos][i] = (cos, sin)(pos * theta^(-2 i / d_a)), evaluated
+// in double and rounded once to fp32.
+__global__ void rope_table_kernel(float2* tab, RopeDesc rd, double theta) {
+  int e = blockIdx.x * blockDim.x + threadIdx.x;
+  if (e >= rd.entries) return;
+  int a = e >= rd.off[2] ? 2 : (e >= rd.off[1] ? 1 : 0);
+  int r = e - rd.off[a];
+  int pos = r / rd.pairs[a];
+  int i = r - pos * rd.pairs[a];
+  double freq = pow(theta, -2.0 * (double)i / (double)(2 * rd.pairs[a]));
+  double phi = (double)pos * freq;
+  tab[e] = make_float2((float)cos(phi), (float)sin(phi));
+}
+
+// ---------------------------------------------------------------------------------------
+// Q / K body.  A CTA owns one block of 128 rows; a lane owns 8 consecutive channels of
+// D/16 consecutive rows, so RoPE pairs and 3 Hadamard stages stay in registers and the
+// remaining log2(D/8) stages are xor-shuffles inside the D/8 lanes that share a row.
+enum { kStageColSum = 0, kStageAmax = 1, kStageQuant8 = 2, kStageQuant4 = 3 };
+
+template <int D, int TENSOR /*0 = Q, 1 = K*/, int STAGE>
+__device__ __forceinline__ void qk_body(const PrepArgs& a, unsigned char* smem) {
+  constexpr int LPR = D / 8;         // lanes per row
+  constexpr int RPL = LPR / 2;       // rows per lane (a warp covers 16 rows)
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int lr = lane % LPR, hb = lane / LPR;
+  const int blk = blockIdx.x, bh = a.bh0 + blockIdx.y;
+  const int b = bh / a.H, h = bh - b * a.H;
+  const __nv_bfloat16* base = (TENSOR == 0 ? a.q : a.k) + b * a.stride_b + h * a.stride_h;
+  const bool do_rope = a.flags & VC_FLAG_ROPE;
+  const bool do_had = (a.flags & VC_FLAG_HADAMARD) && STAGE != kStageColSum;
+  const bool gather = TENSOR == 1 && a.perm != nullptr && STAGE >= kStageQuant8;
+
+  // RoPE table -> shared memory (or read through L2 when it does not fit)
+  const float2* tab = a.rope;
+  float* red = reinterpret_cast<float*>(smem);            // [8][D] floats of scratch
+  if (do_rope && a.rope_in_smem) {
+    float2* st = reinterpret_cast<float2*>(smem + 8 * D * 4);
+    for (int e = tid; e < a.rd.entries; e += kThreads) st[e] = a.rope[e];
+    tab = st;
+    __syncthreads();
+  }
+  // per-lane constants of the 4 channel pairs it owns
+  int p_axis[4], p_idx[4];
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    int p = 4 * lr + j;
+    int ax = p >= a.rd.pair_start[2] ? 2 : (p >= a.rd.pair_start[1] ? 1 : 0);
+    p_axis[j] = ax;
+    p_idx[j] = a.rd.off[ax] + (p - a.rd.pair_start[ax]);
+  }
+  float kmean[8];
+#pragma unroll
+  for (int c = 0; c < 8; ++c) kmean[c] = 0.f;
+  if (TENSOR == 1 && STAGE != kStageColSum && (a.flags & VC_FLAG_K_SMOOTH)) {
+#pragma unroll
+    for (int c = 0; c < 8; ++c) kmean[c] = a.k_mean[(size_t)bh * D + 8 * lr + c];
+  }
+
+  float x[RPL][8];
+#pragma unroll
+  for (int i = 0; i < RPL; ++i) {
+    const int row = 16 * warp + RPL * hb + i;
+    const int t = blk * kBlock + row;
+    const bool valid = t < a.N;
+    int src = t;
+    if (gather && valid) src = a.perm[(size_t)bh * a.N + t];
+    uint4 raw = make_uint4(0, 0, 0, 0);
+    if (valid) raw = __ldg(reinterpret_cast<const uint4*>(base + (int64_t)src * a.stride_n + 8 * lr));
+    const unsigned int w[4] = {raw.x, raw.y, raw.z, raw.w};
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      x[i][2 * j] = __uint_as_float(w[j] << 16);
+      x[i][2 * j + 1] = __uint_as_float(w[j] & 0xffff0000u);
+    }
+    if (do_rope && valid) {
+      const unsigned int q1 = div40((unsigned)src, a.rd.mul_w);
+      const unsigned int tx = src - q1 * a.rd.grid_w;
+      const unsigned int tt = div40(q1, a.rd.mul_h);
+      const unsigned int ty = q1 - tt * a.rd.grid_h;
+      const unsigned int pos[3] = {tt, ty, tx};
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const int ax = p_axis[j];
+        const float2 cs = tab[p_idx[j] + (int)pos[ax] * a.rd.pairs[ax]];
+        const float x0 = x[i][2 * j], x1 = x[i][2 * j + 1];
+        x[i][2 * j] = x0 * cs.x - x1 * cs.y;
+        x[i][2 * j + 1] = x0 * cs.y + x1 * cs.x;
+      }
+    }
+    if (TENSOR == 1 && STAGE != kStageColSum && valid) {
+#pragma unroll
+      for (int c = 0; c < 8; ++c) x[i][c] -= kmean[c];
+    }
+    if (do_had) {
+      // in-register stages (channel bits 0..2)
+#pragma unroll
+      for (int s = 1; s < 8; s <<= 1) {
+#pragma unroll
+        for (int c = 0; c < 8; ++c) {
+          if (!(c & s)) {
+            const float u = x[i][c], v = x[i][c | s];
+            x[i][c] = u + v;
+            x[i][c | s] = u - v;
+          }
+        }
+      }
+      // cross-lane stages (channel bits 3..)
+#pragma unroll
+      for (int s = 1; s < LPR; s <<= 1) {
+        const bool upper = lr & s;
+#pragma unroll
+        for (int c = 0; c < 8; ++c) {
+          const float other = __shfl_xor_sync(0xffffffffu, x[i][c], s);
+          x[i][c] = upper ? other - x[i][c] : x[i][c] + other;
+        }
+      }
+      const float rs = D == 128 ? 0.08838834764831845f : 0.125f;   // 1/sqrt(D)
+#pragma unroll
+      for (int c = 0; c < 8; ++c) x[i][c] *= rs;
+    }
+  }
+
+  if constexpr (STAGE == kStageColSum) {
+    float s[8];
+#pragma unroll
+    for (int c = 0; c < 8; ++c) {
+      s[c] = 0.f;
+#pragma unroll
+      for (int i = 0; i < RPL; ++i) s[c] += x[i][c];
+#pragma unroll
+      for (int m = LPR; m < 32; m <<= 1) s[c] += __shfl_xor_sync(0xffffffffu, s[c], m);
+    }
+    if (hb == 0) {
+#pragma unroll
+      for (int c = 0; c < 8; ++c) red[warp * D + 8 * lr + c] = s[c];
+    }
+    __syncthreads();
+    if (tid < D) {
+      float t = 0.f;
+#pragma unroll
+      for (int w8 = 0; w8 < 8; ++w8) t += red[w8 * D + tid];
+      a.k_part[((size_t)bh * a.nb + blk) * D + tid] = t;
+    }
+    return;
+  }
+
+  // amax of the block (and of the head for the 4-bit outer scale)
+  float amax = 0.f;
+  if constexpr (STAGE != kStageQuant4) {
+#pragma unroll
+    for (int i = 0; i < RPL; ++i)
+#pragma unroll
+      for (int c = 0; c < 8; ++c) amax = fmaxf(amax, fabsf(x[i][c]));
+    amax = warp_max(amax);
+    __syncthreads();
+    if (lane == 0) red[warp] = amax;
+    __syncthreads();
+    amax = red[0];
+#pragma unroll
+    for (int w8 = 1; w8 < 8; ++w8) amax = fmaxf(amax, red[w8]);
+  }
+  if constexpr (STAGE == kStageAmax) {
+    if (tid == 0) atomicMax(&a.qk_amax[TENSOR * a.BH + bh], __float_as_uint(amax));
+    return;
+  }
+
+  if constexpr (STAGE == kStageQuant8) {
+    const float inv = amax > 0.f ? 448.0f / amax : 0.f;
+    if (tid == 0) (TENSOR == 0 ? a.q_scale : a.k_scale)[(size_t)bh * a.nb + blk] = amax > 0.f ? amax / 448.0f : 1.0f;
+    uint8_t* dst = (TENSOR == 0 ? a.q_codes : a.k_codes) + ((size_t)bh * a.n_pad + (size_t)blk * kBlock) * D;
+#pragma unroll
+    for (int i = 0; i < RPL; ++i) {
+      const int row = 16 * warp + RPL * hb + i;
+      unsigned int w[2];
+#pragma unroll
+      for (int j = 0; j < 2; ++j) {
+        const unsigned int lo = __nv_cvt_float2_to_fp8x2(make_float2(x[i][4 * j] * inv, x[i][4 * j + 1] * inv), __NV_SATFINITE, __NV_E4M3);
+        const unsigned int hi = __nv_cvt_float2_to_fp8x2(make_float2(x[i][4 * j + 2] * inv, x[i][4 * j + 3] * inv), __NV_SATFINITE, __NV_E4M3);
+        w[j] = lo | (hi << 16);
+      }
+      *reinterpret_cast<uint2*>(dst + (size_t)row * D + 8 * lr) = make_uint2(w[0], w[1]);
+    }
+  }
+
+  if constexpr (STAGE == kStageQuant4) {
+    // NVFP4: outer scale g per (b, h), microscale per token per 16 channels (= 2 lanes)
+    const float g = (TENSOR == 0 ? a.q_scale : a.k_scale)[bh];
+    const float inv6 = 1.0f / (6.0f * g);
+    uint8_t* dst = (TENSOR == 0 ? a.q_codes : a.k_codes) + ((size_t)bh * a.n_pad + (size_t)blk * kBlock) * (D / 2);
+    uint8_t* mdst = (TENSOR == 0 ? a.q_micro : a.k_micro) + ((size_t)bh * a.n_pad + (size_t)blk * kBlock) * (D / 16);
+#pragma unroll
+    for (int i = 0; i < RPL; ++i) {
+      const int row = 16 * warp + RPL * hb + i;
+      float m = 0.f;
+#pragma unroll
+      for (int c = 0; c < 8; ++c) m = fmaxf(m, fabsf(x[i][c]));
+      m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 1));
+      const unsigned int sb = __nv_cvt_float_to_fp8(m * inv6, __NV_SATFINITE, __NV_E4M3);
+      const float sdec = e4m3_to_float(sb);
+      const float rcp = sdec > 0.f ? 1.0f / (g * sdec) : 0.f;
+      unsigned int packed = 0;
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const unsigned int two = __nv_cvt_float2_to_fp4x2(make_float2(x[i][2 * j] * rcp, x[i][2 * j + 1] * rcp), __NV_E2M1, cudaRoundNearest);
+        packed |= (two & 0xffu) << (8 * j);
+      }
+      if (!(sdec > 0.f)) packed = 0;
+      *reinterpret_cast<unsigned int*>(dst + (size_t)row * (D / 2) + 4 * lr) = packed;
+      if (!(lr & 1)) mdst[(size_t)row * (D / 16) + (lr >> 1)] = (uint8_t)sb;
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------------------
+// V body.  The gathered 128 x D block is staged in shared memory with coalesced 16-byte
+// loads; a thread then owns one channel pair and 128 / (256 / (D/2)) consecutive tokens,
+// so block means and the channel-major (token-contiguous) code rows need no transposition.
+enum { kVStats = 0, kVQuant8 = 1, kVQuant4 = 2 };
+
+template <int D, int STAGE>
+__device__ __forceinline__ void v_body(const PrepArgs& a, unsigned char* smem) {
+  constexpr int LPR = D / 8;
+  constexpr int CP = D / 2;             // channel pairs
+  constexpr int TG = kThreads / CP;     // token groups
+  constexpr int TPG = kBlock / TG;      // tokens per thread
+  const int tid = threadIdx.x;
+  const int blk = blockIdx.x, bh = a.bh0 + blockIdx.y;
+  const int b = bh / a.H, h = bh - b * a.H;
+  const __nv_bfloat16* base = a.v + b * a.stride_b + h * a.stride_h;
+  uint4* tile4 = reinterpret_cast<uint4*>(smem);                       // [128][D] bf16
+  float* red = reinterpret_cast<float*>(smem + kBlock * D * 2);        // [TG][D]
+
+  for (int idx = tid; idx < kBlock * LPR; idx += kThreads) {
+    const int row = idx / LPR, ch = idx - row * LPR;
+    const int t = blk * kBlock + row;
+    uint4 val = make_uint4(0, 0, 0, 0);
+    if (t < a.N) {
+      const int src = a.perm ? a.perm[(size_t)bh * a.N + t] : t;
+      val = __ldg(reinterpret_cast<const uint4*>(base + (int64_t)src * a.stride_n + 8 * ch));
+    }
+    tile4[idx] = val;
+  }
+  __syncthreads();
+
+  const int cp = tid % CP, tg = tid / CP;
+  const int n_valid = min(kBlock, a.N - blk * kBlock);
+  const unsigned int* tile32 = reinterpret_cast<const unsigned int*>(smem);
+  float v0[TPG], v1[TPG];
+#pragma unroll
+  for (int i = 0; i < TPG; ++i) {
+    const unsigned int w = tile32[(tg * TPG + i) * CP + cp];
+    v0[i] = __uint_as_float(w << 16);
+    v1[i] = __uint_as_float(w & 0xffff0000u);
+  }
+  const bool smooth = a.flags & VC_FLAG_V_SMOOTH;
+  const size_t mu_at = ((size_t)bh * a.nb + blk) * D + 2 * cp;
+  float mu0 = 0.f, mu1 = 0.f;
+
+  if constexpr (STAGE == kVStats) {
+    if (smooth) {
+      float s0 = 0.f, s1 = 0.f;
+#pragma unroll
+      for (int i = 0; i < TPG; ++i) { s0 += v0[i]; s1 += v1[i]; }
+      red[tg * D + 2 * cp] = s0;
+      red[tg * D + 2 * cp + 1] = s1;
+      __syncthreads();
+      s0 = 0.f; s1 = 0.f;
+#pragma unroll
+      for (int g = 0; g < TG; ++g) { s0 += red[g * D + 2 * cp]; s1 += red[g * D + 2 * cp + 1]; }
+      mu0 = s0 / (float)n_valid;
+      mu1 = s1 / (float)n_valid;
+      __syncthreads();
+    }
+    if (tg == 0) { a.v_mu[mu_at] = mu0; a.v_mu[mu_at + 1] = mu1; }
+    float m0 = 0.f, m1 = 0.f;
+#pragma unroll
+    for (int i = 0; i < TPG; ++i) {
+      if (tg * TPG + i < n_valid) {
+        m0 = fmaxf(m0, fabsf(v0[i] - mu0));
+        m1 = fmaxf(m1, fabsf(v1[i] - mu1));
+      }
+    }
+    red[tg * D + 2 * cp] = m0;
+    red[tg * D + 2 * cp + 1] = m1;
+    __syncthreads();
+    if (tg == 0) {
+#pragma unroll
+      for (int g = 1; g < TG; ++g) { m0 = fmaxf(m0, red[g * D + 2 * cp]); m1 = fmaxf(m1, red[g * D + 2 * cp + 1]); }
+      atomicMax(&a.v_amax[(size_t)bh * D + 2 * cp], __float_as_uint(m0));
+      atomicMax(&a.v_amax[(size_t)bh * D + 2 * cp + 1], __float_as_uint(m1));
+    }
+    return;
+  }
+
+  mu0 = a.v_mu[mu_at];
+  mu1 = a.v_mu[mu_at + 1];
+  float r0[TPG], r1[TPG];
+#pragma unroll
+  for (int i = 0; i < TPG; ++i) {
+    const bool valid = tg * TPG + i < n_valid;
+    r0[i] = valid ? v0[i] - mu0 : 0.f;
+    r1[i] = valid ? v1[i] - mu1 : 0.f;
+  }
+  const size_t tok0 = (size_t)blk * kBlock + tg * TPG;
+
+  if constexpr (STAGE == kVQuant8) {
+    const float am0 = __uint_as_float(a.v_amax[(size_t)bh * D + 2 * cp]);
+    const float am1 = __uint_as_float(a.v_amax[(size_t)bh * D + 2 * cp + 1]);
+    const float inv0 = am0 > 0.f ? 448.0f / am0 : 0.f, inv1 = am1 > 0.f ? 448.0f / am1 : 0.f;
+    unsigned int w0[TPG / 4], w1[TPG / 4];
+#pragma unroll
+    for (int j = 0; j < TPG / 4; ++j) {
+      unsigned int lo = __nv_cvt_float2_to_fp8x2(make_float2(r0[4 * j] * inv0, r0[4 * j + 1] * inv0), __NV_SATFINITE, __NV_E4M3);
+      unsigned int hi = __nv_cvt_float2_to_fp8x2(make_float2(r0[4 * j + 2] * inv0, r0[4 * j + 3] * inv0), __NV_SATFINITE, __NV_E4M3);
+      w0[j] = lo | (hi << 16);
+      lo = __nv_cvt_float2_to_fp8x2(make_float2(r1[4 * j] * inv1, r1[4 * j + 1] * inv1), __NV_SATFINITE, __NV_E4M3);
+      hi = __nv_cvt_float2_to_fp8x2(make_float2(r1[4 * j + 2] * inv1, r1[4 * j + 3] * inv1), __NV_SATFINITE, __NV_E4M3);
+      w1[j] = lo | (hi << 16);
+    }
+    uint4* d0 = reinterpret_cast<uint4*>(a.v_codes + ((size_t)bh * D + 2 * cp) * a.n_pad + tok0);
+    uint4* d1 = reinterpret_cast<uint4*>(a.v_codes + ((size_t)bh * D + 2 * cp + 1) * a.n_pad + tok0);
+#pragma unroll
+    for (int j = 0; j < TPG / 16; ++j) {
+      d0[j] = make_uint4(w0[4 * j], w0[4 * j + 1], w0[4 * j + 2], w0[4 * j + 3]);
+      d1[j] = make_uint4(w1[4 * j], w1[4 * j + 1], w1[4 * j + 2], w1[4 * j + 3]);
+    }
+    if (tg == 0) {   // block means stored divided by the value scale (App. B)
+      const float a0 = mu0 * (am0 > 0.f ? inv0 : 1.0f), a1 = mu1 * (am1 > 0.f ? inv1 : 1.0f);
+      *reinterpret_cast<__nv_bfloat162*>(a.v_means + mu_at) = __floats2bfloat162_rn(a0, a1);
+    }
+  }
+
+  if constexpr (STAGE == kVQuant4) {
+    // NVFP4 along tokens: one microscale per channel per 16 consecutive permuted tokens
+    const float sixth = 1.0f / 6.0f;
+#pragma unroll
+    for (int half = 0; half < 2; ++half) {
+      const float* r = half == 0 ? r0 : r1;
+      const int c = 2 * cp + half;
+      unsigned int packed[TPG / 8];
+      unsigned int micro = 0;
+#pragma unroll
+      for (int gq = 0; gq < TPG / 16; ++gq) {
+        float m = 0.f;
+#pragma unroll
+        for (int i = 0; i < 16; ++i) m = fmaxf(m, fabsf(r[16 * gq + i]));
+        const unsigned int sb = __nv_cvt_float_to_fp8(m * sixth, __NV_SATFINITE, __NV_E4M3);
+        const float sdec = e4m3_to_float(sb);
+        const float rcp = sdec > 0.f ? 1.0f / sdec : 0.f;
+        micro |= sb << (8 * gq);
+#pragma unroll
+        for (int wi = 0; wi < 2; ++wi) {
+          unsigned int word = 0;
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            const int i = 16 * gq + 8 * wi + 2 * j;
+            const unsigned int two = __nv_cvt_float2_to_fp4x2(make_float2(r[i] * rcp, r[i + 1] * rcp), __NV_E2M1, cudaRoundNearest);
+            word |= (two & 0xffu) << (8 * j);
+          }
+          packed[2 * gq + wi] = sdec > 0.f ? word : 0u;
+        }
+      }
+      uint8_t* d = a.v_codes + ((size_t)bh * D + c) * (a.n_pad / 2) + tok0 / 2;
+      uint8_t* md = a.v_micro + ((size_t)bh * D + c) * (a.n_pad / 16) + tok0 / 16;
+      if constexpr (TPG == 32) {
+        *reinterpret_cast<uint4*>(d) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
+        *reinterpret_cast<unsigned short*>(md) = (unsigned short)micro;
+      } else {
+        *reinterpret_cast<uint2*>(d) = make_uint2(packed[0], packed[1]);
+        *md = (uint8_t)micro;
+      }
+    }
+    if (tg == 0)
+      *reinterpret_cast<__nv_bfloat162*>(a.v_means + mu_at) = __floats2bfloat162_rn(mu0, mu1);
+  }
+}
+
+// ---------------------------------------------------------------------------------------
+// Launch 1: statistics.  z = 0: K column sums; z = 1: V block means + residual amax;
+// z = 2 (4-bit): head amax of the rotated Q.
+template <int D, int BITS>
+__global__ void __launch_bounds__(kThreads) prep_stats_kernel(const PrepArgs a) {
+  extern __shared__ __align__(16) unsigned char smem[];
+  if (blockIdx.z == 0) {
+    if (a.flags & VC_FLAG_K_SMOOTH) qk_body<D, 1, kStageColSum>(a, smem);
+  } else if (blockIdx.z == 1) {
+    v_body<D, kVStats>(a, smem);
+  } else {
+    if constexpr (BITS == 4) qk_body<D, 0, kStageAmax>(a, smem);
+  }
+}
+
+// Launch 2: per-head finalization: K channel mean, V scale, g_Q.
+template <int D, int BITS>
+__global__ void prep_finalize_kernel(const PrepArgs a, int which) {
+  const int bh = a.bh0 + blockIdx.x, c = threadIdx.x;
+  if (which == 0) {
+    if (c < D) {
+      double s = 0.0;
+      if (a.flags & VC_FLAG_K_SMOOTH)
+        for (int j = 0; j < a.nb; ++j) s += (double)a.k_part[((size_t)bh * a.nb + j) * D + c];
+      a.k_mean[(size_t)bh * D + c] = (float)(s / (double)a.N);
+      float vs = 1.0f;
+      if (BITS == 8) {
+        const float am = __uint_as_float(a.v_amax[(size_t)bh * D + c]);
+        vs = am > 0.f ? am / 448.0f : 1.0f;
+      }
+      a.v_scale[(size_t)bh * D + c] = vs;
+    }
+    if (BITS == 4 && c == 0) {
+      const float am = __uint_as_float(a.qk_amax[bh]);
+      a.q_scale[bh] = am > 0.f ? am / 2688.0f : 1.0f;
+    }
+  } else if (BITS == 4 && c == 0) {
+    const float am = __uint_as_float(a.qk_amax[a.BH + bh]);
+    a.k_scale[bh] = am > 0.f ? am / 2688.0f : 1.0f;
+  }
+}
+
+// Launch 3 (4-bit only): head amax of the centered, rotated K.
+template <int D>
+__global__ void __launch_bounds__(kThreads) prep_kamax_kernel(const PrepArgs a) {
+  extern __shared__ __align__(16) unsigned char smem[];
+  qk_body<D, 1, kStageAmax>(a, smem);
+}
+
+// Launch 4: quantization.  z = 0: Q; z = 1: K; z = 2: V.
+template <int D, int BITS>
+__global__ void __launch_bounds__(kThreads) prep_quant_kernel(const PrepArgs a) {
+  extern __shared__ __align__(16) unsigned char smem[];
+  if (blockIdx.z == 0) {
+    qk_body<D, 0, BITS == 8 ? kStageQuant8 : kStageQuant4>(a, smem);
+  } else if (blockIdx.z == 1) {
+    qk_body<D, 1, BITS == 8 ? kStageQuant8 : kStageQuant4>(a, smem);
+  } else {
+    v_body<D, BITS == 8 ? kVQuant8 : kVQuant4>(a, smem);
+  }
+}
+
+template <int D, int BITS>
+cudaError_t run(const Problem& pr, PrepArgs a, const WorkLayout& wl, uint8_t* work, cudaStream_t s) {
+  const size_t rope_bytes = (size_t)a.rd.entries * 8;
+  const size_t qk_smem = 8 * D * 4 + ((a.flags & VC_FLAG_ROPE) && a.rope_in_smem ? rope_bytes : 0);
+  const size_t v_smem = (size_t)kBlock * D * 2 + (kThreads / (D / 2)) * D * 4;
+  const size_t smem = qk_smem > v_smem ? qk_smem : v_smem;
+  cudaError_t e;
+  if (smem > 48 * 1024) {
+    if ((e = cudaFuncSetAttribute(prep_stats_kernel<D, BITS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
+    if ((e = cudaFuncSetAttribute(prep_quant_kernel<D, BITS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
+    if ((e = cudaFuncSetAttribute(prep_kamax_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
+  }
+  if ((e = cudaMemsetAsync(work + wl.status, 0, 4, s)) != cudaSuccess) return e;
+  if ((e = cudaMemsetAsync(work + wl.amax, 0, wl.amax_bytes, s)) != cudaSuccess) return e;
+  if (a.flags & VC_FLAG_ROPE) {
+    rope_table_kernel<<<(a.rd.entries + 255) / 256, 256, 0, s>>>(
+        reinterpret_cast<float2*>(work + wl.rope), a.rd, (double)pr.rope_theta);
+    count_launches(1);
+  }
+  int group = pr.heads_per_pass > 0 ? pr.heads_per_pass : pr.BH;
+  if (group > 32768) group = 32768;
+  for (int bh0 = 0; bh0 < pr.BH; bh0 += group) {
+    const int nh = pr.BH - bh0 < group ? pr.BH - bh0 : group;
+    a.bh0 = bh0;
+    prep_stats_kernel<D, BITS><<<dim3(pr.nb, nh, BITS == 4 ? 3 : 2), kThreads, smem, s>>>(a);
+    prep_finalize_kernel<D, BITS><<<nh, D, 0, s>>>(a, 0);
+    count_launches(2);
+    if (BITS == 4) {
+      prep_kamax_kernel<D><<<dim3(pr.nb, nh, 1), kThreads, smem, s>>>(a);
+      prep_finalize_kernel<D, BITS><<<nh, 32, 0, s>>>(a, 1);
+      count_launches(2);
+    }
+    prep_quant_kernel<D, BITS><<<dim3(pr.nb, nh, 3), kThreads, smem, s>>>(a);
+    count_launches(1);
+  }
+  return cudaGetLastError();
+}
+
+}  // namespace
+
+cudaError_t launch_prep(const Problem& pr, const QuantLayout& ql, const WorkLayout& wl,
+                        const void* q, const void* k, const void* v, const int32_t* perm,
+                        uint8_t* quant, uint8_t* work, cudaStream_t stream) {
+  PrepArgs a{};
+  a.q = (const __nv_bfloat16*)q; a.k = (const __nv_bfloat16*)k; a.v = (const __nv_bfloat16*)v;
+  a.perm = perm;
+  a.stride_b = pr.stride_b; a.stride_h = pr.stride_h; a.stride_n = pr.stride_n;
+  a.H = pr.H; a.N = pr.N; a.n_pad = pr.n_pad; a.nb = pr.nb; a.bh0 = 0; a.flags = pr.flags; a.BH = pr.BH;
+  a.q_codes = quant + ql.q_codes; a.k_codes = quant + ql.k_codes; a.v_codes = quant + ql.v_codes;
+  a.q_micro = quant + ql.q_micro; a.k_micro = quant + ql.k_micro; a.v_micro = quant + ql.v_micro;
+  a.q_scale = (float*)(quant + ql.q_scale); a.k_scale = (float*)(quant + ql.k_scale);
+  a.v_scale = (float*)(quant + ql.v_scale); a.k_mean = (float*)(quant + ql.k_mean);
+  a.v_means = (__nv_bfloat16*)(quant + ql.v_means);
+  a.rope = (const float2*)(work + wl.rope);
+  a.k_part = (float*)(work + wl.k_part); a.v_mu = (float*)(work + wl.v_mu);
+  a.v_amax = (unsigned int*)(work + wl.amax);
+  a.qk_amax = a.v_amax + (size_t)pr.BH * pr.d;
+  const int len[3] = {pr.grid_t, pr.grid_h, pr.grid_w};
+  int ps = 0;
+  for (int ax = 0; ax < 3; ++ax) {
+    a.rd.pair_start[ax] = ps;
+    a.rd.pairs[ax] = pr.rope_dim[ax] / 2;
+    a.rd.off[ax] = wl.rope_off[ax];
+    a.rd.len[ax] = len[ax];
+    ps += pr.rope_dim[ax] / 2;
+  }
+  a.rd.entries = wl.rope_entries;
+  a.rd.grid_h = pr.grid_h; a.rd.grid_w = pr.grid_w;
+  a.rd.mul_w = ((1ull << 40) + pr.grid_w - 1) / pr.grid_w;
+  a.rd.mul_h = ((1ull << 40) + pr.grid_h - 1) / pr.grid_h;
+  a.rope_in_smem = (size_t)wl.rope_entries * 8 <= 96 * 1024;
+  if (pr.d == 128) return pr.bits == 8 ? run<128, 8>(pr, a, wl, work, stream) : run<128, 4>(pr, a, wl, work, stream);
+  return pr.bits == 8 ? run<64, 8>(pr, a, wl, work, stream) : run<64, 4>(pr, a, wl, work, stream);
+}
+
+}  // namespace vc

@@ -1,0 +1,142 @@
+"""Parity of the CUDA path (through the C ABI) against the CPU oracle, element by element.
+
+Three stages so that a failure can be attributed: (1) vc_prep against the oracle's bundle;
+(2) vc_attn_fwd fed the ORACLE's bundle against the oracle's emulated output; (3) vc_attn
+end to end.  Tolerances (from the benchmark spec): quantized codes identical except
+<= 0.1% of elements one code step apart; outputs within 2e-2 * max|V| elementwise and
+cosine >= 0.999 against the emulation.
+"""
+import numpy as np
+import pytest
+import torch
+
+import paper_2609_15810_b200 as vc
+import vc_inputs
+from paper_2609_15810_b200.binding import Params, alloc_buffers
+from oracle import attention as OA
+from oracle import compare as CMP
+
+import helpers as Hh
+
+pytestmark = pytest.mark.gpu
+
+SMALL = [  # name, B, H, N, d, grid
+    ("n128", 1, 1, 128, 128, (2, 8, 8)),
+    ("n129", 1, 2, 129, 128, (1, 3, 43)),
+    ("n255", 2, 1, 255, 128, (3, 5, 17)),
+    ("n300_d64", 1, 2, 300, 64, (3, 10, 10)),
+    ("n1024", 1, 2, 1024, 128, (4, 16, 16)),
+]
+
+
+def _inputs(B, H, N, d, grid, seed, kind="gauss"):
+    w = vc_inputs.Workload("t", B, H, N, d, grid, (8,), seed, kind)
+    return [t.cuda() for t in vc_inputs.make_qkv(w)]
+
+
+@pytest.mark.parametrize("bits", [8, 4])
+@pytest.mark.parametrize("perm_kind", ["identity", "random"])
+@pytest.mark.parametrize("case", SMALL, ids=[c[0] for c in SMALL])
+def test_prep_matches_oracle(case, perm_kind, bits):
+    _, B, H, N, d, grid = case
+    q, k, v = _inputs(B, H, N, d, grid, seed=11)
+    perm = None if perm_kind == "identity" else vc_inputs.random_perm(B, H, N, 5).cuda()
+    p = Params.make(B, H, N, d, grid, bits=bits)
+    quant, _ = Hh.run_prep(p, q, k, v, perm)
+    got = Hh.gpu_sections(p, quant)
+    for b in range(B):
+        for h in range(H):
+            ref, _ = Hh.oracle_prep(p, q, k, v, perm, b, h)
+            Hh.check_prep_head(p, got, b * H + h, ref, what=f"{case[0]} b{b} h{h}")
+
+
+@pytest.mark.parametrize("flags", [0, vc.VC_FLAG_ROPE, vc.VC_FLAG_HADAMARD, vc.VC_FLAG_K_SMOOTH | vc.VC_FLAG_V_SMOOTH])
+def test_prep_stage_switches(flags):
+    B, H, N, d, grid = 1, 2, 300, 128, (3, 10, 10)
+    q, k, v = _inputs(B, H, N, d, grid, seed=12)
+    p = Params.make(B, H, N, d, grid, bits=8, flags=flags)
+    quant, _ = Hh.run_prep(p, q, k, v, None)
+    got = Hh.gpu_sections(p, quant)
+    for h in range(H):
+        ref, _ = Hh.oracle_prep(p, q, k, v, None, 0, h)
+        Hh.check_prep_head(p, got, h, ref, what=f"flags{flags} h{h}")
+
+
+def test_prep_strided_inputs_and_head_groups():
+    """[B, N, H, d] storage viewed as [B, H, N, d], preprocessed two heads at a time."""
+    B, H, N, d, grid = 1, 4, 300, 128, (3, 10, 10)
+    q, k, v = _inputs(B, H, N, d, grid, seed=13)
+    qs, ks, vs = [t.permute(0, 2, 1, 3).contiguous() for t in (q, k, v)]          # [B, N, H, d]
+    p = Params.make(B, H, N, d, grid, bits=8, stride_b=N * H * d, stride_h=d, stride_n=H * d, heads_per_pass=2)
+    quant, _ = Hh.run_prep(p, qs, ks, vs, None)
+    p0 = Params.make(B, H, N, d, grid, bits=8)
+    quant0, _ = Hh.run_prep(p0, q, k, v, None)
+    assert torch.equal(quant, quant0)
+
+
+@pytest.mark.parametrize("p_format", [vc.VC_P_EXPCAST_E4M3, vc.VC_P_EXP_E4M3])
+@pytest.mark.parametrize("case", SMALL, ids=[c[0] for c in SMALL])
+def test_attn_fwd_on_oracle_bundle(case, p_format):
+    """Stage 2: isolates the attention kernel from code flips in prep."""
+    _, B, H, N, d, grid = case
+    q, k, v = _inputs(B, H, N, d, grid, seed=21)
+    perm = vc_inputs.random_perm(B, H, N, 6).cuda()
+    p = Params.make(B, H, N, d, grid, bits=8, p_format=p_format)
+    quant, work = alloc_buffers(p)
+    quant.zero_()
+    bundles, refs = [], []
+    fmt = OA.P_EXPCAST if p_format == vc.VC_P_EXPCAST_E4M3 else OA.P_EXP_E4M3
+    for b in range(B):
+        for h in range(H):
+            bundle, cfg = Hh.oracle_prep(p, q, k, v, perm, b, h)
+            bundles.append(bundle)
+            refs.append(OA.emulate_head(bundle, cfg, p_format=fmt))
+    Hh.upload_bundle(p, quant, bundles)
+    o = torch.empty(B, H, N, d, dtype=torch.bfloat16, device="cuda")
+    vc.vc_attn_fwd(p, quant, o, work)
+    vc.vc_poll_status(work)
+    vmax = float(v.float().abs().max())
+    for i, ref in enumerate(refs):
+        m = Hh.check_output(o.view(B * H, N, d)[i].float().cpu().numpy(), ref, vmax)
+        assert m["max_err_over_vmax"] < 1e-2, m
+
+
+@pytest.mark.parametrize("perm_kind", ["identity", "random", "kmeans"])
+def test_vc_attn_end_to_end_config1(perm_kind):
+    """Stage 3 on the tiny correctness configuration (B=1, H=2, N=1024, d=128, 8-bit)."""
+    w = vc_inputs.WORKLOADS["c1"]
+    q, k, v = [t.cuda() for t in vc_inputs.make_qkv(w)]
+    perm = {"identity": None, "random": vc_inputs.random_perm(w.B, w.H, w.N, 7).cuda(),
+            "kmeans": vc_inputs.kmeans_perm_all(v, k=8)}[perm_kind]
+    p = Params.make(w.B, w.H, w.N, w.d, w.grid, bits=8)
+    quant, work = alloc_buffers(p)
+    o = torch.empty(w.B, w.H, w.N, w.d, dtype=torch.bfloat16, device="cuda")
+    vc.vc_attn(p, q, k, v, perm, o, quant, work)
+    vc.vc_poll_status(work)
+    vmax = float(v.float().abs().max())
+    for h in range(w.H):
+        bundle, cfg = Hh.oracle_prep(p, q, k, v, perm, 0, h)
+        ref = OA.emulate_head(bundle, cfg)
+        got = o[0, h].float().cpu().numpy()
+        Hh.check_output(got, ref, vmax)
+        exact = OA.reference_head(q[0, h].float().cpu().numpy(), k[0, h].float().cpu().numpy(),
+                                  v[0, h].float().cpu().numpy(), cfg)
+        m0 = CMP.output_metrics(got, exact, vmax)
+        assert m0["cos"] > 0.999 and m0["max_err_over_vmax"] < 2e-2, m0
+
+
+def test_bad_arguments_are_rejected_on_the_host():
+    p = Params.make(1, 1, 128, 128, (2, 8, 8))
+    quant, work = alloc_buffers(p)
+    x = torch.zeros(1, 1, 128, 128, dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(vc.VcError):
+        vc.vc_prep(p, None, x, x, None, quant, work)
+    with pytest.raises(vc.VcError):
+        vc.vc_prep(p, x.view(-1)[1:], x, x, None, quant, work)          # misaligned
+    for bad in (dict(d=96), dict(N=0), dict(bits=5), dict(grid_w=9), dict(flags=64), dict(rope_dim_t=3)):
+        pb = Params.make(1, 1, 128, 128, (2, 8, 8))
+        for kk, vv in bad.items():
+            setattr(pb, kk, vv)
+        assert vc.vc_quant_bytes(pb) == 0
+        with pytest.raises(vc.VcError):
+            vc.vc_prep(pb, x, x, x, None, quant, work)

@@ -1,0 +1,41 @@
+"""The C-ABI library loads and exports every symbol include/vc_attn.h declares (no GPU)."""
+import ctypes
+import os
+import re
+
+import paper_2609_15810_b200 as vc
+from paper_2609_15810_b200.binding import Params
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _declared_symbols():
+    text = open(os.path.join(ROOT, "include", "vc_attn.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(vc_[a-z_0-9]+)\s*\(", text)))
+
+
+def test_every_declared_symbol_is_exported():
+    lib = vc.load_library()
+    names = _declared_symbols()
+    assert {"vc_prep", "vc_attn_fwd", "vc_attn", "vc_quant_bytes", "vc_workspace_bytes"} <= set(names)
+    for n in names:
+        assert hasattr(lib, n), n
+
+
+def test_sizes_and_argument_validation_without_a_gpu():
+    p = Params.make(1, 40, 32760, 128, (21, 30, 52), bits=8)
+    n_pad = 32768
+    qb = vc.vc_quant_bytes(p)
+    assert qb >= 3 * 40 * n_pad * 128 and qb < 3 * 40 * n_pad * 128 * 1.02
+    assert vc.vc_workspace_bytes(p) > 0
+    p4 = Params.make(1, 40, 32760, 128, (21, 30, 52), bits=4)
+    assert vc.vc_quant_bytes(p4) < 0.6 * qb
+    for bad in (dict(d=100), dict(N=-1), dict(bits=3), dict(grid_t=20), dict(p_format=9)):
+        pb = Params.make(1, 2, 1024, 128, (4, 16, 16))
+        for k, v in bad.items():
+            setattr(pb, k, v)
+        assert vc.vc_quant_bytes(pb) == 0 and vc.vc_workspace_bytes(pb) == 0
+    assert vc.vc_status_string(0) == "ok" and "timed out" in vc.vc_status_string(5)
+    assert ctypes.sizeof(Params) == 96
+    assert vc.vc_launch_count() == 0
