@@ -1,0 +1,285 @@
+#!/usr/bin/env python
+"""Benchmark of the VC-Attention hot path (prep + quantized attention forward) on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c3] [--bits 8]
+    python bench.py --impl reference ...      # the CPU oracle on the host cores
+
+One step = one pass of the whole hot path (vc_attn: preprocessing pass + attention
+forward) over one synthetic batch shaped like the named workload, inputs resident in HBM.
+Metric: attention TFLOP/s = 4 B H N^2 d / time.  Prints ONE JSON line on rank 0.
+"""
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import torch  # noqa: E402
+
+import vc_inputs  # noqa: E402
+
+METRIC = "quantized attn fwd TFLOPS (hot path: prep + attention forward)"
+UNIT = "TFLOP/s"
+
+
+def _peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return {"hbm_gbs": p["hbm_gbs"], "bf16_burst": p["bf16_tflops"], "bf16_sustained": p["bf16_tflops_sustained"],
+                "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_burst": 1590.0, "bf16_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index, self.proc, self.lines = index, None, []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.Q,
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.lines:
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 8:
+                continue
+            try:
+                sm.append(float(f[0])); mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for name, val in zip(names, f[4:8]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def run_reference(args, w, bits):
+    """The oracle as it stands, timed on the host cores on a bounded sample of the workload."""
+    import numpy as np
+    from oracle import attention as OA
+    from oracle import prep as OP
+    rows_per_step = args.ref_rows
+    q, k, v = [t[0, 0].float().numpy() for t in vc_inputs.make_qkv(w, heads=[0])]
+    cfg = OP.PrepConfig(N=w.N, d=w.d, grid=w.grid, bits=bits)
+    rows = np.linspace(0, w.N - 1, rows_per_step).astype(np.int64)
+
+    def step():
+        bundle = OP.prep_head(q, k, v, None, cfg)
+        OA.emulate_head(bundle, cfg, rows=rows)
+
+    for _ in range(args.warmup):
+        step()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        step()
+    dt = (time.perf_counter() - t0) / args.steps
+    flops = 4.0 * rows_per_step * w.N * w.d            # the sampled rows against all keys
+    value = flops / dt / 1e12
+    sample = f"per step: preprocessing of 1 head in full + {rows_per_step} query rows x all {w.N} keys of that head"
+    return {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f64", "data": "synthetic", "impl": "reference",
+            "config": {"workload": w.name, "B": w.B, "H": w.H, "N": w.N, "d": w.d, "bits": bits, "sample": sample},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": os.cpu_count(), "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+
+
+def cpu_baseline(w, bits, budget_rows=256):
+    import numpy as np
+    from oracle import attention as OA
+    from oracle import prep as OP
+    q, k, v = [t[0, 0].float().numpy() for t in vc_inputs.make_qkv(w, heads=[0])]
+    cfg = OP.PrepConfig(N=w.N, d=w.d, grid=w.grid, bits=bits)
+    rows = np.linspace(0, w.N - 1, budget_rows).astype(np.int64)
+    t0 = time.perf_counter()
+    bundle = OP.prep_head(q, k, v, None, cfg)
+    t1 = time.perf_counter()
+    OA.emulate_head(bundle, cfg, rows=rows)
+    t2 = time.perf_counter()
+    flops = 4.0 * budget_rows * w.N * w.d
+    return {"value": flops / (t2 - t0) / 1e12, "unit": UNIT, "cores": os.cpu_count(), "kind": "oracle",
+            "sample": f"preprocessing of 1 of {w.B * w.H} heads in full ({t1 - t0:.1f} s) + {budget_rows} of {w.N} query "
+                      f"rows x all keys of that head ({t2 - t1:.1f} s); NumPy, threads as BLAS picks"}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="c3")
+    ap.add_argument("--bits", type=int, default=8)
+    ap.add_argument("--perm", default="kmeans", choices=["kmeans", "identity", "random"])
+    ap.add_argument("--heads-per-pass", type=int, default=0)
+    ap.add_argument("--ref-rows", type=int, default=128)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    args = ap.parse_args()
+    w = vc_inputs.WORKLOADS[args.workload]
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+
+    if args.impl == "reference":
+        if rank == 0:
+            print(json.dumps(run_reference(args, w, args.bits)), flush=True)
+        return
+
+    import paper_2609_15810_b200 as vc
+    from paper_2609_15810_b200.binding import Params, alloc_buffers
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+
+    # every rank runs the same workload on its own GPU (heads are independent: no collective)
+    q, k, v = vc_inputs.make_qkv(w, device=dev)
+    if args.perm == "kmeans":
+        perm = vc_inputs.kmeans_perm_all(v)
+    elif args.perm == "random":
+        perm = vc_inputs.random_perm(w.B, w.H, w.N, w.seed, device=dev)
+    else:
+        perm = None
+    p = Params.make(w.B, w.H, w.N, w.d, w.grid, bits=args.bits, heads_per_pass=args.heads_per_pass)
+    quant, work = alloc_buffers(p, device=dev)
+    o = torch.empty(w.B, w.H, w.N, w.d, dtype=torch.bfloat16, device=dev)
+    stream = torch.cuda.current_stream()
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 3)):
+        vc.vc_attn(p, q, k, v, perm, o, quant, work)
+    vc.vc_poll_status(work)
+
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
+    launches0 = vc.vc_launch_count()
+    barrier()
+    t_start, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t_start.record(stream)
+    for s in range(args.steps):
+        ev[s][0].record(stream)
+        vc.vc_prep(p, q, k, v, perm, quant, work)
+        ev[s][1].record(stream)
+        vc.vc_attn_fwd(p, quant, o, work)
+        ev[s][2].record(stream)
+    t_end.record(stream)
+    barrier()
+    launches = vc.vc_launch_count() - launches0
+    clocks = sampler.stop()
+    vc.vc_poll_status(work)
+    ms_total = t_start.elapsed_time(t_end)
+    prep_ms = statistics.mean(e[0].elapsed_time(e[1]) for e in ev)
+    attn_ms = statistics.mean(e[1].elapsed_time(e[2]) for e in ev)
+    ms_step = ms_total / args.steps
+    if world > 1:
+        t = torch.tensor([ms_step], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_step = float(t.item())
+    value = world * w.flops / (ms_step * 1e-3) / 1e12
+
+    # end to end through the host-buffer entry point: H2D of Q, K, V, pi and D2H of O inside the timer
+    e2e = None
+    if not args.no_e2e:
+        hq, hk, hv = [t.cpu().pin_memory() for t in (q, k, v)]
+        hperm = perm.cpu().pin_memory() if perm is not None else None
+        ho = torch.empty(o.shape, dtype=o.dtype).pin_memory()
+        n_e2e = max(2, min(args.steps, 5))
+        vc.vc_attn_host(p, hq, hk, hv, hperm, ho, q, k, v, perm, o, quant, work)
+        barrier()
+        t0 = time.perf_counter()
+        for _ in range(n_e2e):
+            vc.vc_attn_host(p, hq, hk, hv, hperm, ho, q, k, v, perm, o, quant, work)
+        barrier()
+        e2e_ms = (time.perf_counter() - t0) * 1e3 / n_e2e
+        if world > 1:
+            t = torch.tensor([e2e_ms], device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            e2e_ms = float(t.item())
+        nbytes = q.numel() * 2
+        e2e = {"value": world * w.flops / (e2e_ms * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": e2e_ms,
+               "h2d_bytes_per_step": 3 * nbytes + (perm.numel() * 4 if perm is not None else 0),
+               "d2h_bytes_per_step": nbytes, "steps": n_e2e}
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    peaks = _peaks()
+    # dominant kernel: the attention forward (dense contraction on the tensor cores).  Its peak is
+    # the measured bf16 figure x the nominal FP8:bf16 ratio of 2 (x4 for FP4); the kernel runs inside
+    # a long step, so the sustained figure applies.
+    ratio = 2.0 if args.bits == 8 else 2.0   # the 4-bit path's P V product is FP8-rate at best: see the design doc
+    peak = peaks["bf16_sustained"] * ratio
+    achieved = w.flops / (attn_ms * 1e-3) / 1e12
+    n_pad = 128 * ((w.N + 127) // 128)
+    prep_bytes = w.B * w.H * (3 * w.N * w.d * 2 + 2 * w.N * 4 + 3 * n_pad * w.d * (1 if args.bits == 8 else 0.5625)
+                              + (2 * (n_pad // 128) * 4 + w.d * 4) + (n_pad // 128) * w.d * 2)
+    prep_gbs = prep_bytes / (prep_ms * 1e-3) / 1e9
+    out = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "e4m3" if args.bits == 8 else "nvfp4", "data": "synthetic",
+        "config": {"workload": w.name, "B": w.B, "H": w.H, "N": w.N, "d": w.d, "grid": list(w.grid),
+                   "bits": args.bits, "perm": args.perm, "l2": "inputs larger than L2 (Q+K+V = %.0f MB)" % (3 * q.numel() * 2 / 1e6),
+                   "step": "vc_prep + vc_attn_fwd"},
+        "clocks": clocks, "gpu_launches": launches, "e2e": e2e,
+        "roofline": {"bound": "tensor", "kernel": "vc_attn_fwd", "achieved": achieved, "peak": peak, "unit": UNIT,
+                     "frac": achieved / peak, "traffic": None,
+                     "peak_source": f"{peaks['source']}: bf16 sustained {peaks['bf16_sustained']} TF/s x {ratio:g} (nominal FP8:bf16)",
+                     "frac_of_nominal_fp8_4500": achieved / 4500.0, "ms": attn_ms},
+        "prep": {"ms": prep_ms, "algorithmic_gb": prep_bytes / 1e9, "gbs": prep_gbs,
+                 "frac_of_measured_hbm": prep_gbs / peaks["hbm_gbs"], "frac_of_8tbs": prep_gbs / 8000.0},
+    }
+    if not args.no_cpu_baseline:
+        out["cpu_baseline"] = cpu_baseline(w, args.bits)
+    print(json.dumps(out), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()
