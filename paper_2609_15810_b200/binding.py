@@ -31,7 +31,7 @@ class Params(ctypes.Structure):
                 ("rope_dim_t", ctypes.c_int32), ("rope_dim_h", ctypes.c_int32), ("rope_dim_w", ctypes.c_int32),
                 ("rope_theta", ctypes.c_float),
                 ("stride_b", ctypes.c_int64), ("stride_h", ctypes.c_int64), ("stride_n", ctypes.c_int64),
-                ("heads_per_pass", ctypes.c_int32), ("reserved", ctypes.c_int32)]
+                ("heads_per_pass", ctypes.c_int32), ("kernel_variant", ctypes.c_int32)]
 
     @classmethod
     def make(cls, B, H, N, d, grid, bits=8, p_format=VC_P_DEFAULT, flags=VC_FLAG_ALL, **kw):

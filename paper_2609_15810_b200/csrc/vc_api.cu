@@ -21,6 +21,7 @@ vc_status resolve(const vc_params* p, Problem* out) {
   pr.BH = pr.B * pr.H;
   pr.grid_t = p->grid_t; pr.grid_h = p->grid_h; pr.grid_w = p->grid_w;
   if (pr.grid_t < 1 || pr.grid_h < 1 || pr.grid_w < 1) return VC_ERR_INVALID_ARG;
+  if (pr.grid_h > (1 << 18) || pr.grid_w > (1 << 18)) return VC_ERR_INVALID_ARG;
   if ((int64_t)pr.grid_t * pr.grid_h * pr.grid_w != pr.N) return VC_ERR_INVALID_ARG;
   pr.bits = p->bits;
   if (pr.bits != 8 && pr.bits != 4) return VC_ERR_INVALID_ARG;
@@ -55,6 +56,8 @@ vc_status resolve(const vc_params* p, Problem* out) {
   pr.n_pad = kBlock * ((pr.N + kBlock - 1) / kBlock);
   pr.nb = pr.n_pad / kBlock;
   pr.heads_per_pass = p->heads_per_pass > 0 ? p->heads_per_pass : 0;
+  pr.kernel_variant = p->kernel_variant;
+  if (pr.kernel_variant < 0 || pr.kernel_variant > 1) return VC_ERR_INVALID_ARG;
   *out = pr;
   return VC_OK;
 }
@@ -106,6 +109,7 @@ WorkLayout work_layout(const Problem& pr) {
   W.v_mu = place(BH * nb * d * 4);
   W.amax_bytes = BH * d * 4 + 2 * BH * 4;
   W.amax = place(W.amax_bytes);
+  W.mu_mma = place(BH * ((nb + 15) / 16) * d * 128);
   W.total = off;
   return W;
 }
