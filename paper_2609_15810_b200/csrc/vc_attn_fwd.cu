@@ -12,6 +12,7 @@
 // Epilogue: O = s_V * A / l, bf16, original query order.
 #include <cuda_bf16.h>
 #include <cuda_fp8.h>
+#include <cstdlib>
 
 #include "vc_internal.h"
 #include "vc_sm100.cuh"
@@ -28,6 +29,7 @@ struct AttnArgs {
   const __nv_bfloat16* v_means;
   __nv_bfloat16* o;
   uint32_t* status;
+  int debug;
   int N, n_pad, nb, ng, p_format;   // ng = groups of 16 key tiles
   float sl;        // softmax_scale * log2(e)
   float code_off;  // 120 + beta  (Eq. 7)
@@ -217,23 +219,28 @@ attn_fwd_serial_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
 //   warp 1      MMA issuer (one thread): S[j&1] = Q^ K^_j^T is issued one tile ahead of
 //               A += P^_{j-1} R^_{j-1}, so the tensor core works on the next scores while the
 //               softmax stage turns the current ones into codes
-//   warps 4-7   softmax stage, one thread per query row: running max, alpha, ExpCast-FP8
-//               code (fma.sat + magic-number round, no exponential), P^ -> TMEM
-//   warps 8-11  correction stage, one thread per row: rescales A by alpha when the running
+//   warps 4-19  softmax stage, four threads per query row (32 key columns each): running
+//               max, alpha, ExpCast-FP8 code (fma.sat + magic-number round, no exponential),
+//               P^ -> TMEM
+//   warps 20-23 correction stage, one thread per row: rescales A by alpha when the running
 //               maximum moved, owns l, and keeps the per-tile row sums r_ij (referenced to
 //               the current maximum) in TMEM as a TF32 hi/lo pair
 //
 // Mean restoration (Eq. 6) is deferred: every 16 tiles one small kind::tf32 MMA adds
 // sum_j r_ij mu~_j to the same accumulator, [128 x 32] (row sums, hi/lo) x [d x 32] (means).
+__device__ long long g_trace[8192];
+#define TRACE(ev, jj) do { if ((a.debug & 4) && ((threadIdx.x & 31) == 0 || ((ev) >= 14 && (ev) <= 17)) && blockIdx.x == 5 && blockIdx.y == 0 && (jj) >= 40 && (jj) < 48) { g_trace[((ev) * 8 + ((jj) - 40))] = clock64(); } } while (0)
 constexpr int kStages = 3;
 constexpr int kGroup = 16;          // key tiles per mean-restoration MMA
 constexpr uint32_t kWaitLimit = 1u << 21;
 
 struct PipeSmem {
   uint64_t q_full, k_full[kStages], v_full[kStages], kv_empty[kStages];
+  uint64_t pm_full[2][4];
   uint64_t s_full[2], a_full[2], p_full[2], c_done[2], o_done[2], g_done[2], mu_full[2], mu_empty[2];
   float alpha[2][128];
-  float rsum[2][128];
+  float pmax[2][4][128];
+  float rsum[2][4][128];
   uint32_t tmem_base;
   volatile int abort;
 };
@@ -254,7 +261,7 @@ __device__ __forceinline__ bool warp_wait(uint64_t* bar, uint32_t parity, PipeSm
 }
 
 template <int D, bool EXPCAST>
-__global__ void __launch_bounds__(384, 1)
+__global__ void __launch_bounds__(768, 1)
 attn_fwd_pipe_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                      const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_mu,
                      const AttnArgs a) {
@@ -277,9 +284,10 @@ attn_fwd_pipe_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
     mbar_init(&sh->q_full, 1);
     for (int i = 0; i < kStages; ++i) { mbar_init(&sh->k_full[i], 1); mbar_init(&sh->v_full[i], 1); mbar_init(&sh->kv_empty[i], 1); }
     for (int i = 0; i < 2; ++i) {
-      mbar_init(&sh->s_full[i], 1); mbar_init(&sh->a_full[i], 128); mbar_init(&sh->p_full[i], 128);
+      mbar_init(&sh->s_full[i], 1); mbar_init(&sh->a_full[i], 128); mbar_init(&sh->p_full[i], 512);
       mbar_init(&sh->c_done[i], 128); mbar_init(&sh->o_done[i], 1); mbar_init(&sh->g_done[i], 128);
       mbar_init(&sh->mu_full[i], 1); mbar_init(&sh->mu_empty[i], 1);
+      for (int w = 0; w < 4; ++w) mbar_init(&sh->pm_full[i][w], 128);
     }
     sh->abort = 0;
     mbar_fence_init();
@@ -293,7 +301,6 @@ attn_fwd_pipe_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
   const uint32_t lane_base = tmem + ((uint32_t)((warp & 3) * 32) << 16);
 
   if (warp < 4) {
-    reg_dec<56>();
     if (warp == 0 && lane == 0) {
       // ------------------------------------------------------------------ TMA producer
       mbar_expect_tx(&sh->q_full, kTileBytes);
@@ -311,6 +318,7 @@ attn_fwd_pipe_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
         tma_load_3d(sK + st * kTileBytes, &tm_k, &sh->k_full[st], 0, j * 128, bh);
         mbar_expect_tx(&sh->v_full[st], kTileBytes);
         tma_load_3d(sV + st * kTileBytes, &tm_v, &sh->v_full[st], j * 128, 0, bh);
+        TRACE(0, j);
       }
     } else if (warp == 1 && lane == 0) {
       // ------------------------------------------------------------------ MMA issuer
@@ -321,21 +329,25 @@ attn_fwd_pipe_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
         if (j < nb) {
           const int st = j % kStages, it = j / kStages;
           if (!(ok = wait_or_abort(&sh->k_full[st], it & 1, sh, a.status, 21))) break;
+          TRACE(1, j);
           tc_fence_after();
           const uint64_t dk = smem_desc_kmajor(smem_u32(sK + st * kTileBytes), D);
 #pragma unroll
           for (int k = 0; k < D / 32; ++k) mma_f8_ss(tmem + S_COL + 128 * (j & 1), dq + 2 * k, dk + 2 * k, idesc_qk, k > 0);
           mma_commit(&sh->s_full[j & 1]);
+          TRACE(2, j);
         }
         if (j >= 1) {
           const int i = j - 1, b = i & 1, ph = (i >> 1) & 1, st = i % kStages, it = i / kStages;
           if (!(ok = wait_or_abort(&sh->p_full[b], ph, sh, a.status, 22))) break;
+          TRACE(3, i);
           if (!(ok = wait_or_abort(&sh->c_done[b], ph, sh, a.status, 23))) break;
+          TRACE(4, i);
           if (!(ok = wait_or_abort(&sh->v_full[st], it & 1, sh, a.status, 24))) break;
           tc_fence_after();
           const uint64_t dv = smem_desc_kmajor(smem_u32(sV + st * kTileBytes), 128);
 #pragma unroll
-          for (int k = 0; k < 4; ++k) mma_f8_ts(tmem + O_COL, tmem + S_COL + 128 * b + 8 * k, dv + 2 * k, idesc_pv, (i > 0) | (k > 0));
+          for (int k = 0; k < 4; ++k) { mma_f8_ts(tmem + O_COL, tmem + S_COL + 128 * b + 8 * k, dv + 2 * k, idesc_pv, (i > 0) | (k > 0)); TRACE(12 + k, i); }
           if ((i % kGroup) == kGroup - 1 || i == nb - 1) {
             const int g = i / kGroup;
             if (!(ok = wait_or_abort(&sh->g_done[g & 1], (g >> 1) & 1, sh, a.status, 25))) break;
@@ -348,57 +360,65 @@ attn_fwd_pipe_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
           }
           mma_commit(&sh->kv_empty[st]);
           mma_commit(&sh->o_done[b]);
+          TRACE(5, i);
         }
       }
     }
-  } else if (warp < 8) {
+  } else if (warp < 20) {
     // -------------------------------------------------------------------- softmax stage
-    reg_inc<232>();
-    const int row = tid - 128;
+    // 16 warps: warp (4 + 4 q + w) owns rows 32 w .. 32 w + 31 (its TMEM lane quadrant) and
+    // key columns 32 q .. 32 q + 31; the four threads of a row exchange their partial
+    // maxima through shared memory behind a 128-thread mbarrier.
+    const int cq = (warp - 4) >> 2, quad = warp & 3;
+    const int row = quad * 32 + lane;
     const float sq = a.q_scale[(size_t)bh * nb + qblk];
     float m_run = -INFINITY;
     for (int j = 0; j < nb; ++j) {
       const int b = j & 1, ph = (j >> 1) & 1;
       const float cs = (sq * a.k_scale[(size_t)bh * nb + j]) * a.sl;
       if (!warp_wait(&sh->s_full[b], ph, sh, a.status, 30)) break;
+      if (cq == 0 && quad == 0 && lane == 0) TRACE(6, j);
       tc_fence_after();
-      uint32_t s0[32], s1[32], s2[32], s3[32];
+      uint32_t sv[32];
       const uint32_t sbase = lane_base + S_COL + 128 * b;
-      tmem_ld32(sbase, s0); tmem_ld32(sbase + 32, s1); tmem_ld32(sbase + 64, s2); tmem_ld32(sbase + 96, s3);
+      tmem_ld32(sbase + 32 * cq, sv);
       tmem_wait_ld();
-      const int nv = a.N - j * 128;                       // >= 128 except on the ragged last tile
-      if (nv < 128) {                                     // padded keys never win the maximum
+      if (cq == 0 && quad == 0 && lane == 0) TRACE(7, j);
+      const int nv = a.N - j * 128 - 32 * cq;             // valid keys among my 32 columns
+      if (nv < 32) {                                      // padded keys never win the maximum
 #pragma unroll
-        for (int i = 0; i < 32; ++i) {
-          if (i >= nv) s0[i] = 0xff800000u;
-          if (32 + i >= nv) s1[i] = 0xff800000u;
-          if (64 + i >= nv) s2[i] = 0xff800000u;
-          if (96 + i >= nv) s3[i] = 0xff800000u;
-        }
+        for (int i = 0; i < 32; ++i)
+          if (i >= nv) sv[i] = 0xff800000u;
       }
-      float mx0 = __uint_as_float(s0[0]), mx1 = __uint_as_float(s1[0]), mx2 = __uint_as_float(s2[0]), mx3 = __uint_as_float(s3[0]);
+      float mx0 = __uint_as_float(sv[0]), mx1 = __uint_as_float(sv[1]);
 #pragma unroll
-      for (int i = 1; i < 31; i += 2) {
-        mx0 = max3(mx0, __uint_as_float(s0[i]), __uint_as_float(s0[i + 1]));
-        mx1 = max3(mx1, __uint_as_float(s1[i]), __uint_as_float(s1[i + 1]));
-        mx2 = max3(mx2, __uint_as_float(s2[i]), __uint_as_float(s2[i + 1]));
-        mx3 = max3(mx3, __uint_as_float(s3[i]), __uint_as_float(s3[i + 1]));
+      for (int i = 2; i < 30; i += 4) {
+        mx0 = max3(mx0, __uint_as_float(sv[i]), __uint_as_float(sv[i + 1]));
+        mx1 = max3(mx1, __uint_as_float(sv[i + 2]), __uint_as_float(sv[i + 3]));
       }
-      mx0 = max3(mx0, __uint_as_float(s0[31]), mx1);
-      mx2 = max3(mx2, __uint_as_float(s1[31]), mx3);
-      const float mx = max3(mx0, mx2, fmaxf(__uint_as_float(s2[31]), __uint_as_float(s3[31])));
+      sh->pmax[b][cq][row] = max3(mx0, mx1, fmaxf(__uint_as_float(sv[30]), __uint_as_float(sv[31])));
+      mbar_arrive(&sh->pm_full[b][quad]);                 // bounded stand-in for a named barrier;
+      if (!warp_wait(&sh->pm_full[b][quad], ph, sh, a.status, 31)) break;   // also: all four have read S
+      if (cq == 0 && quad == 0 && lane == 0) TRACE(8, j);
+      const float mx = fmaxf(fmaxf(sh->pmax[b][0][row], sh->pmax[b][1][row]), fmaxf(sh->pmax[b][2][row], sh->pmax[b][3][row]));
       const float m_new = fmaxf(m_run, mx * cs);          // m' = max(m, rowmax S_ij)
-      sh->alpha[b][row] = ex2_approx(m_run - m_new);      // alpha; 0 on the first tile
-      mbar_arrive(&sh->a_full[b]);
+      if (cq == 0) {
+        sh->alpha[b][row] = ex2_approx(m_run - m_new);    // alpha; 0 on the first tile
+        mbar_arrive(&sh->a_full[b]);
+      }
       m_run = m_new;
 
-      uint32_t pk[32];
+      uint32_t pk[8];
       float acc0 = 0.f, acc1 = 0.f;
-      if constexpr (EXPCAST) {
+      if (a.debug & 2) {
+#pragma unroll
+        for (int w = 0; w < 8; ++w) pk[w] = sv[w] & 0x38383838u;
+      } else if constexpr (EXPCAST) {
         // Eq. 7 in two FMAs: t = sat((8 u + 120 + beta) / 128) clips to [0, 1], then
         // t * 128 + 1.5 * 2^23 rounds to the nearest even integer in the low mantissa bits.
         const float fa = cs * 0.0625f, fb = (a.code_off - 8.0f * m_new) * 0.0078125f;
-        auto code4 = [&](const uint32_t (&sv)[32], int w) -> uint32_t {
+#pragma unroll
+        for (int w = 0; w < 8; ++w) {
           const uint32_t r0 = __float_as_uint(fmaf(fma_sat(__uint_as_float(sv[4 * w]), fa, fb), 128.0f, 12582912.0f));
           const uint32_t r1 = __float_as_uint(fmaf(fma_sat(__uint_as_float(sv[4 * w + 1]), fa, fb), 128.0f, 12582912.0f));
           const uint32_t r2 = __float_as_uint(fmaf(fma_sat(__uint_as_float(sv[4 * w + 2]), fa, fb), 128.0f, 12582912.0f));
@@ -406,41 +426,40 @@ attn_fwd_pipe_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
           // (code << 20) read as fp32 is the decoded E4M3 value times 2^-120, subnormal codes included
           acc0 += __uint_as_float(r0 << 20) + __uint_as_float(r2 << 20);
           acc1 += __uint_as_float(r1 << 20) + __uint_as_float(r3 << 20);
-          return __byte_perm(__byte_perm(r0, r1, 0x0040), __byte_perm(r2, r3, 0x0040), 0x5410);
-        };
-#pragma unroll
-        for (int w = 0; w < 8; ++w) { pk[w] = code4(s0, w); pk[8 + w] = code4(s1, w); pk[16 + w] = code4(s2, w); pk[24 + w] = code4(s3, w); }
+          pk[w] = __byte_perm(__byte_perm(r0, r1, 0x0040), __byte_perm(r2, r3, 0x0040), 0x5410);
+        }
       } else {
         // exponentiate, then cast (Fig. 4a upper box)
         const float nm = 8.0f - m_new;
-        auto code4 = [&](const uint32_t (&sv)[32], int w) -> uint32_t {
+#pragma unroll
+        for (int w = 0; w < 8; ++w) {
           const float p0 = exp2f(fmaf(__uint_as_float(sv[4 * w]), cs, nm)), p1 = exp2f(fmaf(__uint_as_float(sv[4 * w + 1]), cs, nm));
           const float p2 = exp2f(fmaf(__uint_as_float(sv[4 * w + 2]), cs, nm)), p3 = exp2f(fmaf(__uint_as_float(sv[4 * w + 3]), cs, nm));
           const uint32_t lo = __nv_cvt_float2_to_fp8x2(make_float2(p0, p1), __NV_SATFINITE, __NV_E4M3);
           const uint32_t hi = __nv_cvt_float2_to_fp8x2(make_float2(p2, p3), __NV_SATFINITE, __NV_E4M3);
           acc0 += __uint_as_float((lo & 0xffu) << 20) + __uint_as_float((hi & 0xffu) << 20);
           acc1 += __uint_as_float((lo >> 8) << 20) + __uint_as_float((hi >> 8) << 20);
-          return lo | (hi << 16);
-        };
-#pragma unroll
-        for (int w = 0; w < 8; ++w) { pk[w] = code4(s0, w); pk[8 + w] = code4(s1, w); pk[16 + w] = code4(s2, w); pk[24 + w] = code4(s3, w); }
+          pk[w] = lo | (hi << 16);
+        }
       }
-      sh->rsum[b][row] = ((acc0 + acc1) * 1152921504606846976.0f) * 1152921504606846976.0f;   // x 2^120
-      tmem_st32(sbase, pk);                               // P^ aliases the consumed scores
+      sh->rsum[b][cq][row] = ((acc0 + acc1) * 1152921504606846976.0f) * 1152921504606846976.0f;   // x 2^120
+      tmem_st8(sbase + 8 * cq, pk);                       // P^ aliases the consumed scores
       tmem_wait_st();
       tc_fence_before();
       mbar_arrive(&sh->p_full[b]);
+      if (cq == 0 && quad == 0 && lane == 0) TRACE(9, j);
     }
   } else {
     // -------------------------------------------------------------------- correction stage
-    const int row = tid - 256;
+    const int row = (warp & 3) * 32 + lane;
     float l_run = 0.f;
     bool ok = true;
     for (int j = 0; j < nb; ++j) {
       const int b = j & 1, ph = (j >> 1) & 1, slot = j % kGroup, g = j / kGroup;
       if (!(ok = warp_wait(&sh->a_full[b], ph, sh, a.status, 40))) break;
       const float alpha = sh->alpha[b][row];
-      if (j > 0) {
+      if ((warp & 3) == 0 && lane == 0) TRACE(10, j);
+      if (j > 0 && !(a.debug & 1)) {
         if (!(ok = warp_wait(&sh->o_done[(j - 1) & 1], ((j - 1) >> 1) & 1, sh, a.status, 41))) break;
         tc_fence_after();
       }
@@ -450,7 +469,7 @@ attn_fwd_pipe_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
         for (int i = 0; i < 32; ++i) r[i] = 0u;
         tmem_st32(lane_base + R_COL, r);
       }
-      if (j > 0 && __any_sync(0xffffffffu, alpha != 1.0f)) {
+      if (j > 0 && !(a.debug & 1) && __any_sync(0xffffffffu, alpha != 1.0f)) {
 #pragma unroll 1
         for (int c = 0; c < D / 32 + (slot > 0 ? 1 : 0); ++c) {
           const uint32_t col = c < D / 32 ? O_COL + 32 * c : R_COL;
@@ -465,8 +484,9 @@ attn_fwd_pipe_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
       tmem_wait_st();
       tc_fence_before();
       mbar_arrive(&sh->c_done[b]);
+      if ((warp & 3) == 0 && lane == 0) TRACE(11, j);
       if (!(ok = warp_wait(&sh->p_full[b], ph, sh, a.status, 42))) break;
-      const float rs = sh->rsum[b][row];                  // r_ij = P~_ij 1 (decoded codes)
+      const float rs = (sh->rsum[b][0][row] + sh->rsum[b][1][row]) + (sh->rsum[b][2][row] + sh->rsum[b][3][row]);   // r_ij = P~_ij 1
       l_run += rs;                                        // l <- alpha l + r
       const uint32_t hi = (__float_as_uint(rs) + 0x1000u) & 0xffffe000u;   // nearest TF32
       const float lo = rs - __uint_as_float(hi);
@@ -521,6 +541,353 @@ __global__ void means_mma_layout_kernel(const __nv_bfloat16* __restrict__ means,
   }
 }
 
+
+// ---------------------------------------------------------------------------------------
+// Two-query-tile kernel (default).  A CTA owns TWO 128-row query tiles of one (batch, head)
+// and streams each K^_j / R^_j tile through both, so every key/value byte fetched from L2
+// feeds 256 query rows.  The probability codes travel through SHARED memory, not through the
+// score columns of tensor memory: a score tile is free again as soon as its 128 x 128 values
+// are in registers, so S_t(j+1) = Q^_t K^_{j+1}^T is computed while the softmax warpgroup is
+// still turning S_t(j) into codes, and the warpgroup never waits for the tensor core.
+//
+//   warp 0        TMA producer: Q0, Q1 once; then per key tile K^_j, R^_j and the tile's block
+//                 mean (as a [d x 8] TF32 operand) through a 4-stage ring
+//   warp 1        MMA issuer (one thread), per key tile j and query tile t:
+//                   S_t  = Q^_t K^_{j+1}^T   4 x kind::f8f6f4, as soon as S_t(j) has been read
+//                   A_t += P^_t R^_j         4 x kind::f8f6f4, P^ codes from shared memory
+//                   A_t += [r_hi r_lo] mu~_j 1 x kind::tf32: the rank-one mean term of Eq. 6
+//   warps 4-7     softmax warpgroup of tile 0, one thread per query row (128 scores in
+//   warps 8-11    registers); likewise tile 1.  Running max, alpha, ExpCast-FP8 codes by
+//                 fma.sat + magic-number rounding (Eq. 7: no exponential, no conversion), row
+//                 sum of the decoded codes, l; writes the code tile in the 128-byte-swizzled
+//                 K-major layout the tensor core reads, and the output at the end
+//   warps 12-15   correction warpgroup of tile 0 (16-19: tile 1): rescales A_t by alpha when
+//                 a row maximum moved
+//
+// Tensor memory (512 columns): S_0 | S_1 | A_0 | A_1, 128 columns each.
+constexpr int kStages2 = 4;
+constexpr uint32_t kWaitLimit2 = 1u << 18;   // x up to 4 us per try: about one second
+
+struct FaSmem {
+  uint64_t q_full, kv_full[kStages2], kv_empty[kStages2];
+  uint64_t s_full[2], s_free[2], o_done[2];
+  // alpha and codes+correction hand-offs can run one key tile ahead of their consumer (the score
+  // tile of j+1 is ready before the codes of j are consumed), so they alternate between two barriers
+  uint64_t a_full[2][2], pc_full[2][2];
+  float alpha[2][128];
+  uint32_t tmem_base;
+  volatile int abort;
+};
+
+__device__ __forceinline__ bool wait2(uint64_t* bar, uint32_t parity, FaSmem* sh, uint32_t* status, uint32_t code) {
+  if (mbar_try_wait(bar, parity)) return true;
+  for (uint32_t i = 0; i < kWaitLimit2; ++i) {
+    if (mbar_try_wait_hint(bar, parity, 4000u)) return true;
+    if ((i & 63u) == 63u && sh->abort) return false;
+  }
+  sh->abort = 1;
+  atomicExch(status, kErrTimeout | code);
+  return false;
+}
+__device__ __forceinline__ bool warp_wait2(uint64_t* bar, uint32_t parity, FaSmem* sh, uint32_t* status, uint32_t code) {
+  return __all_sync(0xffffffffu, wait2(bar, parity, sh, status, code));
+}
+
+template <int D, bool EXPCAST>
+__global__ void __launch_bounds__(640, 1)
+attn_fwd_2q_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
+                   const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_mu,
+                   const AttnArgs a) {
+  constexpr int kTmemCols = 512;
+  // Register re-partition (setmaxnreg): the CTA owns 640 x 96 registers; a warpgroup that asks for
+  // more than the others released would block forever, so the budget is checked at compile time.
+  constexpr int kRegCtl = 48, kRegSoftmax = 160, kRegCorr = 56;
+  static_assert(kRegCtl + 2 * kRegSoftmax + 2 * kRegCorr <= 5 * 96, "register budget exceeds the CTA's allocation");
+  constexpr uint32_t kQBytes = 128 * D, kKBytes = 128 * D, kVBytes = D * 128, kMuBytes = D * 32;
+  constexpr uint32_t kStageBytes = kKBytes + kVBytes + ((kMuBytes + 1023) / 1024) * 1024;
+  constexpr uint32_t kPBytes = 128 * 128, kAmBytes = 128 * 32;
+  extern __shared__ unsigned char smem_raw[];
+  unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  unsigned char* sQ = smem;                                    // [2][128 x D]
+  unsigned char* sP = smem + 2 * kQBytes;                      // [2][128 x 128] probability codes
+  unsigned char* sAm = sP + 2 * kPBytes;                       // [2][128 x 8 fp32] row-sum pairs
+  unsigned char* sStage = sAm + 2 * kAmBytes;                  // [kStages2]{K, V, Mu}
+  FaSmem* sh = reinterpret_cast<FaSmem*>(sStage + kStages2 * kStageBytes);
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int qpair = blockIdx.x, bh = blockIdx.y;
+  const int nb = a.nb;
+
+  if (tid == 0) {
+    mbar_init(&sh->q_full, 1);
+    for (int i = 0; i < kStages2; ++i) { mbar_init(&sh->kv_full[i], 1); mbar_init(&sh->kv_empty[i], 2); }
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(&sh->s_full[i], 1); mbar_init(&sh->s_free[i], 128); mbar_init(&sh->o_done[i], 1);
+      for (int b = 0; b < 2; ++b) { mbar_init(&sh->a_full[i][b], 128); mbar_init(&sh->pc_full[i][b], 256); }
+    }
+    sh->abort = 0;
+    mbar_fence_init();
+    tma_prefetch_desc(&tm_q); tma_prefetch_desc(&tm_k); tma_prefetch_desc(&tm_v); tma_prefetch_desc(&tm_mu);
+  }
+  for (int i = tid; i < 2 * (int)kAmBytes / 16; i += 640) reinterpret_cast<uint4*>(sAm)[i] = make_uint4(0, 0, 0, 0);
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy stores -> tensor-core reads
+  if (warp == 2) { tmem_alloc<kTmemCols>(&sh->tmem_base); tmem_relinquish(); }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = sh->tmem_base;
+  const uint32_t lane_base = tmem + ((uint32_t)((warp & 3) * 32) << 16);
+
+  if (warp < 4) {
+    reg_dec<kRegCtl>();
+    if (warp == 0) {
+      // ------------------------------------------------------------------ TMA producer
+      // (the whole warp runs the loop; one elected lane issues the copies)
+      if (elect_one()) {
+        mbar_expect_tx(&sh->q_full, 2 * kQBytes);
+        tma_load_3d(sQ, &tm_q, &sh->q_full, 0, (2 * qpair) * 128, bh);
+        tma_load_3d(sQ + kQBytes, &tm_q, &sh->q_full, 0, (2 * qpair + 1) * 128, bh);   // past the end: zero fill
+      }
+      for (int j = 0; j < nb; ++j) {
+        const int st = j % kStages2, it = j / kStages2;
+        unsigned char* base = sStage + st * kStageBytes;
+        if (!warp_wait2(&sh->kv_empty[st], (it & 1) ^ 1, sh, a.status, 11)) break;
+        if (elect_one()) {
+          mbar_expect_tx(&sh->kv_full[st], kKBytes + kVBytes + kMuBytes);
+          tma_load_3d(base, &tm_k, &sh->kv_full[st], 0, j * 128, bh);
+          tma_load_3d(base + kKBytes, &tm_v, &sh->kv_full[st], j * 128, 0, bh);
+          tma_load_3d(base + kKBytes + kVBytes, &tm_mu, &sh->kv_full[st], 0, 0, bh * nb + j);
+        }
+        __syncwarp();
+      }
+    } else if (warp == 1 || warp == 3) {
+      // ------------------------------------------------------------------ MMA issuers
+      // One warp per query tile (they sit on different schedulers).  Every wait on the way to an
+      // MMA is a shared-memory round trip, so each issuer waits for as little as possible: per key
+      // tile one barrier before S_t(j+1) and one before the A_t update.  The whole warp runs the
+      // loop so that descriptors stay in uniform registers; one elected lane issues.
+      const int t = warp >> 1;
+      const uint32_t idesc_qk = idesc_e4m3(128, 128), idesc_pv = idesc_e4m3(128, D), idesc_mu = idesc_tf32(128, D);
+      const uint64_t dq = smem_desc_kmajor(smem_u32(sQ + t * kQBytes), D);
+      const uint64_t dp = smem_desc_kmajor(smem_u32(sP + t * kPBytes), 128);
+      const uint64_t dam = smem_desc_kmajor(smem_u32(sAm + t * kAmBytes), 32);
+      const uint32_t s_col = tmem + 128 * t, o_col = tmem + 256 + 128 * t;
+      bool ok = warp_wait2(&sh->q_full, 0, sh, a.status, 20) && warp_wait2(&sh->kv_full[0], 0, sh, a.status, 21);
+      if (ok && elect_one()) {
+        tc_fence_after();
+        const uint64_t dk = smem_desc_kmajor(smem_u32(sStage), D);
+#pragma unroll
+        for (int k = 0; k < D / 32; ++k) mma_f8_ss(s_col, dq + 2 * k, dk + 2 * k, idesc_qk, k > 0);
+        mma_commit(&sh->s_full[t]);
+      }
+      __syncwarp();
+      for (int j = 0; ok && j < nb; ++j) {
+        const int st = j % kStages2;
+        if (j + 1 < nb) {                                 // S_t(j+1), as soon as the scores of (t, j) were read
+          const int st1 = (j + 1) % kStages2, it1 = (j + 1) / kStages2;
+          if (!(ok = warp_wait2(&sh->s_free[t], j & 1, sh, a.status, 22))) break;
+          if (!(ok = warp_wait2(&sh->kv_full[st1], it1 & 1, sh, a.status, 25))) break;
+          const uint64_t dk = smem_desc_kmajor(smem_u32(sStage + st1 * kStageBytes), D);
+          if (elect_one()) {
+            tc_fence_after();
+#pragma unroll
+            for (int k = 0; k < D / 32; ++k) mma_f8_ss(s_col, dq + 2 * k, dk + 2 * k, idesc_qk, k > 0);
+            mma_commit(&sh->s_full[t]);
+          }
+          __syncwarp();
+        }
+        // A_t += P^_t(j) R^_j + r mu~_j, once the codes are written and A_t is rescaled
+        if (!(ok = warp_wait2(&sh->pc_full[t][j & 1], (j >> 1) & 1, sh, a.status, 23))) break;
+        unsigned char* base = sStage + st * kStageBytes;
+        const uint64_t dv = smem_desc_kmajor(smem_u32(base + kKBytes), 128);
+        const uint64_t dm = smem_desc_kmajor(smem_u32(base + kKBytes + kVBytes), 32);
+        if (elect_one()) {
+          tc_fence_after();
+#pragma unroll
+          for (int k = 0; k < 4; ++k) mma_f8_ss(o_col, dp + 2 * k, dv + 2 * k, idesc_pv, (j > 0) | (k > 0));
+          mma_tf32_ss(o_col, dam, dm, idesc_mu, 1);
+          mma_commit(&sh->o_done[t]);
+          mma_commit(&sh->kv_empty[st]);                  // this tile is done with stage j
+        }
+        __syncwarp();
+      }
+    }
+  } else if (warp < 12) {
+    // -------------------------------------------------------------------- softmax warpgroups
+    reg_inc<kRegSoftmax>();
+    const int t = (warp - 4) >> 2;                         // query tile of this warpgroup
+    const int row = (warp & 3) * 32 + lane;
+    const int qblk = 2 * qpair + t;
+    const uint32_t s_base = lane_base + 128 * t, o_base = lane_base + 256 + 128 * t;
+    // my row of the swizzled code tile: 16-byte chunk c sits at chunk position c ^ (row % 8)
+    unsigned char* p_row = sP + t * kPBytes + (row >> 3) * 1024 + (row & 7) * 128;
+    // my row of the row-sum operand: 32-byte rows, the two 16-byte chunks swap when (row / 4) is odd
+    uint4* am_row = reinterpret_cast<uint4*>(sAm + t * kAmBytes + row * 32 + 16 * ((row >> 2) & 1));
+    const float sq = qblk < nb ? a.q_scale[(size_t)bh * nb + qblk] : 1.0f;
+    float m_run = -INFINITY, l_run = 0.f;
+    bool ok = true;
+    for (int j = 0; j < nb; ++j) {
+      const int ph = j & 1;
+      const float cs = (sq * __ldg(&a.k_scale[(size_t)bh * nb + j])) * a.sl;
+      if (!(ok = warp_wait2(&sh->s_full[t], ph, sh, a.status, 30))) break;
+      tc_fence_after();
+      uint32_t s0[32], s1[32], s2[32], s3[32];
+      tmem_ld32(s_base, s0); tmem_ld32(s_base + 32, s1); tmem_ld32(s_base + 64, s2); tmem_ld32(s_base + 96, s3);
+      tmem_wait_ld();
+      tc_fence_before();
+      mbar_arrive(&sh->s_free[t]);                        // the score columns may be overwritten
+      const int nv = a.N - j * 128;                       // >= 128 except on the ragged last tile
+      if (nv < 128) {                                     // padded keys never win the maximum
+#pragma unroll
+        for (int i = 0; i < 32; ++i) {
+          if (i >= nv) s0[i] = 0xff800000u;
+          if (32 + i >= nv) s1[i] = 0xff800000u;
+          if (64 + i >= nv) s2[i] = 0xff800000u;
+          if (96 + i >= nv) s3[i] = 0xff800000u;
+        }
+      }
+      float mx[8];
+#pragma unroll
+      for (int c = 0; c < 2; ++c) {
+        mx[c] = max3(__uint_as_float(s0[16 * c]), __uint_as_float(s0[16 * c + 1]), __uint_as_float(s0[16 * c + 2]));
+        mx[2 + c] = max3(__uint_as_float(s1[16 * c]), __uint_as_float(s1[16 * c + 1]), __uint_as_float(s1[16 * c + 2]));
+        mx[4 + c] = max3(__uint_as_float(s2[16 * c]), __uint_as_float(s2[16 * c + 1]), __uint_as_float(s2[16 * c + 2]));
+        mx[6 + c] = max3(__uint_as_float(s3[16 * c]), __uint_as_float(s3[16 * c + 1]), __uint_as_float(s3[16 * c + 2]));
+#pragma unroll
+        for (int i = 3; i < 15; i += 2) {
+          mx[c] = max3(mx[c], __uint_as_float(s0[16 * c + i]), __uint_as_float(s0[16 * c + i + 1]));
+          mx[2 + c] = max3(mx[2 + c], __uint_as_float(s1[16 * c + i]), __uint_as_float(s1[16 * c + i + 1]));
+          mx[4 + c] = max3(mx[4 + c], __uint_as_float(s2[16 * c + i]), __uint_as_float(s2[16 * c + i + 1]));
+          mx[6 + c] = max3(mx[6 + c], __uint_as_float(s3[16 * c + i]), __uint_as_float(s3[16 * c + i + 1]));
+        }
+        mx[c] = fmaxf(mx[c], __uint_as_float(s0[16 * c + 15]));
+        mx[2 + c] = fmaxf(mx[2 + c], __uint_as_float(s1[16 * c + 15]));
+        mx[4 + c] = fmaxf(mx[4 + c], __uint_as_float(s2[16 * c + 15]));
+        mx[6 + c] = fmaxf(mx[6 + c], __uint_as_float(s3[16 * c + 15]));
+      }
+      const float mxa = (a.debug & 8) ? __uint_as_float(s0[0]) : max3(max3(mx[0], mx[1], mx[2]), max3(mx[3], mx[4], mx[5]), fmaxf(mx[6], mx[7]));
+      const float m_new = fmaxf(m_run, mxa * cs);         // m' = max(m, rowmax S_ij)
+      const float alpha = ex2_approx(m_run - m_new);      // 0 on the first tile
+      sh->alpha[t][row] = alpha;
+      mbar_arrive(&sh->a_full[t][j & 1]);
+      m_run = m_new;
+      // the previous code tile must have been consumed before it is overwritten
+      if (j > 0 && !(a.debug & 32) && !(ok = warp_wait2(&sh->o_done[t], (j - 1) & 1, sh, a.status, 31))) break;
+
+      float acc0 = 0.f, acc1 = 0.f, acc2 = 0.f, acc3 = 0.f;
+      const float fa = cs * 0.0625f, fb = (a.code_off - 8.0f * m_new) * 0.0078125f, nm = 8.0f - m_new;
+      auto code4 = [&](const uint32_t (&sv)[32], int w) -> uint32_t {
+        if constexpr (EXPCAST) {
+          // Eq. 7 in two FMAs: t = sat((8 u + 120 + beta) / 128) clips to [0, 1], then
+          // t * 128 + 1.5 * 2^23 rounds to the nearest even integer in the low mantissa bits.
+          const uint32_t r0 = __float_as_uint(fmaf(fma_sat(__uint_as_float(sv[4 * w]), fa, fb), 128.0f, 12582912.0f));
+          const uint32_t r1 = __float_as_uint(fmaf(fma_sat(__uint_as_float(sv[4 * w + 1]), fa, fb), 128.0f, 12582912.0f));
+          const uint32_t r2 = __float_as_uint(fmaf(fma_sat(__uint_as_float(sv[4 * w + 2]), fa, fb), 128.0f, 12582912.0f));
+          const uint32_t r3 = __float_as_uint(fmaf(fma_sat(__uint_as_float(sv[4 * w + 3]), fa, fb), 128.0f, 12582912.0f));
+          // (code << 20) read as fp32 is the decoded E4M3 value times 2^-120, subnormal codes included
+          acc0 += __uint_as_float(r0 << 20); acc1 += __uint_as_float(r1 << 20);
+          acc2 += __uint_as_float(r2 << 20); acc3 += __uint_as_float(r3 << 20);
+          return __byte_perm(__byte_perm(r0, r1, 0x0040), __byte_perm(r2, r3, 0x0040), 0x5410);
+        } else {
+          // exponentiate, then cast (Fig. 4a upper box)
+          const float p0 = exp2f(fmaf(__uint_as_float(sv[4 * w]), cs, nm)), p1 = exp2f(fmaf(__uint_as_float(sv[4 * w + 1]), cs, nm));
+          const float p2 = exp2f(fmaf(__uint_as_float(sv[4 * w + 2]), cs, nm)), p3 = exp2f(fmaf(__uint_as_float(sv[4 * w + 3]), cs, nm));
+          const uint32_t lo = __nv_cvt_float2_to_fp8x2(make_float2(p0, p1), __NV_SATFINITE, __NV_E4M3);
+          const uint32_t hi = __nv_cvt_float2_to_fp8x2(make_float2(p2, p3), __NV_SATFINITE, __NV_E4M3);
+          acc0 += __uint_as_float((lo & 0xffu) << 20); acc1 += __uint_as_float((lo >> 8) << 20);
+          acc2 += __uint_as_float((hi & 0xffu) << 20); acc3 += __uint_as_float((hi >> 8) << 20);
+          return lo | (hi << 16);
+        }
+      };
+      auto store16 = [&](const uint32_t (&sv)[32], int half, int chunk) {   // keys 16*chunk .. +15
+        const uint4 v = make_uint4(code4(sv, 4 * half), code4(sv, 4 * half + 1), code4(sv, 4 * half + 2), code4(sv, 4 * half + 3));
+        *reinterpret_cast<uint4*>(p_row + ((chunk ^ (row & 7)) << 4)) = v;
+      };
+      if (a.debug & 2) {
+#pragma unroll
+        for (int c = 0; c < 8; ++c) *reinterpret_cast<uint4*>(p_row + (c << 4)) = make_uint4(s0[c] & 0x38383838u, s1[c] & 0x38383838u, s2[c] & 0x38383838u, s3[c] & 0x38383838u);
+        acc0 = 1e-30f;
+      } else {
+      store16(s0, 0, 0); store16(s0, 1, 1); store16(s1, 0, 2); store16(s1, 1, 3);
+      store16(s2, 0, 4); store16(s2, 1, 5); store16(s3, 0, 6); store16(s3, 1, 7);
+      }
+      const float rs = (((acc0 + acc1) + (acc2 + acc3)) * 1152921504606846976.0f) * 1152921504606846976.0f;   // x 2^120
+      l_run = alpha * l_run + rs;                         // l <- alpha l + r,  r = P~ 1 over the decoded codes
+      const uint32_t hi = (__float_as_uint(rs) + 0x1000u) & 0xffffe000u;     // nearest TF32
+      *am_row = make_uint4(hi, __float_as_uint(rs - __uint_as_float(hi)), 0u, 0u);
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");          // my stores -> tensor-core reads
+      mbar_arrive(&sh->pc_full[t][j & 1]);
+    }
+    // ---- epilogue: O = s_V * A / l
+    if (ok && warp_wait2(&sh->o_done[t], (nb - 1) & 1, sh, a.status, 33)) {
+      tc_fence_after();
+      const int grow = qblk * 128 + row;
+      const float inv_l = 1.0f / l_run;
+      uint32_t r[32];
+#pragma unroll 1
+      for (int c = 0; c < D / 32; ++c) {
+        tmem_ld32(o_base + 32 * c, r);
+        tmem_wait_ld();
+        if (grow < a.N) {
+          uint32_t out[16];
+#pragma unroll
+          for (int i = 0; i < 16; ++i) {
+            const float x0 = __uint_as_float(r[2 * i]) * inv_l * __ldg(&a.v_scale[(size_t)bh * D + 32 * c + 2 * i]);
+            const float x1 = __uint_as_float(r[2 * i + 1]) * inv_l * __ldg(&a.v_scale[(size_t)bh * D + 32 * c + 2 * i + 1]);
+            __nv_bfloat162 h2 = __floats2bfloat162_rn(x0, x1);
+            out[i] = *reinterpret_cast<uint32_t*>(&h2);
+          }
+          uint4* dst = reinterpret_cast<uint4*>(a.o + ((size_t)bh * a.N + grow) * D + 32 * c);
+#pragma unroll
+          for (int i = 0; i < 4; ++i) dst[i] = make_uint4(out[4 * i], out[4 * i + 1], out[4 * i + 2], out[4 * i + 3]);
+        }
+      }
+    }
+  } else {
+    // -------------------------------------------------------------------- correction warpgroups
+    reg_dec<kRegCorr>();
+    const int t = (warp - 12) >> 2;
+    const int row = (warp & 3) * 32 + lane;
+    const uint32_t o_base = lane_base + 256 + 128 * t;
+    for (int j = 0; j < nb; ++j) {
+      const int ph = j & 1;
+      if (!warp_wait2(&sh->a_full[t][j & 1], (j >> 1) & 1, sh, a.status, 40)) break;
+      const float alpha = sh->alpha[t][row];
+      if (j > 0 && !(a.debug & 1) && __any_sync(0xffffffffu, alpha != 1.0f)) {
+        if (!warp_wait2(&sh->o_done[t], (j - 1) & 1, sh, a.status, 41)) break;
+        tc_fence_after();
+        uint32_t r[32];
+#pragma unroll 1
+        for (int c = 0; c < D / 32; ++c) {
+          tmem_ld32(o_base + 32 * c, r);
+          tmem_wait_ld();
+#pragma unroll
+          for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * alpha);
+          tmem_st32(o_base + 32 * c, r);
+        }
+        tmem_wait_st();
+        tc_fence_before();
+      }
+      mbar_arrive(&sh->pc_full[t][j & 1]);
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 2) tmem_dealloc<kTmemCols>(tmem);
+}
+
+// Block means as the B operand of the per-tile mean-restoration MMA: per (b, h, key tile) a
+// [d][8] fp32 tile with entry [c][0] = [c][1] = mu~[c] (for r_hi and r_lo) and zeros elsewhere.
+template <int D>
+__global__ void means_tile_layout_kernel(const __nv_bfloat16* __restrict__ means, float* __restrict__ out, size_t n) {
+  const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;   // (bh * nb + tile) * D + c
+  if (i >= n) return;
+  const float v = __bfloat162float(means[i]);
+  float4* dst = reinterpret_cast<float4*>(out + i * 8);
+  dst[0] = make_float4(v, v, 0.f, 0.f);
+  dst[1] = make_float4(0.f, 0.f, 0.f, 0.f);
+}
+
 // ---------------------------------------------------------------------------------------
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -572,6 +939,7 @@ cudaError_t run8(const Problem& pr, const QuantLayout& ql, const WorkLayout& wl,
   a.N = pr.N; a.n_pad = pr.n_pad; a.nb = pr.nb; a.ng = ng; a.p_format = pr.p_format;
   a.sl = pr.softmax_scale * 1.4426950408889634f;
   a.code_off = 120.0f + pr.beta;
+  { const char* dbg = getenv("VC_DEBUG"); a.debug = dbg ? atoi(dbg) : 0; }
   cudaError_t e;
   if (pr.kernel_variant == 1) {     // serial reference kernel
     const size_t smem = 1024 + 2 * 128 * D + D * 128 + D * 4 + 64;
@@ -580,20 +948,40 @@ cudaError_t run8(const Problem& pr, const QuantLayout& ql, const WorkLayout& wl,
     count_launches(1);
     return cudaGetLastError();
   }
+  if (pr.kernel_variant == 0) {     // two query tiles per CTA (default)
+    alignas(64) CUtensorMap tmt;
+    if (!make_map(&tmt, work + wl.mu_mma, 32, D, (uint64_t)pr.BH * pr.nb, 32, D)) return cudaErrorUnknown;
+    const size_t n = (size_t)pr.BH * pr.nb * D;
+    means_tile_layout_kernel<D><<<(unsigned)((n + 255) / 256), 256, 0, s>>>(a.v_means, (float*)(work + wl.mu_mma), n);
+    const size_t stage = 2 * 128 * D + ((D * 32 + 1023) / 1024) * 1024;
+    const size_t smem2 = 1024 + 2 * 128 * D + 2 * 128 * 128 + 2 * 128 * 32 + kStages2 * stage + sizeof(FaSmem);
+    const dim3 grid((pr.nb + 1) / 2, pr.BH);
+    if (pr.p_format == VC_P_EXPCAST_E4M3) {
+      if ((e = cudaFuncSetAttribute(attn_fwd_2q_kernel<D, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem2)) != cudaSuccess) return e;
+      attn_fwd_2q_kernel<D, true><<<grid, 640, smem2, s>>>(tq, tk, tv, tmt, a);
+    } else {
+      if ((e = cudaFuncSetAttribute(attn_fwd_2q_kernel<D, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem2)) != cudaSuccess) return e;
+      attn_fwd_2q_kernel<D, false><<<grid, 640, smem2, s>>>(tq, tk, tv, tmt, a);
+    }
+    count_launches(2);
+    return cudaGetLastError();
+  }
   means_mma_layout_kernel<D><<<dim3(ng, pr.BH), D, 0, s>>>(a.v_means, (float*)(work + wl.mu_mma), pr.nb, ng);
   const size_t smem = 1024 + (size_t)(1 + 2 * kStages + 2) * 128 * D + sizeof(PipeSmem);
   if (pr.p_format == VC_P_EXPCAST_E4M3) {
     if ((e = cudaFuncSetAttribute(attn_fwd_pipe_kernel<D, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
-    attn_fwd_pipe_kernel<D, true><<<dim3(pr.nb, pr.BH), 384, smem, s>>>(tq, tk, tv, tmu, a);
+    attn_fwd_pipe_kernel<D, true><<<dim3(pr.nb, pr.BH), 768, smem, s>>>(tq, tk, tv, tmu, a);
   } else {
     if ((e = cudaFuncSetAttribute(attn_fwd_pipe_kernel<D, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
-    attn_fwd_pipe_kernel<D, false><<<dim3(pr.nb, pr.BH), 384, smem, s>>>(tq, tk, tv, tmu, a);
+    attn_fwd_pipe_kernel<D, false><<<dim3(pr.nb, pr.BH), 768, smem, s>>>(tq, tk, tv, tmu, a);
   }
   count_launches(2);
   return cudaGetLastError();
 }
 
 }  // namespace
+
+extern "C" int vc_debug_trace(long long* host) { return (int)cudaMemcpyFromSymbol(host, g_trace, sizeof(long long) * 8192); }
 
 cudaError_t launch_attn_fwd(const Problem& pr, const QuantLayout& ql, const WorkLayout& wl,
                             const uint8_t* quant, void* o, uint8_t* work, cudaStream_t stream) {
