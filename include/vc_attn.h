@@ -78,9 +78,9 @@ typedef struct {
   int64_t stride_b, stride_h, stride_n;       /* of Q, K and V, in elements; 0 => packed */
   int32_t heads_per_pass;           /* heads preprocessed per launch group (L2 reuse of
                                        the second read of K and V); 0 => library default */
-  int32_t kernel_variant;           /* attention kernel: 0 = two query tiles per CTA
-                                       (default); 1 = simple serial kernel; 2 = one query
-                                       tile per CTA, pipelined; 1 and 2 are kept for A/B  */
+  int32_t kernel_variant;           /* attention kernel: 0 = pipelined, two query tiles per
+                                       CTA (default); 1 = simple serial kernel, kept for
+                                       A/B measurement and cross-checks                  */
 } vc_params;
 
 /* Device pointers into the quantized bundle written by vc_prep (N_pad = 128*ceil(N/128),

@@ -57,7 +57,7 @@ vc_status resolve(const vc_params* p, Problem* out) {
   pr.nb = pr.n_pad / kBlock;
   pr.heads_per_pass = p->heads_per_pass > 0 ? p->heads_per_pass : 0;
   pr.kernel_variant = p->kernel_variant;
-  if (pr.kernel_variant < 0 || pr.kernel_variant > 2) return VC_ERR_INVALID_ARG;
+  if (pr.kernel_variant < 0 || pr.kernel_variant > 1) return VC_ERR_INVALID_ARG;
   *out = pr;
   return VC_OK;
 }
@@ -109,7 +109,7 @@ WorkLayout work_layout(const Problem& pr) {
   W.v_mu = place(BH * nb * d * 4);
   W.amax_bytes = BH * d * 4 + 2 * BH * 4;
   W.amax = place(W.amax_bytes);
-  W.mu_mma = place(BH * nb * d * 32);   // >= the grouped layout BH * ceil(nb/16) * d * 128
+  W.mu_mma = place(BH * nb * d * 32);
   W.total = off;
   return W;
 }

@@ -1,18 +1,17 @@
 // Quantized attention forward of VC-Attention for sm_100a (Eq. 1, Eq. 6, Eq. 7).
 //
-// One CTA owns one 128-row query tile of one (batch, head) and streams the permuted
-// key/value tiles of 128 tokens through it:
-//   TMA (cp.async.bulk.tensor, 128-byte swizzle)  K^_j, R^_j  -> shared memory
-//   tcgen05.mma kind::f8f6f4 (E4M3 x E4M3, FP32)  S = Q^ K^_j^T -> tensor memory
-//   softmax stage, one thread per query row        running max, alpha, ExpCast-FP8 code
-//                                                  (one FMA + round, no exponential)
-//   P^ codes -> tensor memory (A operand)          tcgen05.st
-//   tcgen05.mma                                    A += P^ R^_j
-//   mean restoration                               A = alpha A + r mu~_j  (Eq. 6)
-// Epilogue: O = s_V * A / l, bf16, original query order.
+// Two kernels share the arithmetic:
+//   attn_fwd_2q_kernel      the default: warp-specialized, two 128-row query tiles per CTA,
+//                           TMA ring for K^/R^ tiles, tcgen05 MMAs with accumulators in tensor
+//                           memory, ExpCast-FP8 softmax warpgroups, correction warpgroups
+//                           (described in front of the kernel)
+//   attn_fwd_serial_kernel  one query tile per CTA, every step in program order behind
+//                           __syncthreads; kept as an independent cross-check and for A/B timing
+// Both read the bundle vc_prep writes: E4M3 codes of Q (query order), K (permuted order, row
+// major) and the V residual (channel-major), per-block scales, per-channel value scale and the
+// block means divided by it.  Epilogue: O = s_V * A / l, bf16, original query order.
 #include <cuda_bf16.h>
 #include <cuda_fp8.h>
-#include <cstdlib>
 
 #include "vc_internal.h"
 #include "vc_sm100.cuh"
@@ -29,8 +28,7 @@ struct AttnArgs {
   const __nv_bfloat16* v_means;
   __nv_bfloat16* o;
   uint32_t* status;
-  int debug;
-  int N, n_pad, nb, ng, p_format;   // ng = groups of 16 key tiles
+  int N, n_pad, nb, p_format;
   float sl;        // softmax_scale * log2(e)
   float code_off;  // 120 + beta  (Eq. 7)
 };
@@ -41,6 +39,8 @@ __device__ __forceinline__ float decode_pos_e4m3(uint32_t code) {
   return code >= 8u ? __uint_as_float((code + 960u) << 20) : (float)code * 0.001953125f;
 }
 
+// Serial kernel: TMA -> S = Q^ K^_j^T -> one thread per row (max, alpha, codes, row sum) ->
+// P^ to tensor memory -> A = alpha A + r mu~_j on CUDA cores -> A += P^ R^_j, tile after tile.
 template <int D>
 __global__ void __launch_bounds__(128)
 attn_fwd_serial_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
@@ -210,336 +210,6 @@ attn_fwd_serial_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
   if (warp == 0) tmem_dealloc<kTmemCols>(tmem);
 }
 
-
-// ---------------------------------------------------------------------------------------
-// Pipelined, warp-specialized kernel.  One CTA per SM-resident 128-row query tile:
-//
-//   warp 0      TMA producer: Q once, then K^_j / R^_j tiles through a 3-stage ring, and one
-//               block-mean table per group of 16 key tiles
-//   warp 1      MMA issuer (one thread): S[j&1] = Q^ K^_j^T is issued one tile ahead of
-//               A += P^_{j-1} R^_{j-1}, so the tensor core works on the next scores while the
-//               softmax stage turns the current ones into codes
-//   warps 4-19  softmax stage, four threads per query row (32 key columns each): running
-//               max, alpha, ExpCast-FP8 code (fma.sat + magic-number round, no exponential),
-//               P^ -> TMEM
-//   warps 20-23 correction stage, one thread per row: rescales A by alpha when the running
-//               maximum moved, owns l, and keeps the per-tile row sums r_ij (referenced to
-//               the current maximum) in TMEM as a TF32 hi/lo pair
-//
-// Mean restoration (Eq. 6) is deferred: every 16 tiles one small kind::tf32 MMA adds
-// sum_j r_ij mu~_j to the same accumulator, [128 x 32] (row sums, hi/lo) x [d x 32] (means).
-__device__ long long g_trace[8192];
-#define TRACE(ev, jj) do { if ((a.debug & 4) && ((threadIdx.x & 31) == 0 || ((ev) >= 14 && (ev) <= 17)) && blockIdx.x == 5 && blockIdx.y == 0 && (jj) >= 40 && (jj) < 48) { g_trace[((ev) * 8 + ((jj) - 40))] = clock64(); } } while (0)
-constexpr int kStages = 3;
-constexpr int kGroup = 16;          // key tiles per mean-restoration MMA
-constexpr uint32_t kWaitLimit = 1u << 21;
-
-struct PipeSmem {
-  uint64_t q_full, k_full[kStages], v_full[kStages], kv_empty[kStages];
-  uint64_t pm_full[2][4];
-  uint64_t s_full[2], a_full[2], p_full[2], c_done[2], o_done[2], g_done[2], mu_full[2], mu_empty[2];
-  float alpha[2][128];
-  float pmax[2][4][128];
-  float rsum[2][4][128];
-  uint32_t tmem_base;
-  volatile int abort;
-};
-
-__device__ __forceinline__ bool wait_or_abort(uint64_t* bar, uint32_t parity, PipeSmem* sh, uint32_t* status, uint32_t code) {
-  for (uint32_t i = 0; i < kWaitLimit; ++i) {
-    if (mbar_try_wait(bar, parity)) return true;
-    if ((i & 255u) == 255u && sh->abort) return false;
-  }
-  sh->abort = 1;
-  atomicExch(status, kErrTimeout | code);
-  return false;
-}
-
-// Warp-uniform variant for the stages that execute .sync.aligned instructions afterwards.
-__device__ __forceinline__ bool warp_wait(uint64_t* bar, uint32_t parity, PipeSmem* sh, uint32_t* status, uint32_t code) {
-  return __all_sync(0xffffffffu, wait_or_abort(bar, parity, sh, status, code));
-}
-
-template <int D, bool EXPCAST>
-__global__ void __launch_bounds__(768, 1)
-attn_fwd_pipe_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
-                     const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_mu,
-                     const AttnArgs a) {
-  constexpr int kTmemCols = 512;
-  constexpr uint32_t S_COL = 0, O_COL = 256, R_COL = 384;
-  constexpr uint32_t kTileBytes = 128 * D;
-  extern __shared__ unsigned char smem_raw[];
-  unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  unsigned char* sQ = smem;
-  unsigned char* sK = smem + kTileBytes;                       // [kStages][128 x D]
-  unsigned char* sV = sK + kStages * kTileBytes;               // [kStages][D x 128]
-  unsigned char* sMu = sV + kStages * kTileBytes;              // [2][D x 32 fp32]
-  PipeSmem* sh = reinterpret_cast<PipeSmem*>(sMu + 2 * kTileBytes);
-
-  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int qblk = blockIdx.x, bh = blockIdx.y;
-  const int nb = a.nb;
-
-  if (tid == 0) {
-    mbar_init(&sh->q_full, 1);
-    for (int i = 0; i < kStages; ++i) { mbar_init(&sh->k_full[i], 1); mbar_init(&sh->v_full[i], 1); mbar_init(&sh->kv_empty[i], 1); }
-    for (int i = 0; i < 2; ++i) {
-      mbar_init(&sh->s_full[i], 1); mbar_init(&sh->a_full[i], 128); mbar_init(&sh->p_full[i], 512);
-      mbar_init(&sh->c_done[i], 128); mbar_init(&sh->o_done[i], 1); mbar_init(&sh->g_done[i], 128);
-      mbar_init(&sh->mu_full[i], 1); mbar_init(&sh->mu_empty[i], 1);
-      for (int w = 0; w < 4; ++w) mbar_init(&sh->pm_full[i][w], 128);
-    }
-    sh->abort = 0;
-    mbar_fence_init();
-    tma_prefetch_desc(&tm_q); tma_prefetch_desc(&tm_k); tma_prefetch_desc(&tm_v); tma_prefetch_desc(&tm_mu);
-  }
-  if (warp == 2) { tmem_alloc<kTmemCols>(&sh->tmem_base); tmem_relinquish(); }
-  tc_fence_before();
-  __syncthreads();
-  tc_fence_after();
-  const uint32_t tmem = sh->tmem_base;
-  const uint32_t lane_base = tmem + ((uint32_t)((warp & 3) * 32) << 16);
-
-  if (warp < 4) {
-    if (warp == 0 && lane == 0) {
-      // ------------------------------------------------------------------ TMA producer
-      mbar_expect_tx(&sh->q_full, kTileBytes);
-      tma_load_3d(sQ, &tm_q, &sh->q_full, 0, qblk * 128, bh);
-      for (int j = 0; j < nb; ++j) {
-        const int st = j % kStages, it = j / kStages;
-        if (j % kGroup == 0) {
-          const int g = j / kGroup;
-          if (!wait_or_abort(&sh->mu_empty[g & 1], ((g >> 1) & 1) ^ 1, sh, a.status, 10)) break;
-          mbar_expect_tx(&sh->mu_full[g & 1], kTileBytes);
-          tma_load_3d(sMu + (g & 1) * kTileBytes, &tm_mu, &sh->mu_full[g & 1], 0, 0, bh * a.ng + g);
-        }
-        if (!wait_or_abort(&sh->kv_empty[st], (it & 1) ^ 1, sh, a.status, 11)) break;
-        mbar_expect_tx(&sh->k_full[st], kTileBytes);
-        tma_load_3d(sK + st * kTileBytes, &tm_k, &sh->k_full[st], 0, j * 128, bh);
-        mbar_expect_tx(&sh->v_full[st], kTileBytes);
-        tma_load_3d(sV + st * kTileBytes, &tm_v, &sh->v_full[st], j * 128, 0, bh);
-        TRACE(0, j);
-      }
-    } else if (warp == 1 && lane == 0) {
-      // ------------------------------------------------------------------ MMA issuer
-      const uint32_t idesc_qk = idesc_e4m3(128, 128), idesc_pv = idesc_e4m3(128, D), idesc_mu = idesc_tf32(128, D);
-      const uint64_t dq = smem_desc_kmajor(smem_u32(sQ), D);
-      bool ok = wait_or_abort(&sh->q_full, 0, sh, a.status, 20);
-      for (int j = 0; ok && j <= nb; ++j) {
-        if (j < nb) {
-          const int st = j % kStages, it = j / kStages;
-          if (!(ok = wait_or_abort(&sh->k_full[st], it & 1, sh, a.status, 21))) break;
-          TRACE(1, j);
-          tc_fence_after();
-          const uint64_t dk = smem_desc_kmajor(smem_u32(sK + st * kTileBytes), D);
-#pragma unroll
-          for (int k = 0; k < D / 32; ++k) mma_f8_ss(tmem + S_COL + 128 * (j & 1), dq + 2 * k, dk + 2 * k, idesc_qk, k > 0);
-          mma_commit(&sh->s_full[j & 1]);
-          TRACE(2, j);
-        }
-        if (j >= 1) {
-          const int i = j - 1, b = i & 1, ph = (i >> 1) & 1, st = i % kStages, it = i / kStages;
-          if (!(ok = wait_or_abort(&sh->p_full[b], ph, sh, a.status, 22))) break;
-          TRACE(3, i);
-          if (!(ok = wait_or_abort(&sh->c_done[b], ph, sh, a.status, 23))) break;
-          TRACE(4, i);
-          if (!(ok = wait_or_abort(&sh->v_full[st], it & 1, sh, a.status, 24))) break;
-          tc_fence_after();
-          const uint64_t dv = smem_desc_kmajor(smem_u32(sV + st * kTileBytes), 128);
-#pragma unroll
-          for (int k = 0; k < 4; ++k) { mma_f8_ts(tmem + O_COL, tmem + S_COL + 128 * b + 8 * k, dv + 2 * k, idesc_pv, (i > 0) | (k > 0)); TRACE(12 + k, i); }
-          if ((i % kGroup) == kGroup - 1 || i == nb - 1) {
-            const int g = i / kGroup;
-            if (!(ok = wait_or_abort(&sh->g_done[g & 1], (g >> 1) & 1, sh, a.status, 25))) break;
-            if (!(ok = wait_or_abort(&sh->mu_full[g & 1], (g >> 1) & 1, sh, a.status, 26))) break;
-            tc_fence_after();
-            const uint64_t dm = smem_desc_kmajor(smem_u32(sMu + (g & 1) * kTileBytes), 128);
-#pragma unroll
-            for (int k = 0; k < 4; ++k) mma_tf32_ts(tmem + O_COL, tmem + R_COL + 8 * k, dm + 2 * k, idesc_mu, 1);
-            mma_commit(&sh->mu_empty[g & 1]);
-          }
-          mma_commit(&sh->kv_empty[st]);
-          mma_commit(&sh->o_done[b]);
-          TRACE(5, i);
-        }
-      }
-    }
-  } else if (warp < 20) {
-    // -------------------------------------------------------------------- softmax stage
-    // 16 warps: warp (4 + 4 q + w) owns rows 32 w .. 32 w + 31 (its TMEM lane quadrant) and
-    // key columns 32 q .. 32 q + 31; the four threads of a row exchange their partial
-    // maxima through shared memory behind a 128-thread mbarrier.
-    const int cq = (warp - 4) >> 2, quad = warp & 3;
-    const int row = quad * 32 + lane;
-    const float sq = a.q_scale[(size_t)bh * nb + qblk];
-    float m_run = -INFINITY;
-    for (int j = 0; j < nb; ++j) {
-      const int b = j & 1, ph = (j >> 1) & 1;
-      const float cs = (sq * a.k_scale[(size_t)bh * nb + j]) * a.sl;
-      if (!warp_wait(&sh->s_full[b], ph, sh, a.status, 30)) break;
-      if (cq == 0 && quad == 0 && lane == 0) TRACE(6, j);
-      tc_fence_after();
-      uint32_t sv[32];
-      const uint32_t sbase = lane_base + S_COL + 128 * b;
-      tmem_ld32(sbase + 32 * cq, sv);
-      tmem_wait_ld();
-      if (cq == 0 && quad == 0 && lane == 0) TRACE(7, j);
-      const int nv = a.N - j * 128 - 32 * cq;             // valid keys among my 32 columns
-      if (nv < 32) {                                      // padded keys never win the maximum
-#pragma unroll
-        for (int i = 0; i < 32; ++i)
-          if (i >= nv) sv[i] = 0xff800000u;
-      }
-      float mx0 = __uint_as_float(sv[0]), mx1 = __uint_as_float(sv[1]);
-#pragma unroll
-      for (int i = 2; i < 30; i += 4) {
-        mx0 = max3(mx0, __uint_as_float(sv[i]), __uint_as_float(sv[i + 1]));
-        mx1 = max3(mx1, __uint_as_float(sv[i + 2]), __uint_as_float(sv[i + 3]));
-      }
-      sh->pmax[b][cq][row] = max3(mx0, mx1, fmaxf(__uint_as_float(sv[30]), __uint_as_float(sv[31])));
-      mbar_arrive(&sh->pm_full[b][quad]);                 // bounded stand-in for a named barrier;
-      if (!warp_wait(&sh->pm_full[b][quad], ph, sh, a.status, 31)) break;   // also: all four have read S
-      if (cq == 0 && quad == 0 && lane == 0) TRACE(8, j);
-      const float mx = fmaxf(fmaxf(sh->pmax[b][0][row], sh->pmax[b][1][row]), fmaxf(sh->pmax[b][2][row], sh->pmax[b][3][row]));
-      const float m_new = fmaxf(m_run, mx * cs);          // m' = max(m, rowmax S_ij)
-      if (cq == 0) {
-        sh->alpha[b][row] = ex2_approx(m_run - m_new);    // alpha; 0 on the first tile
-        mbar_arrive(&sh->a_full[b]);
-      }
-      m_run = m_new;
-
-      uint32_t pk[8];
-      float acc0 = 0.f, acc1 = 0.f;
-      if (a.debug & 2) {
-#pragma unroll
-        for (int w = 0; w < 8; ++w) pk[w] = sv[w] & 0x38383838u;
-      } else if constexpr (EXPCAST) {
-        // Eq. 7 in two FMAs: t = sat((8 u + 120 + beta) / 128) clips to [0, 1], then
-        // t * 128 + 1.5 * 2^23 rounds to the nearest even integer in the low mantissa bits.
-        const float fa = cs * 0.0625f, fb = (a.code_off - 8.0f * m_new) * 0.0078125f;
-#pragma unroll
-        for (int w = 0; w < 8; ++w) {
-          const uint32_t r0 = __float_as_uint(fmaf(fma_sat(__uint_as_float(sv[4 * w]), fa, fb), 128.0f, 12582912.0f));
-          const uint32_t r1 = __float_as_uint(fmaf(fma_sat(__uint_as_float(sv[4 * w + 1]), fa, fb), 128.0f, 12582912.0f));
-          const uint32_t r2 = __float_as_uint(fmaf(fma_sat(__uint_as_float(sv[4 * w + 2]), fa, fb), 128.0f, 12582912.0f));
-          const uint32_t r3 = __float_as_uint(fmaf(fma_sat(__uint_as_float(sv[4 * w + 3]), fa, fb), 128.0f, 12582912.0f));
-          // (code << 20) read as fp32 is the decoded E4M3 value times 2^-120, subnormal codes included
-          acc0 += __uint_as_float(r0 << 20) + __uint_as_float(r2 << 20);
-          acc1 += __uint_as_float(r1 << 20) + __uint_as_float(r3 << 20);
-          pk[w] = __byte_perm(__byte_perm(r0, r1, 0x0040), __byte_perm(r2, r3, 0x0040), 0x5410);
-        }
-      } else {
-        // exponentiate, then cast (Fig. 4a upper box)
-        const float nm = 8.0f - m_new;
-#pragma unroll
-        for (int w = 0; w < 8; ++w) {
-          const float p0 = exp2f(fmaf(__uint_as_float(sv[4 * w]), cs, nm)), p1 = exp2f(fmaf(__uint_as_float(sv[4 * w + 1]), cs, nm));
-          const float p2 = exp2f(fmaf(__uint_as_float(sv[4 * w + 2]), cs, nm)), p3 = exp2f(fmaf(__uint_as_float(sv[4 * w + 3]), cs, nm));
-          const uint32_t lo = __nv_cvt_float2_to_fp8x2(make_float2(p0, p1), __NV_SATFINITE, __NV_E4M3);
-          const uint32_t hi = __nv_cvt_float2_to_fp8x2(make_float2(p2, p3), __NV_SATFINITE, __NV_E4M3);
-          acc0 += __uint_as_float((lo & 0xffu) << 20) + __uint_as_float((hi & 0xffu) << 20);
-          acc1 += __uint_as_float((lo >> 8) << 20) + __uint_as_float((hi >> 8) << 20);
-          pk[w] = lo | (hi << 16);
-        }
-      }
-      sh->rsum[b][cq][row] = ((acc0 + acc1) * 1152921504606846976.0f) * 1152921504606846976.0f;   // x 2^120
-      tmem_st8(sbase + 8 * cq, pk);                       // P^ aliases the consumed scores
-      tmem_wait_st();
-      tc_fence_before();
-      mbar_arrive(&sh->p_full[b]);
-      if (cq == 0 && quad == 0 && lane == 0) TRACE(9, j);
-    }
-  } else {
-    // -------------------------------------------------------------------- correction stage
-    const int row = (warp & 3) * 32 + lane;
-    float l_run = 0.f;
-    bool ok = true;
-    for (int j = 0; j < nb; ++j) {
-      const int b = j & 1, ph = (j >> 1) & 1, slot = j % kGroup, g = j / kGroup;
-      if (!(ok = warp_wait(&sh->a_full[b], ph, sh, a.status, 40))) break;
-      const float alpha = sh->alpha[b][row];
-      if ((warp & 3) == 0 && lane == 0) TRACE(10, j);
-      if (j > 0 && !(a.debug & 1)) {
-        if (!(ok = warp_wait(&sh->o_done[(j - 1) & 1], ((j - 1) >> 1) & 1, sh, a.status, 41))) break;
-        tc_fence_after();
-      }
-      uint32_t r[32];
-      if (slot == 0) {                                    // new group: clear the row-sum slots
-#pragma unroll
-        for (int i = 0; i < 32; ++i) r[i] = 0u;
-        tmem_st32(lane_base + R_COL, r);
-      }
-      if (j > 0 && !(a.debug & 1) && __any_sync(0xffffffffu, alpha != 1.0f)) {
-#pragma unroll 1
-        for (int c = 0; c < D / 32 + (slot > 0 ? 1 : 0); ++c) {
-          const uint32_t col = c < D / 32 ? O_COL + 32 * c : R_COL;
-          tmem_ld32(lane_base + col, r);
-          tmem_wait_ld();
-#pragma unroll
-          for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * alpha);
-          tmem_st32(lane_base + col, r);
-        }
-      }
-      l_run *= alpha;
-      tmem_wait_st();
-      tc_fence_before();
-      mbar_arrive(&sh->c_done[b]);
-      if ((warp & 3) == 0 && lane == 0) TRACE(11, j);
-      if (!(ok = warp_wait(&sh->p_full[b], ph, sh, a.status, 42))) break;
-      const float rs = (sh->rsum[b][0][row] + sh->rsum[b][1][row]) + (sh->rsum[b][2][row] + sh->rsum[b][3][row]);   // r_ij = P~_ij 1
-      l_run += rs;                                        // l <- alpha l + r
-      const uint32_t hi = (__float_as_uint(rs) + 0x1000u) & 0xffffe000u;   // nearest TF32
-      const float lo = rs - __uint_as_float(hi);
-      tmem_st2(lane_base + R_COL + 2 * slot, hi, __float_as_uint(lo));
-      tmem_wait_st();
-      tc_fence_before();
-      if (slot == kGroup - 1 || j == nb - 1) mbar_arrive(&sh->g_done[g & 1]);
-    }
-    // ---- epilogue: O = s_V * A / l
-    if (ok && warp_wait(&sh->o_done[(nb - 1) & 1], ((nb - 1) >> 1) & 1, sh, a.status, 43)) {
-      tc_fence_after();
-      const int grow = qblk * 128 + row;
-      const float inv_l = 1.0f / l_run;
-      uint32_t r[32];
-#pragma unroll 1
-      for (int c = 0; c < D / 32; ++c) {
-        tmem_ld32(lane_base + O_COL + 32 * c, r);
-        tmem_wait_ld();
-        if (grow < a.N) {
-          uint32_t out[16];
-#pragma unroll
-          for (int i = 0; i < 16; ++i) {
-            const float x0 = __uint_as_float(r[2 * i]) * inv_l * __ldg(&a.v_scale[(size_t)bh * D + 32 * c + 2 * i]);
-            const float x1 = __uint_as_float(r[2 * i + 1]) * inv_l * __ldg(&a.v_scale[(size_t)bh * D + 32 * c + 2 * i + 1]);
-            __nv_bfloat162 h2 = __floats2bfloat162_rn(x0, x1);
-            out[i] = *reinterpret_cast<uint32_t*>(&h2);
-          }
-          uint4* dst = reinterpret_cast<uint4*>(a.o + ((size_t)bh * a.N + grow) * D + 32 * c);
-#pragma unroll
-          for (int i = 0; i < 4; ++i) dst[i] = make_uint4(out[4 * i], out[4 * i + 1], out[4 * i + 2], out[4 * i + 3]);
-        }
-      }
-    }
-  }
-  tc_fence_before();
-  __syncthreads();
-  if (warp == 2) tmem_dealloc<kTmemCols>(tmem);
-}
-
-// Block means in the layout the mean-restoration MMA reads: per (b, h) and group of 16 key
-// tiles a [d][32] fp32 tile, entry [c][2 s] = [c][2 s + 1] = mu~ of tile 16 g + s (0 past the end).
-template <int D>
-__global__ void means_mma_layout_kernel(const __nv_bfloat16* __restrict__ means, float* __restrict__ out, int nb, int ng) {
-  const int g = blockIdx.x, bh = blockIdx.y, c = threadIdx.x;
-  float4* dst = reinterpret_cast<float4*>(out + (((size_t)bh * ng + g) * D + c) * 32);
-#pragma unroll
-  for (int s4 = 0; s4 < 8; ++s4) {
-    const int t0 = g * kGroup + 2 * s4, t1 = t0 + 1;
-    const float v0 = t0 < nb ? __bfloat162float(means[((size_t)bh * nb + t0) * D + c]) : 0.f;
-    const float v1 = t1 < nb ? __bfloat162float(means[((size_t)bh * nb + t1) * D + c]) : 0.f;
-    dst[s4] = make_float4(v0, v0, v1, v1);
-  }
-}
 
 
 // ---------------------------------------------------------------------------------------
@@ -765,14 +435,14 @@ attn_fwd_2q_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         mx[4 + c] = fmaxf(mx[4 + c], __uint_as_float(s2[16 * c + 15]));
         mx[6 + c] = fmaxf(mx[6 + c], __uint_as_float(s3[16 * c + 15]));
       }
-      const float mxa = (a.debug & 8) ? __uint_as_float(s0[0]) : max3(max3(mx[0], mx[1], mx[2]), max3(mx[3], mx[4], mx[5]), fmaxf(mx[6], mx[7]));
+      const float mxa = max3(max3(mx[0], mx[1], mx[2]), max3(mx[3], mx[4], mx[5]), fmaxf(mx[6], mx[7]));
       const float m_new = fmaxf(m_run, mxa * cs);         // m' = max(m, rowmax S_ij)
       const float alpha = ex2_approx(m_run - m_new);      // 0 on the first tile
       sh->alpha[t][row] = alpha;
       mbar_arrive(&sh->a_full[t][j & 1]);
       m_run = m_new;
       // the previous code tile must have been consumed before it is overwritten
-      if (j > 0 && !(a.debug & 32) && !(ok = warp_wait2(&sh->o_done[t], (j - 1) & 1, sh, a.status, 31))) break;
+      if (j > 0 && !(ok = warp_wait2(&sh->o_done[t], (j - 1) & 1, sh, a.status, 31))) break;
 
       float acc0 = 0.f, acc1 = 0.f, acc2 = 0.f, acc3 = 0.f;
       const float fa = cs * 0.0625f, fb = (a.code_off - 8.0f * m_new) * 0.0078125f, nm = 8.0f - m_new;
@@ -803,14 +473,8 @@ attn_fwd_2q_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         const uint4 v = make_uint4(code4(sv, 4 * half), code4(sv, 4 * half + 1), code4(sv, 4 * half + 2), code4(sv, 4 * half + 3));
         *reinterpret_cast<uint4*>(p_row + ((chunk ^ (row & 7)) << 4)) = v;
       };
-      if (a.debug & 2) {
-#pragma unroll
-        for (int c = 0; c < 8; ++c) *reinterpret_cast<uint4*>(p_row + (c << 4)) = make_uint4(s0[c] & 0x38383838u, s1[c] & 0x38383838u, s2[c] & 0x38383838u, s3[c] & 0x38383838u);
-        acc0 = 1e-30f;
-      } else {
       store16(s0, 0, 0); store16(s0, 1, 1); store16(s1, 0, 2); store16(s1, 1, 3);
       store16(s2, 0, 4); store16(s2, 1, 5); store16(s3, 0, 6); store16(s3, 1, 7);
-      }
       const float rs = (((acc0 + acc1) + (acc2 + acc3)) * 1152921504606846976.0f) * 1152921504606846976.0f;   // x 2^120
       l_run = alpha * l_run + rs;                         // l <- alpha l + r,  r = P~ 1 over the decoded codes
       const uint32_t hi = (__float_as_uint(rs) + 0x1000u) & 0xffffe000u;     // nearest TF32
@@ -850,10 +514,9 @@ attn_fwd_2q_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
     const int row = (warp & 3) * 32 + lane;
     const uint32_t o_base = lane_base + 256 + 128 * t;
     for (int j = 0; j < nb; ++j) {
-      const int ph = j & 1;
       if (!warp_wait2(&sh->a_full[t][j & 1], (j >> 1) & 1, sh, a.status, 40)) break;
       const float alpha = sh->alpha[t][row];
-      if (j > 0 && !(a.debug & 1) && __any_sync(0xffffffffu, alpha != 1.0f)) {
+      if (j > 0 && __any_sync(0xffffffffu, alpha != 1.0f)) {
         if (!warp_wait2(&sh->o_done[t], (j - 1) & 1, sh, a.status, 41)) break;
         tc_fence_after();
         uint32_t r[32];
@@ -922,12 +585,10 @@ bool make_map(CUtensorMap* m, const void* base, uint64_t dim0, uint64_t dim1, ui
 template <int D>
 cudaError_t run8(const Problem& pr, const QuantLayout& ql, const WorkLayout& wl, const uint8_t* quant,
                  void* o, uint8_t* work, cudaStream_t s) {
-  alignas(64) CUtensorMap tq, tk, tv, tmu;
-  const int ng = (pr.nb + kGroup - 1) / kGroup;
+  alignas(64) CUtensorMap tq, tk, tv;
   if (!make_map(&tq, quant + ql.q_codes, D, pr.n_pad, pr.BH, D, 128) ||
       !make_map(&tk, quant + ql.k_codes, D, pr.n_pad, pr.BH, D, 128) ||
-      !make_map(&tv, quant + ql.v_codes, pr.n_pad, D, pr.BH, 128, D) ||
-      !make_map(&tmu, work + wl.mu_mma, 128, D, (uint64_t)pr.BH * ng, 128, D))
+      !make_map(&tv, quant + ql.v_codes, pr.n_pad, D, pr.BH, 128, D))
     return cudaErrorUnknown;
   AttnArgs a{};
   a.q_scale = (const float*)(quant + ql.q_scale);
@@ -936,10 +597,9 @@ cudaError_t run8(const Problem& pr, const QuantLayout& ql, const WorkLayout& wl,
   a.v_means = (const __nv_bfloat16*)(quant + ql.v_means);
   a.o = (__nv_bfloat16*)o;
   a.status = (uint32_t*)(work + wl.status);
-  a.N = pr.N; a.n_pad = pr.n_pad; a.nb = pr.nb; a.ng = ng; a.p_format = pr.p_format;
+  a.N = pr.N; a.n_pad = pr.n_pad; a.nb = pr.nb; a.p_format = pr.p_format;
   a.sl = pr.softmax_scale * 1.4426950408889634f;
   a.code_off = 120.0f + pr.beta;
-  { const char* dbg = getenv("VC_DEBUG"); a.debug = dbg ? atoi(dbg) : 0; }
   cudaError_t e;
   if (pr.kernel_variant == 1) {     // serial reference kernel
     const size_t smem = 1024 + 2 * 128 * D + D * 128 + D * 4 + 64;
@@ -966,22 +626,10 @@ cudaError_t run8(const Problem& pr, const QuantLayout& ql, const WorkLayout& wl,
     count_launches(2);
     return cudaGetLastError();
   }
-  means_mma_layout_kernel<D><<<dim3(ng, pr.BH), D, 0, s>>>(a.v_means, (float*)(work + wl.mu_mma), pr.nb, ng);
-  const size_t smem = 1024 + (size_t)(1 + 2 * kStages + 2) * 128 * D + sizeof(PipeSmem);
-  if (pr.p_format == VC_P_EXPCAST_E4M3) {
-    if ((e = cudaFuncSetAttribute(attn_fwd_pipe_kernel<D, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
-    attn_fwd_pipe_kernel<D, true><<<dim3(pr.nb, pr.BH), 768, smem, s>>>(tq, tk, tv, tmu, a);
-  } else {
-    if ((e = cudaFuncSetAttribute(attn_fwd_pipe_kernel<D, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
-    attn_fwd_pipe_kernel<D, false><<<dim3(pr.nb, pr.BH), 768, smem, s>>>(tq, tk, tv, tmu, a);
-  }
-  count_launches(2);
-  return cudaGetLastError();
+  return cudaErrorNotSupported;
 }
 
 }  // namespace
-
-extern "C" int vc_debug_trace(long long* host) { return (int)cudaMemcpyFromSymbol(host, g_trace, sizeof(long long) * 8192); }
 
 cudaError_t launch_attn_fwd(const Problem& pr, const QuantLayout& ql, const WorkLayout& wl,
                             const uint8_t* quant, void* o, uint8_t* work, cudaStream_t stream) {

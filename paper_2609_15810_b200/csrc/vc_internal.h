@@ -40,7 +40,7 @@ struct WorkLayout {
   size_t v_mu;       // fp32 [BH][nb][d] block means of the gathered V
   size_t amax;       // uint32 [BH][d] residual amax bits (8-bit V) then [2][BH] Q/K head amax (4-bit)
   size_t amax_bytes;
-  size_t mu_mma;     // fp32 [BH][ceil(nb/16)][d][32] block means in the layout of the mean-restoration MMA
+  size_t mu_mma;     // fp32 [BH][nb][d][8]: block means as the B operand of the mean-restoration MMA
   size_t total;
   int rope_off[3];   // entry offset of each axis table
   int rope_entries;
