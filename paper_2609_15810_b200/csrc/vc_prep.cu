@@ -96,15 +96,7 @@ __device__ __forceinline__ void qk_body(const PrepArgs& a, unsigned char* smem) 
   const bool do_had = (a.flags & VC_FLAG_HADAMARD) && STAGE != kStageColSum;
   const bool gather = TENSOR == 1 && a.perm != nullptr && STAGE >= kStageQuant8;
 
-  // RoPE table -> shared memory (or read through L2 when it does not fit)
-  const float2* tab = a.rope;
   float* red = reinterpret_cast<float*>(smem);            // [8][D] floats of scratch
-  if (do_rope && a.rope_in_smem) {
-    float2* st = reinterpret_cast<float2*>(smem + 8 * D * 4);
-    for (int e = tid; e < a.rd.entries; e += kThreads) st[e] = a.rope[e];
-    tab = st;
-    __syncthreads();
-  }
   // per-lane constants of the 4 channel pairs it owns
   int p_axis[4], p_idx[4];
 #pragma unroll
@@ -122,16 +114,35 @@ __device__ __forceinline__ void qk_body(const PrepArgs& a, unsigned char* smem) 
     for (int c = 0; c < 8; ++c) kmean[c] = a.k_mean[(size_t)bh * D + 8 * lr + c];
   }
 
+  // all row loads of the thread are issued before any arithmetic: bytes in flight, not
+  // instruction count, set the speed of this pass
+  int srcs[RPL];
+#pragma unroll
+  for (int i = 0; i < RPL; ++i) {
+    const int t = blk * kBlock + 16 * warp + RPL * hb + i;
+    srcs[i] = t < a.N ? t : -1;
+    if (gather && t < a.N) srcs[i] = __ldg(&a.perm[(size_t)bh * a.N + t]);
+  }
+  uint4 raws[RPL];
+#pragma unroll
+  for (int i = 0; i < RPL; ++i) {
+    raws[i] = make_uint4(0, 0, 0, 0);
+    if (srcs[i] >= 0) raws[i] = __ldg(reinterpret_cast<const uint4*>(base + (int64_t)srcs[i] * a.stride_n + 8 * lr));
+  }
+  // RoPE table -> shared memory while the rows are in flight (read through L2 if it does not fit)
+  const float2* tab = a.rope;
+  if (do_rope && a.rope_in_smem) {
+    float2* st = reinterpret_cast<float2*>(smem + 8 * D * 4);
+    for (int e = tid; e < a.rd.entries; e += kThreads) st[e] = __ldg(&a.rope[e]);
+    tab = st;
+    __syncthreads();
+  }
   float x[RPL][8];
 #pragma unroll
   for (int i = 0; i < RPL; ++i) {
-    const int row = 16 * warp + RPL * hb + i;
-    const int t = blk * kBlock + row;
-    const bool valid = t < a.N;
-    int src = t;
-    if (gather && valid) src = a.perm[(size_t)bh * a.N + t];
-    uint4 raw = make_uint4(0, 0, 0, 0);
-    if (valid) raw = __ldg(reinterpret_cast<const uint4*>(base + (int64_t)src * a.stride_n + 8 * lr));
+    const bool valid = srcs[i] >= 0;
+    const int src = valid ? srcs[i] : 0;
+    const uint4 raw = raws[i];
     const unsigned int w[4] = {raw.x, raw.y, raw.z, raw.w};
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
@@ -296,15 +307,25 @@ __device__ __forceinline__ void v_body(const PrepArgs& a, unsigned char* smem) {
   uint4* tile4 = reinterpret_cast<uint4*>(smem);                       // [128][D] bf16
   float* red = reinterpret_cast<float*>(smem + kBlock * D * 2);        // [TG][D]
 
-  for (int idx = tid; idx < kBlock * LPR; idx += kThreads) {
-    const int row = idx / LPR, ch = idx - row * LPR;
-    const int t = blk * kBlock + row;
-    uint4 val = make_uint4(0, 0, 0, 0);
-    if (t < a.N) {
-      const int src = a.perm ? a.perm[(size_t)bh * a.N + t] : t;
-      val = __ldg(reinterpret_cast<const uint4*>(base + (int64_t)src * a.stride_n + 8 * ch));
+  {
+    constexpr int NL = kBlock * LPR / kThreads;   // 16-byte chunks per thread
+    int srcs[NL];
+#pragma unroll
+    for (int i = 0; i < NL; ++i) {
+      const int row = (tid + i * kThreads) / LPR;
+      const int t = blk * kBlock + row;
+      srcs[i] = t < a.N ? (a.perm ? __ldg(&a.perm[(size_t)bh * a.N + t]) : t) : -1;
     }
-    tile4[idx] = val;
+    uint4 vals[NL];
+#pragma unroll
+    for (int i = 0; i < NL; ++i) {
+      const int idx = tid + i * kThreads;
+      const int ch = idx % LPR;
+      vals[i] = make_uint4(0, 0, 0, 0);
+      if (srcs[i] >= 0) vals[i] = __ldg(reinterpret_cast<const uint4*>(base + (int64_t)srcs[i] * a.stride_n + 8 * ch));
+    }
+#pragma unroll
+    for (int i = 0; i < NL; ++i) tile4[tid + i * kThreads] = vals[i];
   }
   __syncthreads();
 
@@ -445,7 +466,7 @@ __device__ __forceinline__ void v_body(const PrepArgs& a, unsigned char* smem) {
 // Launch 1: statistics.  z = 0: K column sums; z = 1: V block means + residual amax;
 // z = 2 (4-bit): head amax of the rotated Q.
 template <int D, int BITS>
-__global__ void __launch_bounds__(kThreads) prep_stats_kernel(const PrepArgs a) {
+__global__ void __launch_bounds__(kThreads, 2) prep_stats_kernel(const PrepArgs a) {
   extern __shared__ __align__(16) unsigned char smem[];
   if (blockIdx.z == 0) {
     if (a.flags & VC_FLAG_K_SMOOTH) qk_body<D, 1, kStageColSum>(a, smem);
@@ -492,7 +513,7 @@ __global__ void __launch_bounds__(kThreads) prep_kamax_kernel(const PrepArgs a) 
 
 // Launch 4: quantization.  z = 0: Q; z = 1: K; z = 2: V.
 template <int D, int BITS>
-__global__ void __launch_bounds__(kThreads) prep_quant_kernel(const PrepArgs a) {
+__global__ void __launch_bounds__(kThreads, 2) prep_quant_kernel(const PrepArgs a) {
   extern __shared__ __align__(16) unsigned char smem[];
   if (blockIdx.z == 0) {
     qk_body<D, 0, BITS == 8 ? kStageQuant8 : kStageQuant4>(a, smem);
