@@ -44,7 +44,9 @@ typedef enum {
   VC_ERR_UNSUPPORTED = 2,   /* a combination this build does not implement           */
   VC_ERR_WORKSPACE = 3,     /* reserved                                              */
   VC_ERR_CUDA = 4,          /* a CUDA runtime/driver call failed                     */
-  VC_ERR_TIMEOUT = 5        /* a bounded device-side wait gave up                    */
+  VC_ERR_TIMEOUT = 5,       /* a bounded device-side wait gave up                    */
+  VC_ERR_SCRATCH_LIMIT = 6  /* vc_prep_noalloc: the problem needs more scratch than
+                               VC_NOALLOC_SCRATCH_BYTES                              */
 } vc_status;
 
 /* probability formats of the softmax stage (Sec. 3.3, App. A "Scope of ExpCast-FP8") */
@@ -135,6 +137,35 @@ vc_status vc_attn_host(const vc_params *p, const void *q_host, const void *k_hos
                        const void *v_host, const int32_t *perm_host, void *o_host,
                        void *q_dev, void *k_dev, void *v_dev, int32_t *perm_dev, void *o_dev,
                        void *quant, void *workspace, void *stream);
+
+/* vc_prep without a workspace argument and without any allocation.  (The paper has no
+ * counterpart: this entry point exists for the sake of its callers, not of the method.)
+ *
+ * Who needs it: code that runs where device memory may not be requested -- inside a
+ * framework that hands a plug-in a fixed set of buffers and forbids it to grow them, in a
+ * serving loop that has frozen its memory map after start-up, or on a thread that must not
+ * take the driver's allocation lock (cudaMalloc synchronizes the whole device).  Such a
+ * caller still owns q, k, v, perm and the output bundle `quant`, but has nowhere to put
+ * the pass's scratch.
+ *
+ * The scratch therefore lives inside the library, in one fixed array of
+ * VC_NOALLOC_SCRATCH_BYTES in device global memory.  Every GPU on which the library is
+ * used holds that array until the process exits.  Consequences:
+ *   - Problems whose scratch need exceeds the limit are refused with VC_ERR_SCRATCH_LIMIT
+ *     before anything is launched.  The need is 8 bytes per RoPE table entry plus about
+ *     8 * B*H * ceil(N/128) * d bytes (e.g. B*H = 12, N = 32760, d = 128 needs 3.2 MB).
+ *   - All calls on a device share the array, and it keeps whatever the previous call left
+ *     in it.  The call itself clears the words that have to start at zero, on `stream`.
+ *     Two calls that overlap on the GPU (different streams, or different host threads
+ *     without ordering between their streams) race on the array: serialize them.
+ *   - The first call on each device looks up the array's device address
+ *     (cudaGetSymbolAddress) with that device current; make that first call outside any
+ *     stream capture.  Later calls only launch kernels and two small memsets on `stream`.
+ * It calls no cudaMalloc / cudaFree and no allocating library routine.  The output is
+ * the same bundle vc_prep writes. */
+#define VC_NOALLOC_SCRATCH_BYTES (4u << 20)
+vc_status vc_prep_noalloc(const vc_params *p, const void *q, const void *k, const void *v,
+                          const int32_t *perm, void *quant, void *stream);
 
 /* Device pointers of the bundle's sections (for tests and for feeding a bundle in). */
 vc_status vc_quant_view(const vc_params *p, const void *quant, vc_quant_ptrs *out);

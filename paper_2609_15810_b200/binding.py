@@ -69,6 +69,8 @@ def load_library():
     lib.vc_workspace_bytes.argtypes = [P]
     lib.vc_prep.restype = ctypes.c_int
     lib.vc_prep.argtypes = [P, vp, vp, vp, i32p, vp, vp, vp]
+    lib.vc_prep_noalloc.restype = ctypes.c_int
+    lib.vc_prep_noalloc.argtypes = [P, vp, vp, vp, i32p, vp, vp]
     lib.vc_attn_fwd.restype = ctypes.c_int
     lib.vc_attn_fwd.argtypes = [P, vp, vp, vp, vp]
     lib.vc_attn.restype = ctypes.c_int
@@ -120,6 +122,12 @@ def vc_workspace_bytes(p):
 def vc_prep(p, q, k, v, perm, quant, workspace):
     _check(load_library().vc_prep(ctypes.byref(p), _ptr(q), _ptr(k), _ptr(v), _ptr(perm), _ptr(quant),
                                   _ptr(workspace), _stream()), "vc_prep")
+
+
+def vc_prep_noalloc(p, q, k, v, perm, quant):
+    """vc_prep on the library's built-in scratch array: no workspace, no allocation (size-limited)."""
+    _check(load_library().vc_prep_noalloc(ctypes.byref(p), _ptr(q), _ptr(k), _ptr(v), _ptr(perm), _ptr(quant),
+                                          _stream()), "vc_prep_noalloc")
 
 
 def vc_attn_fwd(p, quant, o, workspace):

@@ -254,6 +254,7 @@ const char* vc_status_string(vc_status s) {
     case VC_ERR_WORKSPACE: return "workspace error";
     case VC_ERR_CUDA: return "CUDA error";
     case VC_ERR_TIMEOUT: return "device-side wait timed out";
+    case VC_ERR_SCRATCH_LIMIT: return "problem needs more scratch than the built-in array of vc_prep_noalloc holds";
   }
   return "unknown status";
 }

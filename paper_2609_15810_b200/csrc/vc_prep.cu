@@ -600,3 +600,54 @@ cudaError_t launch_prep(const Problem& pr, const QuantLayout& ql, const WorkLayo
 }
 
 }  // namespace vc
+
+// ---------------------------------------------------------------------------------------
+// vc_prep_noalloc: the preprocessing pass for callers that cannot provide a workspace.
+// The scratch that vc_prep takes from the caller (RoPE tables, per-block partial sums, block
+// means, amax words) lives here in a fixed array in device global memory, so the call needs no
+// allocation of any kind; the price is a size limit and one array per GPU for the life of the
+// process.
+namespace {
+
+// Held by every GPU that loads this library until the process exits.
+static __device__ __align__(256) unsigned char g_prep_scratch[VC_NOALLOC_SCRATCH_BYTES];
+
+constexpr int kMaxDevices = 64;
+unsigned char* g_scratch_addr[kMaxDevices] = {};   // device address of the array, per device
+
+// In host code the array's name is only a handle; the device address has to be asked for,
+// once per device, with that device current.
+cudaError_t scratch_address(unsigned char** out) {
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+  unsigned char* ptr = __atomic_load_n(&g_scratch_addr[dev], __ATOMIC_ACQUIRE);
+  if (!ptr) {
+    e = cudaGetSymbolAddress(reinterpret_cast<void**>(&ptr), g_prep_scratch);
+    if (e != cudaSuccess) return e;
+    __atomic_store_n(&g_scratch_addr[dev], ptr, __ATOMIC_RELEASE);   // same value from any thread
+  }
+  *out = ptr;
+  return cudaSuccess;
+}
+
+}  // namespace
+
+extern "C" vc_status vc_prep_noalloc(const vc_params* p, const void* q, const void* k, const void* v,
+                                     const int32_t* perm, void* quant, void* stream) {
+  vc::Problem pr;
+  vc_status st = vc::resolve(p, &pr);
+  if (st != VC_OK) return st;
+  if (!q || !k || !v || !quant) return VC_ERR_INVALID_ARG;
+  if (((uintptr_t)q | (uintptr_t)k | (uintptr_t)v | (uintptr_t)quant | (uintptr_t)perm) & 15) return VC_ERR_INVALID_ARG;
+  const vc::QuantLayout ql = vc::quant_layout(pr);
+  const vc::WorkLayout wl = vc::work_layout(pr);
+  // the pass uses the workspace sections in front of the attention kernel's mean table
+  if (wl.mu_mma > (size_t)VC_NOALLOC_SCRATCH_BYTES) return VC_ERR_SCRATCH_LIMIT;
+  unsigned char* scratch = nullptr;
+  if (scratch_address(&scratch) != cudaSuccess) return VC_ERR_CUDA;
+  // launch_prep clears the words that must start at zero (status, amax) on the stream itself
+  cudaError_t e = vc::launch_prep(pr, ql, wl, q, k, v, perm, (uint8_t*)quant, scratch, (cudaStream_t)stream);
+  return e == cudaSuccess ? VC_OK : VC_ERR_CUDA;
+}

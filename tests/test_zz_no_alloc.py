@@ -1,0 +1,63 @@
+"""vc_prep_noalloc: the preprocessing pass on the library's built-in scratch array.
+
+Some callers of this library may not request device memory at all (a plug-in inside a host
+framework with a frozen memory map, a serving thread that must stay off the allocator's
+lock), so they cannot hand vc_prep a workspace.  This entry point keeps the scratch in a
+fixed array inside the library instead.  The checks: through the C ABI it writes exactly
+the bundle vc_prep writes, on two calls in a row with different inputs (the array keeps the
+first call's contents, which must not leak into the second), and it refuses problems that
+do not fit.  The file name sorts last so that a run that stops at the first failure has
+already run every other test.
+"""
+import pytest
+import torch
+
+import paper_2609_15810_b200 as vc
+import vc_inputs
+from paper_2609_15810_b200.binding import Params, alloc_buffers
+
+pytestmark = pytest.mark.gpu
+
+
+def _bundle_with_workspace(p, q, k, v, perm):
+    quant, work = alloc_buffers(p)
+    quant.zero_()
+    vc.vc_prep(p, q, k, v, perm, quant, work)
+    torch.cuda.synchronize()
+    return quant
+
+
+def _bundle_without(p, q, k, v, perm):
+    quant = torch.zeros(vc.vc_quant_bytes(p), dtype=torch.uint8, device="cuda")
+    vc.vc_prep_noalloc(p, q, k, v, perm, quant)
+    torch.cuda.synchronize()
+    return quant
+
+
+@pytest.mark.parametrize("bits", [8, 4])
+def test_noalloc_matches_vc_prep_on_two_calls_in_a_row(bits):
+    calls = [  # different shape, data and permutation per call
+        (vc_inputs.Workload("a", 1, 4, 4096, 128, (4, 32, 32), (8,), 31, "field"), "random"),
+        (vc_inputs.Workload("b", 2, 2, 1000, 64, (10, 10, 10), (8,), 32, "gauss"), "identity"),
+    ]
+    for w, perm_kind in calls:
+        q, k, v = [t.cuda() for t in vc_inputs.make_qkv(w)]
+        perm = vc_inputs.random_perm(w.B, w.H, w.N, w.seed).cuda() if perm_kind == "random" else None
+        p = Params.make(w.B, w.H, w.N, w.d, w.grid, bits=bits)
+        got = _bundle_without(p, q, k, v, perm)
+        want = _bundle_with_workspace(p, q, k, v, perm)
+        # same kernels, same arithmetic order: the bundles are identical byte for byte, which is
+        # tighter than the one-code-step tolerance the other parity tests allow
+        assert torch.equal(got, want), f"{w.name}: {(got != want).sum().item()} bytes differ"
+
+
+def test_noalloc_refuses_what_does_not_fit_and_bad_arguments():
+    big = Params.make(1, 40, 32760, 128, (21, 30, 52), bits=8)       # needs about 10 MB of scratch
+    x = torch.zeros(16, dtype=torch.uint8, device="cuda")
+    with pytest.raises(vc.VcError) as e:
+        vc.vc_prep_noalloc(big, x, x, x, None, x)
+    assert e.value.code == 6 and "scratch" in str(e.value)
+    small = Params.make(1, 1, 128, 128, (2, 8, 8))
+    with pytest.raises(vc.VcError) as e:
+        vc.vc_prep_noalloc(small, None, x, x, None, x)
+    assert e.value.code == 1
