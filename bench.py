@@ -40,7 +40,7 @@ def _peaks():
 
 class ClockSampler:
     """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
-    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+    Q = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
          "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
          "clocks_event_reasons.sw_power_cap")
 
@@ -50,7 +50,7 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.Q,
-                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                          "--format=csv,noheader,nounits", "-lms", "50"],
                                          stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
@@ -61,7 +61,9 @@ class ClockSampler:
         for line in self.proc.stdout:
             self.lines.append(line.strip())
 
-    def stop(self):
+    def stop(self, t0=None, t1=None):
+        """Median SM clock and the throttle reasons seen between wall-clock times t0 and t1."""
+        import datetime
         if self.proc is None:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
         self.proc.terminate()
@@ -69,21 +71,27 @@ class ClockSampler:
             self.proc.wait(timeout=5)
         except subprocess.TimeoutExpired:
             self.proc.kill()
-        sm, mx, reasons = [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        rows = []
         for line in self.lines:
             f = [x.strip() for x in line.split(",")]
             if len(f) < 8:
                 continue
             try:
-                sm.append(float(f[0])); mx.append(float(f[1]))
+                ts = datetime.datetime.strptime(f[0], "%Y/%m/%d %H:%M:%S.%f").timestamp()
+                rows.append((ts, float(f[1]), float(f[2]), float(f[3]), [n for n, v in zip(names, f[4:8]) if v.lower().startswith("active")]))
             except ValueError:
                 continue
-            for name, val in zip(names, f[4:8]):
-                if val.lower().startswith("active"):
-                    reasons.add(name)
-        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "reasons": sorted(reasons), "samples": len(sm)}
+        inside = [r for r in rows if t0 is not None and t0 - 0.02 <= r[0] <= t1 + 0.02]
+        window = "timed region"
+        if not inside:      # region shorter than the sampling period: fall back to the samples under load
+            inside = [r for r in rows if r[3] > 300.0] or rows
+            window = "whole run (timed region shorter than the sampling period)"
+        sm = [r[1] for r in inside]
+        reasons = sorted({n for r in inside for n in r[4]})
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max((r[2] for r in inside), default=None),
+                "power_w_max": max((r[3] for r in inside), default=None), "reasons": reasons, "samples": len(sm),
+                "window": window}
 
 
 def run_reference(args, w, bits):
@@ -117,37 +125,43 @@ def run_reference(args, w, bits):
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
 
 
-def cpu_baseline(w, bits, budget_rows=256):
+def cpu_baseline(w, bits, budget_rows=4096, heads=2):
+    """The oracle as it stands on a bounded sample (about 10-30 s of CPU work)."""
     import numpy as np
     from oracle import attention as OA
     from oracle import prep as OP
-    q, k, v = [t[0, 0].float().numpy() for t in vc_inputs.make_qkv(w, heads=[0])]
     cfg = OP.PrepConfig(N=w.N, d=w.d, grid=w.grid, bits=bits)
-    rows = np.linspace(0, w.N - 1, budget_rows).astype(np.int64)
-    t0 = time.perf_counter()
-    bundle = OP.prep_head(q, k, v, None, cfg)
-    t1 = time.perf_counter()
-    OA.emulate_head(bundle, cfg, rows=rows)
-    t2 = time.perf_counter()
-    flops = 4.0 * budget_rows * w.N * w.d
-    return {"value": flops / (t2 - t0) / 1e12, "unit": UNIT, "cores": os.cpu_count(), "kind": "oracle",
-            "sample": f"preprocessing of 1 of {w.B * w.H} heads in full ({t1 - t0:.1f} s) + {budget_rows} of {w.N} query "
-                      f"rows x all keys of that head ({t2 - t1:.1f} s); NumPy, threads as BLAS picks"}
+    rows = np.linspace(0, w.N - 1, min(budget_rows, w.N)).astype(np.int64)
+    tp = ta = 0.0
+    for h in range(heads):
+        q, k, v = [t[0, 0].float().numpy() for t in vc_inputs.make_qkv(w, heads=[h])]
+        t0 = time.perf_counter()
+        bundle = OP.prep_head(q, k, v, None, cfg)
+        t1 = time.perf_counter()
+        OA.emulate_head(bundle, cfg, rows=rows)
+        t2 = time.perf_counter()
+        tp += t1 - t0
+        ta += t2 - t1
+    flops = 4.0 * heads * len(rows) * w.N * w.d
+    return {"value": flops / (tp + ta) / 1e12, "unit": UNIT, "cores": os.cpu_count(), "kind": "oracle",
+            "sample": f"{heads} of {w.B * w.H} heads: preprocessing in full ({tp:.1f} s) + {len(rows)} of {w.N} query rows x "
+                      f"all keys per head ({ta:.1f} s); NumPy, threads as its BLAS picks"}
 
 
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=10)
-    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--steps", type=int, default=30)
+    ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="c3")
     ap.add_argument("--bits", type=int, default=8)
     ap.add_argument("--perm", default="kmeans", choices=["kmeans", "identity", "random"])
     ap.add_argument("--heads-per-pass", type=int, default=0)
-    ap.add_argument("--ref-rows", type=int, default=128)
+    ap.add_argument("--ref-rows", type=int, default=1024)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-sdpa", action="store_true")
     args = ap.parse_args()
     w = vc_inputs.WORKLOADS[args.workload]
     rank = int(os.environ.get("RANK", "0"))
@@ -169,6 +183,8 @@ def main():
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=dev)
 
+    sampler = ClockSampler(local_rank)
+    sampler.start()
     # every rank runs the same workload on its own GPU (heads are independent: no collective)
     q, k, v = vc_inputs.make_qkv(w, device=dev)
     if args.perm == "kmeans":
@@ -192,11 +208,10 @@ def main():
         vc.vc_attn(p, q, k, v, perm, o, quant, work)
     vc.vc_poll_status(work)
 
-    sampler = ClockSampler(local_rank)
-    sampler.start()
     ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
     launches0 = vc.vc_launch_count()
     barrier()
+    wall0 = time.time()
     t_start, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     t_start.record(stream)
     for s in range(args.steps):
@@ -207,8 +222,9 @@ def main():
         ev[s][2].record(stream)
     t_end.record(stream)
     barrier()
+    wall1 = time.time()
     launches = vc.vc_launch_count() - launches0
-    clocks = sampler.stop()
+    clocks = sampler.stop(wall0, wall1)
     vc.vc_poll_status(work)
     ms_total = t_start.elapsed_time(t_end)
     prep_ms = statistics.mean(e[0].elapsed_time(e[1]) for e in ev)
@@ -274,6 +290,21 @@ def main():
         "prep": {"ms": prep_ms, "algorithmic_gb": prep_bytes / 1e9, "gbs": prep_gbs,
                  "frac_of_measured_hbm": prep_gbs / peaks["hbm_gbs"], "frac_of_8tbs": prep_gbs / 8000.0},
     }
+    if not args.no_sdpa:
+        try:    # context only: a library bf16 attention on the same GPU and tensors
+            import torch.nn.functional as F
+            for _ in range(2):
+                F.scaled_dot_product_attention(q, k, v)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(3):
+                F.scaled_dot_product_attention(q, k, v)
+            e1.record()
+            torch.cuda.synchronize()
+            ms = e0.elapsed_time(e1) / 3
+            out["bf16_sdpa"] = {"ms": ms, "tflops": w.flops / (ms * 1e-3) / 1e12, "what": "torch SDPA bf16, default backend, no RoPE/quantization"}
+        except Exception as exc:  # pragma: no cover
+            out["bf16_sdpa"] = {"error": str(exc)[:200]}
     if not args.no_cpu_baseline:
         out["cpu_baseline"] = cpu_baseline(w, args.bits)
     print(json.dumps(out), flush=True)

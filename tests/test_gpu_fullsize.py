@@ -1,0 +1,48 @@
+"""Parity at the full sizes of the benchmark configurations, in the launch configuration
+bench.py times (all heads in one call, k-means permutation), on what the oracle can compute
+one by one: the preprocessing of sampled heads in full, and sampled query tiles (the ragged
+last one included) against all keys of those heads."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2609_15810_b200 as vc
+import vc_inputs
+from paper_2609_15810_b200.binding import Params, alloc_buffers
+from oracle import attention as OA
+from oracle import compare as CMP
+
+import helpers as Hh
+
+pytestmark = pytest.mark.gpu
+
+CASES = [("c2", 8, "kmeans"), ("c3", 8, "kmeans"), ("c3", 4, "random"), ("c4", 4, "kmeans"),
+         ("c5_d64_n4096", 8, "random"), ("c5_d64_n4096", 4, "random"), ("c5_d128_n16384", 8, "kmeans")]
+
+
+@pytest.mark.parametrize("name,bits,perm_kind", CASES, ids=[f"{c[0]}-{c[1]}bit" for c in CASES])
+def test_fullsize_sampled_parity(name, bits, perm_kind):
+    w = vc_inputs.WORKLOADS[name]
+    q, k, v = vc_inputs.make_qkv(w, device="cuda")
+    perm = vc_inputs.kmeans_perm_all(v, iters=2) if perm_kind == "kmeans" else vc_inputs.random_perm(w.B, w.H, w.N, w.seed, device="cuda")
+    p = Params.make(w.B, w.H, w.N, w.d, w.grid, bits=bits)
+    quant, work = alloc_buffers(p)
+    o = torch.empty(w.B, w.H, w.N, w.d, dtype=torch.bfloat16, device="cuda")
+    if bits == 8:
+        vc.vc_attn(p, q, k, v, perm, o, quant, work)
+        vc.vc_poll_status(work)
+    else:
+        vc.vc_prep(p, q, k, v, perm, quant, work)       # the 4-bit attention kernel is not built yet
+    torch.cuda.synchronize()
+    got = Hh.gpu_sections(p, quant)
+    nb = (w.N + 127) // 128
+    tiles = sorted({0, nb // 3, (2 * nb) // 3 + 1, nb - 1})
+    rows = np.concatenate([np.arange(128 * t, min(128 * (t + 1), w.N)) for t in tiles])
+    for (b, h) in [(0, 0), (w.B - 1, w.H - 1)]:
+        ref, cfg = Hh.oracle_prep(p, q, k, v, perm, b, h)
+        stats = Hh.check_prep_head(p, got, b * w.H + h, ref, what=f"{name} b{b} h{h}")
+        if bits == 8:
+            o_ref = OA.emulate_head(ref, cfg, rows=rows)
+            vmax = float(v[b, h].float().abs().max())
+            m = Hh.check_output(o[b, h].float().cpu().numpy()[rows], o_ref, vmax)
+            print(name, bits, (b, h), stats, m)
