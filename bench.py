@@ -162,6 +162,9 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-sdpa", action="store_true")
+    ap.add_argument("--data", default="workload", choices=["workload", "gauss"],
+                    help="gauss: same shapes, inputs drawn with three randn calls (for profiler runs, where the\n"
+                         "thousands of small generator kernels of the workload recipe would dominate the capture)")
     args = ap.parse_args()
     w = vc_inputs.WORKLOADS[args.workload]
     rank = int(os.environ.get("RANK", "0"))
@@ -186,7 +189,11 @@ def main():
     sampler = ClockSampler(local_rank)
     sampler.start()
     # every rank runs the same workload on its own GPU (heads are independent: no collective)
-    q, k, v = vc_inputs.make_qkv(w, device=dev)
+    if args.data == "gauss":
+        g = torch.Generator(device=dev).manual_seed(w.seed)
+        q, k, v = [torch.randn(w.B, w.H, w.N, w.d, generator=g, device=dev).to(torch.bfloat16) for _ in range(3)]
+    else:
+        q, k, v = vc_inputs.make_qkv(w, device=dev)
     if args.perm == "kmeans":
         perm = vc_inputs.kmeans_perm_all(v)
     elif args.perm == "random":
@@ -280,7 +287,7 @@ def main():
         "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "e4m3" if args.bits == 8 else "nvfp4", "data": "synthetic",
         "config": {"workload": w.name, "B": w.B, "H": w.H, "N": w.N, "d": w.d, "grid": list(w.grid),
-                   "bits": args.bits, "perm": args.perm, "l2": "inputs larger than L2 (Q+K+V = %.0f MB)" % (3 * q.numel() * 2 / 1e6),
+                   "bits": args.bits, "perm": args.perm, "data": args.data, "l2": "inputs larger than L2 (Q+K+V = %.0f MB)" % (3 * q.numel() * 2 / 1e6),
                    "step": "vc_prep + vc_attn_fwd"},
         "clocks": clocks, "gpu_launches": launches, "e2e": e2e,
         "roofline": {"bound": "tensor", "kernel": "vc_attn_fwd", "achieved": achieved, "peak": peak, "unit": UNIT,
