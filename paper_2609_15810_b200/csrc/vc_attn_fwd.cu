@@ -215,34 +215,39 @@ attn_fwd_serial_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
 // ---------------------------------------------------------------------------------------
 // Two-query-tile kernel (default).  A CTA owns TWO 128-row query tiles of one (batch, head)
 // and streams each K^_j / R^_j tile through both, so every key/value byte fetched from L2
-// feeds 256 query rows.  The probability codes travel through SHARED memory, not through the
-// score columns of tensor memory: a score tile is free again as soon as its 128 x 128 values
-// are in registers, so S_t(j+1) = Q^_t K^_{j+1}^T is computed while the softmax warpgroup is
-// still turning S_t(j) into codes, and the warpgroup never waits for the tensor core.
+// feeds 256 query rows.  Two decisions keep the softmax stage - the bottleneck on this GPU -
+// as short as the method allows:
+//   * The probability codes travel through SHARED memory, not through tensor memory, so a
+//     score tile is free as soon as its 128 x 128 values are in registers; one score buffer
+//     serves both query tiles in turn and S_t(j+1) is ready long before it is needed.
+//   * The row sums of the decoded codes (Eq. 6: r_ij, and the normalizer l) come from the
+//     tensor core: the value operand carries 16 extra rows of ones, so columns d..d+15 of the
+//     accumulator hold l, rescaled by alpha together with the rest.  The softmax threads do
+//     nothing but max, one fma.sat, one magic-number FMA and byte packing per score.
 //
 //   warp 0        TMA producer: Q0, Q1 once; then per key tile K^_j, R^_j and the tile's block
 //                 mean (as a [d x 8] TF32 operand) through a 4-stage ring
-//   warp 1        MMA issuer (one thread), per key tile j and query tile t:
-//                   S_t  = Q^_t K^_{j+1}^T   4 x kind::f8f6f4, as soon as S_t(j) has been read
-//                   A_t += P^_t R^_j         4 x kind::f8f6f4, P^ codes from shared memory
-//                   A_t += [r_hi r_lo] mu~_j 1 x kind::tf32: the rank-one mean term of Eq. 6
+//   warps 1, 3    MMA issuer of query tile 0 / 1 (one elected lane each), per key tile j:
+//                   S    = Q^_t K^_{j+1}^T     4 x kind::f8f6f4, once the other tile's scores are read
+//                   A_t += P^_t(j) [R^_j | 1]  4 x kind::f8f6f4, N = d + 16, codes from shared memory
+//                   A_t += rho_{j-1} mu~_{j-1} 1 x kind::tf32: the rank-one mean term of Eq. 6, one
+//                                              tile late, because r_{j-1} is read back from A_t first
 //   warps 4-7     softmax warpgroup of tile 0, one thread per query row (128 scores in
-//   warps 8-11    registers); likewise tile 1.  Running max, alpha, ExpCast-FP8 codes by
-//                 fma.sat + magic-number rounding (Eq. 7: no exponential, no conversion), row
-//                 sum of the decoded codes, l; writes the code tile in the 128-byte-swizzled
-//                 K-major layout the tensor core reads, and the output at the end
-//   warps 12-15   correction warpgroup of tile 0 (16-19: tile 1): rescales A_t by alpha when
-//                 a row maximum moved
+//   warps 8-11    registers); likewise tile 1: running max, alpha, ExpCast-FP8 codes (Eq. 7: no
+//                 exponential, no conversion), code tile in the swizzled K-major layout
+//   warps 12-15   correction warpgroup of tile 0 (16-19: tile 1), one thread per row: reads l
+//                 back, r_{j-1} = l_{j-1} - alpha_{j-1} l_{j-2}, rescales A_t by alpha_j when a
+//                 row maximum moved, hands (r_hi, r_lo) alpha_j to the mean MMA, writes the output
 //
-// Tensor memory (512 columns): S_0 | S_1 | A_0 | A_1, 128 columns each.
+// Tensor memory: S (128 columns) | A_0 (d + 16) | A_1 (d + 16).
 constexpr int kStages2 = 4;
 constexpr uint32_t kWaitLimit2 = 1u << 18;   // x up to 4 us per try: about one second
 
 struct FaSmem {
   uint64_t q_full, kv_full[kStages2], kv_empty[kStages2];
-  uint64_t s_full[2], s_free[2], o_done[2];
-  // alpha and codes+correction hand-offs can run one key tile ahead of their consumer (the score
-  // tile of j+1 is ready before the codes of j are consumed), so they alternate between two barriers
+  uint64_t s_full[2], s_free[2], o_done[2], fin_full[2], o_final[2];
+  // alpha and codes+correction hand-offs can run one key tile ahead of their consumer, so they
+  // alternate between two barriers (a parity wait aliases after two phases)
   uint64_t a_full[2][2], pc_full[2][2];
   float alpha[2][128];
   uint32_t tmem_base;
@@ -269,19 +274,20 @@ attn_fwd_2q_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                    const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_mu,
                    const AttnArgs a) {
   constexpr int kTmemCols = 512;
+  constexpr uint32_t O_COL = 128, O_STRIDE = 144, L_COL = D;   // A_t at O_COL + t * O_STRIDE; l in its column d
   // Register re-partition (setmaxnreg): the CTA owns 640 x 96 registers; a warpgroup that asks for
   // more than the others released would block forever, so the budget is checked at compile time.
   constexpr int kRegCtl = 48, kRegSoftmax = 160, kRegCorr = 56;
   static_assert(kRegCtl + 2 * kRegSoftmax + 2 * kRegCorr <= 5 * 96, "register budget exceeds the CTA's allocation");
-  constexpr uint32_t kQBytes = 128 * D, kKBytes = 128 * D, kVBytes = D * 128, kMuBytes = D * 32;
-  constexpr uint32_t kStageBytes = kKBytes + kVBytes + ((kMuBytes + 1023) / 1024) * 1024;
+  constexpr uint32_t kQBytes = 128 * D, kKBytes = 128 * D, kVBytes = D * 128, kOnesBytes = 16 * 128, kMuBytes = D * 32;
+  constexpr uint32_t kStageBytes = kKBytes + kVBytes + kOnesBytes + ((kMuBytes + 1023) / 1024) * 1024;
   constexpr uint32_t kPBytes = 128 * 128, kAmBytes = 128 * 32;
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   unsigned char* sQ = smem;                                    // [2][128 x D]
   unsigned char* sP = smem + 2 * kQBytes;                      // [2][128 x 128] probability codes
   unsigned char* sAm = sP + 2 * kPBytes;                       // [2][128 x 8 fp32] row-sum pairs
-  unsigned char* sStage = sAm + 2 * kAmBytes;                  // [kStages2]{K, V, Mu}
+  unsigned char* sStage = sAm + 2 * kAmBytes;                  // [kStages2]{K, V | ones, Mu}
   FaSmem* sh = reinterpret_cast<FaSmem*>(sStage + kStages2 * kStageBytes);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -293,6 +299,7 @@ attn_fwd_2q_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
     for (int i = 0; i < kStages2; ++i) { mbar_init(&sh->kv_full[i], 1); mbar_init(&sh->kv_empty[i], 2); }
     for (int i = 0; i < 2; ++i) {
       mbar_init(&sh->s_full[i], 1); mbar_init(&sh->s_free[i], 128); mbar_init(&sh->o_done[i], 1);
+      mbar_init(&sh->fin_full[i], 128); mbar_init(&sh->o_final[i], 1);
       for (int b = 0; b < 2; ++b) { mbar_init(&sh->a_full[i][b], 128); mbar_init(&sh->pc_full[i][b], 256); }
     }
     sh->abort = 0;
@@ -300,6 +307,9 @@ attn_fwd_2q_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
     tma_prefetch_desc(&tm_q); tma_prefetch_desc(&tm_k); tma_prefetch_desc(&tm_v); tma_prefetch_desc(&tm_mu);
   }
   for (int i = tid; i < 2 * (int)kAmBytes / 16; i += 640) reinterpret_cast<uint4*>(sAm)[i] = make_uint4(0, 0, 0, 0);
+  // 16 rows of E4M3 1.0 behind every value tile (the rows are uniform, so the swizzle is moot)
+  for (int i = tid; i < kStages2 * (int)kOnesBytes / 4; i += 640)
+    reinterpret_cast<uint32_t*>(sStage + (i / (kOnesBytes / 4)) * kStageBytes + kKBytes + kVBytes)[i % (kOnesBytes / 4)] = 0x38383838u;
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy stores -> tensor-core reads
   if (warp == 2) { tmem_alloc<kTmemCols>(&sh->tmem_base); tmem_relinquish(); }
   tc_fence_before();
@@ -326,23 +336,24 @@ attn_fwd_2q_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
           mbar_expect_tx(&sh->kv_full[st], kKBytes + kVBytes + kMuBytes);
           tma_load_3d(base, &tm_k, &sh->kv_full[st], 0, j * 128, bh);
           tma_load_3d(base + kKBytes, &tm_v, &sh->kv_full[st], j * 128, 0, bh);
-          tma_load_3d(base + kKBytes + kVBytes, &tm_mu, &sh->kv_full[st], 0, 0, bh * nb + j);
+          tma_load_3d(base + kKBytes + kVBytes + kOnesBytes, &tm_mu, &sh->kv_full[st], 0, 0, bh * nb + j);
         }
         __syncwarp();
       }
     } else if (warp == 1 || warp == 3) {
       // ------------------------------------------------------------------ MMA issuers
       // One warp per query tile (they sit on different schedulers).  Every wait on the way to an
-      // MMA is a shared-memory round trip, so each issuer waits for as little as possible: per key
-      // tile one barrier before S_t(j+1) and one before the A_t update.  The whole warp runs the
-      // loop so that descriptors stay in uniform registers; one elected lane issues.
+      // MMA is a shared-memory round trip, so each issuer waits for as little as possible.  The
+      // whole warp runs the loop so that descriptors stay in uniform registers; one lane issues.
       const int t = warp >> 1;
-      const uint32_t idesc_qk = idesc_e4m3(128, 128), idesc_pv = idesc_e4m3(128, D), idesc_mu = idesc_tf32(128, D);
+      const uint32_t idesc_qk = idesc_e4m3(128, 128), idesc_pv = idesc_e4m3(128, D + 16), idesc_mu = idesc_tf32(128, D);
       const uint64_t dq = smem_desc_kmajor(smem_u32(sQ + t * kQBytes), D);
       const uint64_t dp = smem_desc_kmajor(smem_u32(sP + t * kPBytes), 128);
       const uint64_t dam = smem_desc_kmajor(smem_u32(sAm + t * kAmBytes), 32);
-      const uint32_t s_col = tmem + 128 * t, o_col = tmem + 256 + 128 * t;
+      const uint32_t s_col = tmem, o_col = tmem + O_COL + O_STRIDE * t;
       bool ok = warp_wait2(&sh->q_full, 0, sh, a.status, 20) && warp_wait2(&sh->kv_full[0], 0, sh, a.status, 21);
+      // the score buffer alternates S_0(0), S_1(0), S_0(1), ...: tile 1 starts after tile 0's first read
+      if (ok && t == 1) ok = warp_wait2(&sh->s_free[0], 0, sh, a.status, 22);
       if (ok && elect_one()) {
         tc_fence_after();
         const uint64_t dk = smem_desc_kmajor(smem_u32(sStage), D);
@@ -353,9 +364,11 @@ attn_fwd_2q_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
       __syncwarp();
       for (int j = 0; ok && j < nb; ++j) {
         const int st = j % kStages2;
-        if (j + 1 < nb) {                                 // S_t(j+1), as soon as the scores of (t, j) were read
+        if (j + 1 < nb) {
+          // S_t(j+1) may overwrite the buffer once the OTHER tile's latest scores were read:
+          // S_1(j) for tile 0, S_0(j+1) for tile 1
           const int st1 = (j + 1) % kStages2, it1 = (j + 1) / kStages2;
-          if (!(ok = warp_wait2(&sh->s_free[t], j & 1, sh, a.status, 22))) break;
+          if (!(ok = warp_wait2(&sh->s_free[1 - t], (j + t) & 1, sh, a.status, 22))) break;
           if (!(ok = warp_wait2(&sh->kv_full[st1], it1 & 1, sh, a.status, 25))) break;
           const uint64_t dk = smem_desc_kmajor(smem_u32(sStage + st1 * kStageBytes), D);
           if (elect_one()) {
@@ -366,18 +379,29 @@ attn_fwd_2q_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
           }
           __syncwarp();
         }
-        // A_t += P^_t(j) R^_j + r mu~_j, once the codes are written and A_t is rescaled
+        // A_t += P^_t(j) [R^_j | 1] once the codes are written, A_t is rescaled by alpha_j and the
+        // row-sum pair of tile j-1 is in place; then the mean term of tile j-1
         if (!(ok = warp_wait2(&sh->pc_full[t][j & 1], (j >> 1) & 1, sh, a.status, 23))) break;
-        unsigned char* base = sStage + st * kStageBytes;
-        const uint64_t dv = smem_desc_kmajor(smem_u32(base + kKBytes), 128);
-        const uint64_t dm = smem_desc_kmajor(smem_u32(base + kKBytes + kVBytes), 32);
+        const uint64_t dv = smem_desc_kmajor(smem_u32(sStage + st * kStageBytes + kKBytes), 128);
+        const int stp = (j + kStages2 - 1) % kStages2;    // stage of tile j-1
+        const uint64_t dm = smem_desc_kmajor(smem_u32(sStage + stp * kStageBytes + kKBytes + kVBytes + kOnesBytes), 32);
         if (elect_one()) {
           tc_fence_after();
 #pragma unroll
           for (int k = 0; k < 4; ++k) mma_f8_ss(o_col, dp + 2 * k, dv + 2 * k, idesc_pv, (j > 0) | (k > 0));
-          mma_tf32_ss(o_col, dam, dm, idesc_mu, 1);
+          if (j > 0) mma_tf32_ss(o_col, dam, dm, idesc_mu, 1);
           mma_commit(&sh->o_done[t]);
-          mma_commit(&sh->kv_empty[st]);                  // this tile is done with stage j
+          if (j > 0) mma_commit(&sh->kv_empty[stp]);      // this tile is done with stage j-1
+        }
+        __syncwarp();
+      }
+      if (ok && warp_wait2(&sh->fin_full[t], 0, sh, a.status, 27)) {   // mean term of the last tile
+        const int stp = (nb - 1) % kStages2;
+        const uint64_t dm = smem_desc_kmajor(smem_u32(sStage + stp * kStageBytes + kKBytes + kVBytes + kOnesBytes), 32);
+        if (elect_one()) {
+          tc_fence_after();
+          mma_tf32_ss(o_col, dam, dm, idesc_mu, 1);
+          mma_commit(&sh->o_final[t]);
         }
         __syncwarp();
       }
@@ -388,24 +412,20 @@ attn_fwd_2q_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
     const int t = (warp - 4) >> 2;                         // query tile of this warpgroup
     const int row = (warp & 3) * 32 + lane;
     const int qblk = 2 * qpair + t;
-    const uint32_t s_base = lane_base + 128 * t, o_base = lane_base + 256 + 128 * t;
     // my row of the swizzled code tile: 16-byte chunk c sits at chunk position c ^ (row % 8)
     unsigned char* p_row = sP + t * kPBytes + (row >> 3) * 1024 + (row & 7) * 128;
-    // my row of the row-sum operand: 32-byte rows, the two 16-byte chunks swap when (row / 4) is odd
-    uint4* am_row = reinterpret_cast<uint4*>(sAm + t * kAmBytes + row * 32 + 16 * ((row >> 2) & 1));
     const float sq = qblk < nb ? a.q_scale[(size_t)bh * nb + qblk] : 1.0f;
-    float m_run = -INFINITY, l_run = 0.f;
-    bool ok = true;
+    float m_run = -INFINITY;
     for (int j = 0; j < nb; ++j) {
       const int ph = j & 1;
       const float cs = (sq * __ldg(&a.k_scale[(size_t)bh * nb + j])) * a.sl;
-      if (!(ok = warp_wait2(&sh->s_full[t], ph, sh, a.status, 30))) break;
+      if (!warp_wait2(&sh->s_full[t], ph, sh, a.status, 30)) break;
       tc_fence_after();
       uint32_t s0[32], s1[32], s2[32], s3[32];
-      tmem_ld32(s_base, s0); tmem_ld32(s_base + 32, s1); tmem_ld32(s_base + 64, s2); tmem_ld32(s_base + 96, s3);
+      tmem_ld32(lane_base, s0); tmem_ld32(lane_base + 32, s1); tmem_ld32(lane_base + 64, s2); tmem_ld32(lane_base + 96, s3);
       tmem_wait_ld();
       tc_fence_before();
-      mbar_arrive(&sh->s_free[t]);                        // the score columns may be overwritten
+      mbar_arrive(&sh->s_free[t]);                        // the score buffer may be overwritten
       const int nv = a.N - j * 128;                       // >= 128 except on the ragged last tile
       if (nv < 128) {                                     // padded keys never win the maximum
 #pragma unroll
@@ -437,14 +457,12 @@ attn_fwd_2q_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
       }
       const float mxa = max3(max3(mx[0], mx[1], mx[2]), max3(mx[3], mx[4], mx[5]), fmaxf(mx[6], mx[7]));
       const float m_new = fmaxf(m_run, mxa * cs);         // m' = max(m, rowmax S_ij)
-      const float alpha = ex2_approx(m_run - m_new);      // 0 on the first tile
-      sh->alpha[t][row] = alpha;
+      sh->alpha[t][row] = ex2_approx(m_run - m_new);      // alpha; 0 on the first tile
       mbar_arrive(&sh->a_full[t][j & 1]);
       m_run = m_new;
       // the previous code tile must have been consumed before it is overwritten
-      if (j > 0 && !(ok = warp_wait2(&sh->o_done[t], (j - 1) & 1, sh, a.status, 31))) break;
+      if (j > 0 && !warp_wait2(&sh->o_done[t], (j - 1) & 1, sh, a.status, 31)) break;
 
-      float acc0 = 0.f, acc1 = 0.f, acc2 = 0.f, acc3 = 0.f;
       const float fa = cs * 0.0625f, fb = (a.code_off - 8.0f * m_new) * 0.0078125f, nm = 8.0f - m_new;
       auto code4 = [&](const uint32_t (&sv)[32], int w) -> uint32_t {
         if constexpr (EXPCAST) {
@@ -454,9 +472,6 @@ attn_fwd_2q_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
           const uint32_t r1 = __float_as_uint(fmaf(fma_sat(__uint_as_float(sv[4 * w + 1]), fa, fb), 128.0f, 12582912.0f));
           const uint32_t r2 = __float_as_uint(fmaf(fma_sat(__uint_as_float(sv[4 * w + 2]), fa, fb), 128.0f, 12582912.0f));
           const uint32_t r3 = __float_as_uint(fmaf(fma_sat(__uint_as_float(sv[4 * w + 3]), fa, fb), 128.0f, 12582912.0f));
-          // (code << 20) read as fp32 is the decoded E4M3 value times 2^-120, subnormal codes included
-          acc0 += __uint_as_float(r0 << 20); acc1 += __uint_as_float(r1 << 20);
-          acc2 += __uint_as_float(r2 << 20); acc3 += __uint_as_float(r3 << 20);
           return __byte_perm(__byte_perm(r0, r1, 0x0040), __byte_perm(r2, r3, 0x0040), 0x5410);
         } else {
           // exponentiate, then cast (Fig. 4a upper box)
@@ -464,8 +479,6 @@ attn_fwd_2q_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
           const float p2 = exp2f(fmaf(__uint_as_float(sv[4 * w + 2]), cs, nm)), p3 = exp2f(fmaf(__uint_as_float(sv[4 * w + 3]), cs, nm));
           const uint32_t lo = __nv_cvt_float2_to_fp8x2(make_float2(p0, p1), __NV_SATFINITE, __NV_E4M3);
           const uint32_t hi = __nv_cvt_float2_to_fp8x2(make_float2(p2, p3), __NV_SATFINITE, __NV_E4M3);
-          acc0 += __uint_as_float((lo & 0xffu) << 20); acc1 += __uint_as_float((lo >> 8) << 20);
-          acc2 += __uint_as_float((hi & 0xffu) << 20); acc3 += __uint_as_float((hi >> 8) << 20);
           return lo | (hi << 16);
         }
       };
@@ -475,63 +488,84 @@ attn_fwd_2q_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
       };
       store16(s0, 0, 0); store16(s0, 1, 1); store16(s1, 0, 2); store16(s1, 1, 3);
       store16(s2, 0, 4); store16(s2, 1, 5); store16(s3, 0, 6); store16(s3, 1, 7);
-      const float rs = (((acc0 + acc1) + (acc2 + acc3)) * 1152921504606846976.0f) * 1152921504606846976.0f;   // x 2^120
-      l_run = alpha * l_run + rs;                         // l <- alpha l + r,  r = P~ 1 over the decoded codes
-      const uint32_t hi = (__float_as_uint(rs) + 0x1000u) & 0xffffe000u;     // nearest TF32
-      *am_row = make_uint4(hi, __float_as_uint(rs - __uint_as_float(hi)), 0u, 0u);
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");          // my stores -> tensor-core reads
       mbar_arrive(&sh->pc_full[t][j & 1]);
-    }
-    // ---- epilogue: O = s_V * A / l
-    if (ok && warp_wait2(&sh->o_done[t], (nb - 1) & 1, sh, a.status, 33)) {
-      tc_fence_after();
-      const int grow = qblk * 128 + row;
-      const float inv_l = 1.0f / l_run;
-      uint32_t r[32];
-#pragma unroll 1
-      for (int c = 0; c < D / 32; ++c) {
-        tmem_ld32(o_base + 32 * c, r);
-        tmem_wait_ld();
-        if (grow < a.N) {
-          uint32_t out[16];
-#pragma unroll
-          for (int i = 0; i < 16; ++i) {
-            const float x0 = __uint_as_float(r[2 * i]) * inv_l * __ldg(&a.v_scale[(size_t)bh * D + 32 * c + 2 * i]);
-            const float x1 = __uint_as_float(r[2 * i + 1]) * inv_l * __ldg(&a.v_scale[(size_t)bh * D + 32 * c + 2 * i + 1]);
-            __nv_bfloat162 h2 = __floats2bfloat162_rn(x0, x1);
-            out[i] = *reinterpret_cast<uint32_t*>(&h2);
-          }
-          uint4* dst = reinterpret_cast<uint4*>(a.o + ((size_t)bh * a.N + grow) * D + 32 * c);
-#pragma unroll
-          for (int i = 0; i < 4; ++i) dst[i] = make_uint4(out[4 * i], out[4 * i + 1], out[4 * i + 2], out[4 * i + 3]);
-        }
-      }
     }
   } else {
     // -------------------------------------------------------------------- correction warpgroups
     reg_dec<kRegCorr>();
     const int t = (warp - 12) >> 2;
     const int row = (warp & 3) * 32 + lane;
-    const uint32_t o_base = lane_base + 256 + 128 * t;
+    const int qblk = 2 * qpair + t;
+    const uint32_t o_base = lane_base + O_COL + O_STRIDE * t;
+    // my row of the row-sum operand: 32-byte rows, the two 16-byte chunks swap when (row / 4) is odd
+    uint4* am_row = reinterpret_cast<uint4*>(sAm + t * kAmBytes + row * 32 + 16 * ((row >> 2) & 1));
+    float l_resc = 0.f;       // l as it stands in column d after the latest rescale, before the tile's own sum
+    float l_now = 0.f;
+    bool ok = true;
+    auto put_pair = [&](float rho) {                      // (rho_hi, rho_lo, 0, 0) for the mean MMA
+      const uint32_t hi = (__float_as_uint(rho) + 0x1000u) & 0xffffe000u;   // nearest TF32
+      *am_row = make_uint4(hi, __float_as_uint(rho - __uint_as_float(hi)), 0u, 0u);
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    };
     for (int j = 0; j < nb; ++j) {
-      if (!warp_wait2(&sh->a_full[t][j & 1], (j >> 1) & 1, sh, a.status, 40)) break;
+      if (!(ok = warp_wait2(&sh->a_full[t][j & 1], (j >> 1) & 1, sh, a.status, 40))) break;
       const float alpha = sh->alpha[t][row];
-      if (j > 0 && __any_sync(0xffffffffu, alpha != 1.0f)) {
-        if (!warp_wait2(&sh->o_done[t], (j - 1) & 1, sh, a.status, 41)) break;
+      if (j > 0) {
+        if (!(ok = warp_wait2(&sh->o_done[t], (j - 1) & 1, sh, a.status, 41))) break;
         tc_fence_after();
-        uint32_t r[32];
+        l_now = __uint_as_float(tmem_ld1(o_base + L_COL));   // l after tile j-1
+        tmem_wait_ld();
+        const float r_prev = l_now - l_resc;                 // r_{j-1} = P~ 1 over the decoded codes
+        if (__any_sync(0xffffffffu, alpha != 1.0f)) {        // a row maximum moved: A <- alpha A (l included)
+          uint32_t r[16];
 #pragma unroll 1
-        for (int c = 0; c < D / 32; ++c) {
-          tmem_ld32(o_base + 32 * c, r);
-          tmem_wait_ld();
+          for (int c = 0; c < (D + 16) / 16; ++c) {
+            tmem_ld16(o_base + 16 * c, r);
+            tmem_wait_ld();
 #pragma unroll
-          for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * alpha);
-          tmem_st32(o_base + 32 * c, r);
+            for (int i = 0; i < 16; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * alpha);
+            tmem_st16(o_base + 16 * c, r);
+          }
+          tmem_wait_st();
+          tc_fence_before();
         }
-        tmem_wait_st();
-        tc_fence_before();
+        l_resc = l_now * alpha;
+        put_pair(r_prev * alpha);                            // added after the rescale, so referenced to m_j
       }
       mbar_arrive(&sh->pc_full[t][j & 1]);
+    }
+    // ---- last tile's mean term, then the epilogue: O = s_V * A / l
+    if (ok && (ok = warp_wait2(&sh->o_done[t], (nb - 1) & 1, sh, a.status, 42))) {
+      tc_fence_after();
+      l_now = __uint_as_float(tmem_ld1(o_base + L_COL));
+      tmem_wait_ld();
+      put_pair(l_now - l_resc);
+      mbar_arrive(&sh->fin_full[t]);
+    }
+    if (ok && warp_wait2(&sh->o_final[t], 0, sh, a.status, 43)) {
+      tc_fence_after();
+      const int grow = qblk * 128 + row;
+      const float inv_l = 1.0f / l_now;
+#pragma unroll 1
+      for (int c = 0; c < D / 16; ++c) {
+        uint32_t r[16];
+        tmem_ld16(o_base + 16 * c, r);
+        tmem_wait_ld();
+        if (grow < a.N) {
+          uint32_t out[8];
+#pragma unroll
+          for (int i = 0; i < 8; ++i) {
+            const float x0 = __uint_as_float(r[2 * i]) * inv_l * __ldg(&a.v_scale[(size_t)bh * D + 16 * c + 2 * i]);
+            const float x1 = __uint_as_float(r[2 * i + 1]) * inv_l * __ldg(&a.v_scale[(size_t)bh * D + 16 * c + 2 * i + 1]);
+            __nv_bfloat162 h2 = __floats2bfloat162_rn(x0, x1);
+            out[i] = *reinterpret_cast<uint32_t*>(&h2);
+          }
+          uint4* dst = reinterpret_cast<uint4*>(a.o + ((size_t)bh * a.N + grow) * D + 16 * c);
+          dst[0] = make_uint4(out[0], out[1], out[2], out[3]);
+          dst[1] = make_uint4(out[4], out[5], out[6], out[7]);
+        }
+      }
     }
   }
   tc_fence_before();
@@ -613,7 +647,7 @@ cudaError_t run8(const Problem& pr, const QuantLayout& ql, const WorkLayout& wl,
     if (!make_map(&tmt, work + wl.mu_mma, 32, D, (uint64_t)pr.BH * pr.nb, 32, D)) return cudaErrorUnknown;
     const size_t n = (size_t)pr.BH * pr.nb * D;
     means_tile_layout_kernel<D><<<(unsigned)((n + 255) / 256), 256, 0, s>>>(a.v_means, (float*)(work + wl.mu_mma), n);
-    const size_t stage = 2 * 128 * D + ((D * 32 + 1023) / 1024) * 1024;
+    const size_t stage = 2 * 128 * D + 2048 + ((D * 32 + 1023) / 1024) * 1024;
     const size_t smem2 = 1024 + 2 * 128 * D + 2 * 128 * 128 + 2 * 128 * 32 + kStages2 * stage + sizeof(FaSmem);
     const dim3 grid((pr.nb + 1) / 2, pr.BH);
     if (pr.p_format == VC_P_EXPCAST_E4M3) {
