@@ -227,8 +227,9 @@ attn_fwd_serial_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
 //
 //   warp 0        TMA producer: Q0, Q1 once; then per key tile K^_j, R^_j and the tile's block
 //                 mean (as a [d x 8] TF32 operand) through a 4-stage ring
-//   warps 1, 3    MMA issuer of query tile 0 / 1 (one elected lane each), per key tile j:
-//                   S    = Q^_t K^_{j+1}^T     4 x kind::f8f6f4, once the other tile's scores are read
+//   warp 1        score issuer (one elected lane), per key tile j and query tile t:
+//                   S    = Q^_t K^_j^T         4 x kind::f8f6f4, once the previous scores are read
+//   warp 3        accumulator issuer, per key tile j and query tile t:
 //                   A_t += P^_t(j) [R^_j | 1]  4 x kind::f8f6f4, N = d + 16, codes from shared memory
 //                   A_t += rho_{j-1} mu~_{j-1} 1 x kind::tf32: the rank-one mean term of Eq. 6, one
 //                                              tile late, because r_{j-1} is read back from A_t first
@@ -340,67 +341,72 @@ attn_fwd_2q_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         }
         __syncwarp();
       }
-    } else if (warp == 1 || warp == 3) {
-      // ------------------------------------------------------------------ MMA issuers
-      // One warp per query tile (they sit on different schedulers).  Every wait on the way to an
-      // MMA is a shared-memory round trip, so each issuer waits for as little as possible.  The
-      // whole warp runs the loop so that descriptors stay in uniform registers; one lane issues.
-      const int t = warp >> 1;
-      const uint32_t idesc_qk = idesc_e4m3(128, 128), idesc_pv = idesc_e4m3(128, D + 16), idesc_mu = idesc_tf32(128, D);
-      const uint64_t dq = smem_desc_kmajor(smem_u32(sQ + t * kQBytes), D);
-      const uint64_t dp = smem_desc_kmajor(smem_u32(sP + t * kPBytes), 128);
-      const uint64_t dam = smem_desc_kmajor(smem_u32(sAm + t * kAmBytes), 32);
-      const uint32_t s_col = tmem, o_col = tmem + O_COL + O_STRIDE * t;
-      bool ok = warp_wait2(&sh->q_full, 0, sh, a.status, 20) && warp_wait2(&sh->kv_full[0], 0, sh, a.status, 21);
-      // the score buffer alternates S_0(0), S_1(0), S_0(1), ...: tile 1 starts after tile 0's first read
-      if (ok && t == 1) ok = warp_wait2(&sh->s_free[0], 0, sh, a.status, 22);
-      if (ok && elect_one()) {
-        tc_fence_after();
-        const uint64_t dk = smem_desc_kmajor(smem_u32(sStage), D);
-#pragma unroll
-        for (int k = 0; k < D / 32; ++k) mma_f8_ss(s_col, dq + 2 * k, dk + 2 * k, idesc_qk, k > 0);
-        mma_commit(&sh->s_full[t]);
-      }
-      __syncwarp();
+    } else if (warp == 1) {
+      // ------------------------------------------------------------------ score issuer
+      // Issues S_t = Q^_t K^_jT for both query tiles into the ONE score buffer, in the fixed order
+      // S_0(0), S_1(0), S_0(1), S_1(1), ...: each may overwrite the buffer as soon as the previous
+      // one has been read into registers.  (The whole warp runs the loop so that descriptors stay
+      // in uniform registers; one elected lane issues.  A separate warp issues the A_t updates, so
+      // that neither kind of MMA ever waits behind a barrier that only the other kind needs.)
+      const uint32_t idesc_qk = idesc_e4m3(128, 128);
+      const uint64_t dq0 = smem_desc_kmajor(smem_u32(sQ), D), dq1 = smem_desc_kmajor(smem_u32(sQ + kQBytes), D);
+      bool ok = warp_wait2(&sh->q_full, 0, sh, a.status, 20);
       for (int j = 0; ok && j < nb; ++j) {
-        const int st = j % kStages2;
-        if (j + 1 < nb) {
-          // S_t(j+1) may overwrite the buffer once the OTHER tile's latest scores were read:
-          // S_1(j) for tile 0, S_0(j+1) for tile 1
-          const int st1 = (j + 1) % kStages2, it1 = (j + 1) / kStages2;
-          if (!(ok = warp_wait2(&sh->s_free[1 - t], (j + t) & 1, sh, a.status, 22))) break;
-          if (!(ok = warp_wait2(&sh->kv_full[st1], it1 & 1, sh, a.status, 25))) break;
-          const uint64_t dk = smem_desc_kmajor(smem_u32(sStage + st1 * kStageBytes), D);
+        const int st = j % kStages2, it = j / kStages2;
+        if (!(ok = warp_wait2(&sh->kv_full[st], it & 1, sh, a.status, 21))) break;
+        const uint64_t dk = smem_desc_kmajor(smem_u32(sStage + st * kStageBytes), D);
+#pragma unroll
+        for (int t = 0; t < 2; ++t) {
+          // S_0(j) waits for the read of S_1(j-1), S_1(j) for the read of S_0(j)
+          if (t == 0 ? j > 0 : true) {
+            if (!(ok = warp_wait2(&sh->s_free[1 - t], (t == 0 ? j - 1 : j) & 1, sh, a.status, 22))) break;
+          }
           if (elect_one()) {
             tc_fence_after();
+            const uint64_t dq = t == 0 ? dq0 : dq1;
 #pragma unroll
-            for (int k = 0; k < D / 32; ++k) mma_f8_ss(s_col, dq + 2 * k, dk + 2 * k, idesc_qk, k > 0);
+            for (int k = 0; k < D / 32; ++k) mma_f8_ss(tmem, dq + 2 * k, dk + 2 * k, idesc_qk, k > 0);
             mma_commit(&sh->s_full[t]);
           }
           __syncwarp();
         }
-        // A_t += P^_t(j) [R^_j | 1] once the codes are written, A_t is rescaled by alpha_j and the
-        // row-sum pair of tile j-1 is in place; then the mean term of tile j-1
-        if (!(ok = warp_wait2(&sh->pc_full[t][j & 1], (j >> 1) & 1, sh, a.status, 23))) break;
-        const uint64_t dv = smem_desc_kmajor(smem_u32(sStage + st * kStageBytes + kKBytes), 128);
-        const int stp = (j + kStages2 - 1) % kStages2;    // stage of tile j-1
-        const uint64_t dm = smem_desc_kmajor(smem_u32(sStage + stp * kStageBytes + kKBytes + kVBytes + kOnesBytes), 32);
-        if (elect_one()) {
-          tc_fence_after();
-#pragma unroll
-          for (int k = 0; k < 4; ++k) mma_f8_ss(o_col, dp + 2 * k, dv + 2 * k, idesc_pv, (j > 0) | (k > 0));
-          if (j > 0) mma_tf32_ss(o_col, dam, dm, idesc_mu, 1);
-          mma_commit(&sh->o_done[t]);
-          if (j > 0) mma_commit(&sh->kv_empty[stp]);      // this tile is done with stage j-1
-        }
-        __syncwarp();
       }
-      if (ok && warp_wait2(&sh->fin_full[t], 0, sh, a.status, 27)) {   // mean term of the last tile
-        const int stp = (nb - 1) % kStages2;
+    } else if (warp == 3) {
+      // ------------------------------------------------------------------ accumulator issuer
+      // A_t += P^_t(j) [R^_j | 1] once the codes are written, A_t is rescaled by alpha_j and the
+      // row-sum pair of tile j-1 is in place; then the mean term of tile j-1.
+      const uint32_t idesc_pv = idesc_e4m3(128, D + 16), idesc_mu = idesc_tf32(128, D);
+      const uint64_t dp[2] = {smem_desc_kmajor(smem_u32(sP), 128), smem_desc_kmajor(smem_u32(sP + kPBytes), 128)};
+      const uint64_t dam[2] = {smem_desc_kmajor(smem_u32(sAm), 32), smem_desc_kmajor(smem_u32(sAm + kAmBytes), 32)};
+      bool ok = true;
+      for (int j = 0; ok && j < nb; ++j) {
+        const int st = j % kStages2, it = j / kStages2;
+        const int stp = (j + kStages2 - 1) % kStages2;    // stage of tile j-1
+        if (!(ok = warp_wait2(&sh->kv_full[st], it & 1, sh, a.status, 25))) break;
+        const uint64_t dv = smem_desc_kmajor(smem_u32(sStage + st * kStageBytes + kKBytes), 128);
         const uint64_t dm = smem_desc_kmajor(smem_u32(sStage + stp * kStageBytes + kKBytes + kVBytes + kOnesBytes), 32);
+#pragma unroll
+        for (int t = 0; t < 2; ++t) {
+          if (!(ok = warp_wait2(&sh->pc_full[t][j & 1], (j >> 1) & 1, sh, a.status, 23))) break;
+          if (elect_one()) {
+            tc_fence_after();
+            const uint32_t o_col = tmem + O_COL + O_STRIDE * t;
+#pragma unroll
+            for (int k = 0; k < 4; ++k) mma_f8_ss(o_col, dp[t] + 2 * k, dv + 2 * k, idesc_pv, (j > 0) | (k > 0));
+            if (j > 0) mma_tf32_ss(o_col, dam[t], dm, idesc_mu, 1);
+            mma_commit(&sh->o_done[t]);
+            if (j > 0) mma_commit(&sh->kv_empty[stp]);    // this tile is done with stage j-1
+          }
+          __syncwarp();
+        }
+      }
+      const uint64_t dml = smem_desc_kmajor(smem_u32(sStage + ((nb - 1) % kStages2) * kStageBytes + kKBytes + kVBytes + kOnesBytes), 32);
+#pragma unroll
+      for (int t = 0; t < 2; ++t) {                       // mean term of the last tile
+        if (!ok || !(ok = warp_wait2(&sh->fin_full[t], 0, sh, a.status, 27))) break;
         if (elect_one()) {
           tc_fence_after();
-          mma_tf32_ss(o_col, dam, dm, idesc_mu, 1);
+          mma_tf32_ss(tmem + O_COL + O_STRIDE * t, dam[t], dml, idesc_mu, 1);
           mma_commit(&sh->o_final[t]);
         }
         __syncwarp();
