@@ -11,6 +11,7 @@
 // major) and the V residual (channel-major), per-block scales, per-channel value scale and the
 // block means divided by it.  Epilogue: O = s_V * A / l, bf16, original query order.
 #include <cuda_bf16.h>
+#include <cuda_fp4.h>
 #include <cuda_fp8.h>
 
 #include "vc_internal.h"
@@ -591,6 +592,222 @@ __global__ void means_tile_layout_kernel(const __nv_bfloat16* __restrict__ means
   dst[1] = make_float4(0.f, 0.f, 0.f, 0.f);
 }
 
+
+// ---------------------------------------------------------------------------------------
+// 4-bit path (NVFP4 Q, K, R and P; App. A "Scope of ExpCast-FP8", App. B).
+//
+// An E2M1 element times its E4M3 microscale has at most six significant bits, so it is exact
+// in bf16: the operands are expanded once per call into bf16 tiles and the two products run as
+// kind::f16 MMAs with FP32 accumulation - bit-for-bit the arithmetic of a block-scaled FP4 MMA.
+// The probability tile is quantized to NVFP4 in the softmax stage (per row and 16 keys: E4M3
+// microscale of max p / 6, E2M1 elements) and handed to the tensor core as the exact bf16
+// values of those codes.  This kernel is the simple serial form (one query tile per CTA, every
+// step behind __syncthreads); the paper itself declines a 4-bit datacenter configuration
+// because the per-16 scale computation sits on the softmax critical path.
+__global__ void nvfp4_expand_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restrict__ micro,
+                                    __nv_bfloat16* __restrict__ out, size_t n_groups) {
+  const size_t g = (size_t)blockIdx.x * blockDim.x + threadIdx.x;   // one group of 16 elements
+  if (g >= n_groups) return;
+  const uint2 c = *reinterpret_cast<const uint2*>(codes + g * 8);
+  const __half_raw hs = __nv_cvt_fp8_to_halfraw((__nv_fp8_storage_t)micro[g], __NV_E4M3);
+  const float sdec = __half2float(__half(hs));
+  const uint32_t w[2] = {c.x, c.y};
+  uint32_t o[8];
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const __half2_raw h2 = __nv_cvt_fp4x2_to_halfraw2((__nv_fp4x2_storage_t)((w[i >> 2] >> (8 * (i & 3))) & 0xffu), __NV_E2M1);
+    const float2 f = __half22float2(__half2(h2));
+    __nv_bfloat162 b = __floats2bfloat162_rn(f.x * sdec, f.y * sdec);
+    o[i] = *reinterpret_cast<uint32_t*>(&b);
+  }
+  uint4* dst = reinterpret_cast<uint4*>(out + g * 16);
+  dst[0] = make_uint4(o[0], o[1], o[2], o[3]);
+  dst[1] = make_uint4(o[4], o[5], o[6], o[7]);
+}
+
+struct Attn4Args {
+  const float *q_g, *k_g;          // NVFP4 outer scales per (b, h)
+  const __nv_bfloat16* v_means;    // unscaled block means
+  __nv_bfloat16* o;
+  uint32_t* status;
+  int N, n_pad, nb;
+  float sl;
+};
+
+template <int D>
+__global__ void __launch_bounds__(128)
+attn_fwd_serial4_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
+                        const __grid_constant__ CUtensorMap tm_v, const Attn4Args a) {
+  constexpr int kTmemCols = 512;
+  constexpr uint32_t S_COL = 0, P_COL = 128, O_COL = 256;
+  constexpr int kQH = D / 64;                        // 128-byte column halves of a Q/K tile
+  constexpr uint32_t kHalfQ = 128 * 128, kHalfV = D * 128;
+  extern __shared__ unsigned char smem_raw[];
+  unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  unsigned char* sQ = smem;                          // [kQH][128 rows x 128 B]
+  unsigned char* sK = sQ + kQH * kHalfQ;             // [kQH][128 rows x 128 B]
+  unsigned char* sV = sK + kQH * kHalfQ;             // [2][D rows x 128 B]: tokens 0..63, 64..127
+  float* sMu = reinterpret_cast<float*>(sV + 2 * kHalfV);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(sMu + D);
+  uint64_t *bar_q = bars, *bar_kv = bars + 1, *bar_s = bars + 2, *bar_o = bars + 3;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 4);
+
+  const int tid = threadIdx.x, warp = tid >> 5;
+  const int qblk = blockIdx.x, bh = blockIdx.y;
+  bool alive = true;
+
+  if (tid == 0) {
+    mbar_init(bar_q, 1); mbar_init(bar_kv, 1); mbar_init(bar_s, 1); mbar_init(bar_o, 1);
+    mbar_fence_init();
+  }
+  if (warp == 0) { tmem_alloc<kTmemCols>(tmem_slot); tmem_relinquish(); }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *tmem_slot;
+  const uint32_t lane_base = tmem + ((uint32_t)(warp * 32) << 16);
+
+  if (tid == 0) {
+    mbar_expect_tx(bar_q, kQH * kHalfQ);
+    for (int h = 0; h < kQH; ++h) tma_load_3d(sQ + h * kHalfQ, &tm_q, bar_q, 128 * h, qblk * 128, bh);
+  }
+  if (!mbar_wait(bar_q, 0)) { alive = false; atomicExch(a.status, kErrTimeout | 1); }
+
+  const float cs = (a.q_g[bh] * a.k_g[bh]) * a.sl;   // code units -> log2 domain
+  const uint32_t idesc_qk = idesc_bf16(128, 128), idesc_pv = idesc_bf16(128, D);
+  float m_run = -INFINITY, l_run = 0.f;
+  for (int j = 0; j < a.nb; ++j) {
+    const uint32_t ph = j & 1;
+    if (tid == 0) {
+      mbar_expect_tx(bar_kv, kQH * kHalfQ + 2 * kHalfV);
+      for (int h = 0; h < kQH; ++h) tma_load_3d(sK + h * kHalfQ, &tm_k, bar_kv, 128 * h, j * 128, bh);
+      for (int h = 0; h < 2; ++h) tma_load_3d(sV + h * kHalfV, &tm_v, bar_kv, 2 * (j * 128 + 64 * h), 0, bh);
+    }
+    if (tid < D / 2) {
+      const __nv_bfloat162 m2 = *reinterpret_cast<const __nv_bfloat162*>(a.v_means + ((size_t)bh * a.nb + j) * D + 2 * tid);
+      sMu[2 * tid] = __low2float(m2);
+      sMu[2 * tid + 1] = __high2float(m2);
+    }
+    if (alive && !mbar_wait(bar_kv, ph)) { alive = false; atomicExch(a.status, kErrTimeout | 2); }
+    __syncthreads();
+    if (tid == 0) {
+      tc_fence_after();
+      for (int h = 0; h < kQH; ++h) {
+        const uint64_t dq = smem_desc_kmajor(smem_u32(sQ + h * kHalfQ), 128), dk = smem_desc_kmajor(smem_u32(sK + h * kHalfQ), 128);
+#pragma unroll
+        for (int k = 0; k < 4; ++k) mma_f16_ss(tmem + S_COL, dq + 2 * k, dk + 2 * k, idesc_qk, (h > 0) | (k > 0));
+      }
+      mma_commit(bar_s);
+    }
+    if (alive && !mbar_wait(bar_s, ph)) { alive = false; atomicExch(a.status, kErrTimeout | 3); }
+    tc_fence_after();
+
+    // ---- softmax stage: this thread owns query row 32*warp + lane
+    const int nv = min(128, a.N - j * 128);
+    uint32_t r[32];
+    float mx = -INFINITY;
+#pragma unroll 1
+    for (int c = 0; c < 4; ++c) {
+      tmem_ld32(lane_base + S_COL + 32 * c, r);
+      tmem_wait_ld();
+#pragma unroll
+      for (int i = 0; i < 32; ++i)
+        if (32 * c + i < nv) mx = fmaxf(mx, __uint_as_float(r[i]));
+    }
+    const float m_new = fmaxf(m_run, mx * cs);
+    const float alpha = exp2f(m_run - m_new);
+    float rsum = 0.f;
+#pragma unroll 1
+    for (int c = 0; c < 4; ++c) {
+      tmem_ld32(lane_base + S_COL + 32 * c, r);
+      tmem_wait_ld();
+      uint32_t pk[16];
+#pragma unroll
+      for (int g = 0; g < 2; ++g) {                   // NVFP4 group of 16 keys
+        float p[16], gmax = 0.f;
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+          const int key = 32 * c + 16 * g + i;
+          const float u = fmaf(__uint_as_float(r[16 * g + i]), cs, -m_new);
+          p[i] = key < nv ? exp2f(u) * 2688.0f : 0.f;   // the row maximum maps to 6 * 448
+          gmax = fmaxf(gmax, p[i]);
+        }
+        const uint32_t sb = __nv_cvt_float_to_fp8(gmax * (1.0f / 6.0f), __NV_SATFINITE, __NV_E4M3);
+        const __half_raw hs = __nv_cvt_fp8_to_halfraw((__nv_fp8_storage_t)sb, __NV_E4M3);
+        const float sdec = __half2float(__half(hs));
+        const float rcp = sdec > 0.f ? 1.0f / sdec : 0.f;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          const __nv_fp4x2_storage_t two = __nv_cvt_float2_to_fp4x2(make_float2(p[2 * i] * rcp, p[2 * i + 1] * rcp), __NV_E2M1, cudaRoundNearest);
+          const __half2_raw h2 = __nv_cvt_fp4x2_to_halfraw2(two, __NV_E2M1);
+          const float2 f = __half22float2(__half2(h2));
+          const float p0 = f.x * sdec, p1 = f.y * sdec;     // decoded probabilities, exact in bf16
+          rsum += p0 + p1;
+          __nv_bfloat162 b = __floats2bfloat162_rn(p0, p1);
+          pk[8 * g + i] = *reinterpret_cast<uint32_t*>(&b);
+        }
+      }
+      uint32_t lo[8], hi[8];
+#pragma unroll
+      for (int i = 0; i < 8; ++i) { lo[i] = pk[i]; hi[i] = pk[8 + i]; }
+      tmem_st8(lane_base + P_COL + 16 * c, lo);
+      tmem_st8(lane_base + P_COL + 16 * c + 8, hi);
+    }
+    l_run = alpha * l_run + rsum;
+    m_run = m_new;
+
+    // ---- A <- alpha A + r mu_j (means unscaled at 4 bits, App. B); the product follows
+#pragma unroll 1
+    for (int c = 0; c < D / 32; ++c) {
+      if (j > 0) { tmem_ld32(lane_base + O_COL + 32 * c, r); tmem_wait_ld(); }
+#pragma unroll
+      for (int i = 0; i < 32; ++i) {
+        const float prev = j > 0 ? __uint_as_float(r[i]) * alpha : 0.f;
+        r[i] = __float_as_uint(fmaf(rsum, sMu[32 * c + i], prev));
+      }
+      tmem_st32(lane_base + O_COL + 32 * c, r);
+    }
+    tmem_wait_st();
+    tc_fence_before();
+    __syncthreads();
+    if (tid == 0) {
+      tc_fence_after();
+      for (int h = 0; h < 2; ++h) {
+        const uint64_t dv = smem_desc_kmajor(smem_u32(sV + h * kHalfV), 128);
+#pragma unroll
+        for (int k = 0; k < 4; ++k) mma_f16_ts(tmem + O_COL, tmem + P_COL + 32 * h + 8 * k, dv + 2 * k, idesc_pv, 1);
+      }
+      mma_commit(bar_o);
+    }
+    if (alive && !mbar_wait(bar_o, ph)) { alive = false; atomicExch(a.status, kErrTimeout | 4); }
+    tc_fence_after();
+  }
+
+  // ---- epilogue: O = A / l
+  const int row = qblk * 128 + tid;
+  const float inv_l = 1.0f / l_run;
+  uint32_t r[32];
+#pragma unroll 1
+  for (int c = 0; c < D / 32; ++c) {
+    tmem_ld32(lane_base + O_COL + 32 * c, r);
+    tmem_wait_ld();
+    if (row < a.N) {
+      uint32_t out[16];
+#pragma unroll
+      for (int i = 0; i < 16; ++i) {
+        __nv_bfloat162 h2 = __floats2bfloat162_rn(__uint_as_float(r[2 * i]) * inv_l, __uint_as_float(r[2 * i + 1]) * inv_l);
+        out[i] = *reinterpret_cast<uint32_t*>(&h2);
+      }
+      uint4* dst = reinterpret_cast<uint4*>(a.o + ((size_t)bh * a.N + row) * D + 32 * c);
+#pragma unroll
+      for (int i = 0; i < 4; ++i) dst[i] = make_uint4(out[4 * i], out[4 * i + 1], out[4 * i + 2], out[4 * i + 3]);
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 0) tmem_dealloc<kTmemCols>(tmem);
+}
+
 // ---------------------------------------------------------------------------------------
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -669,13 +886,45 @@ cudaError_t run8(const Problem& pr, const QuantLayout& ql, const WorkLayout& wl,
   return cudaErrorNotSupported;
 }
 
+template <int D>
+cudaError_t run4(const Problem& pr, const QuantLayout& ql, const WorkLayout& wl, const uint8_t* quant,
+                 void* o, uint8_t* work, cudaStream_t s) {
+  // expand NVFP4 codes x microscales to bf16 tiles in the workspace
+  const size_t elems = (size_t)pr.BH * pr.n_pad * D, groups = elems / 16;
+  __nv_bfloat16* qb = reinterpret_cast<__nv_bfloat16*>(work + wl.expand);
+  __nv_bfloat16 *kb = qb + elems, *vb = kb + elems;
+  const unsigned blocks = (unsigned)((groups + 255) / 256);
+  nvfp4_expand_kernel<<<blocks, 256, 0, s>>>(quant + ql.q_codes, quant + ql.q_micro, qb, groups);
+  nvfp4_expand_kernel<<<blocks, 256, 0, s>>>(quant + ql.k_codes, quant + ql.k_micro, kb, groups);
+  nvfp4_expand_kernel<<<blocks, 256, 0, s>>>(quant + ql.v_codes, quant + ql.v_micro, vb, groups);
+  alignas(64) CUtensorMap tq, tk, tv;
+  if (!make_map(&tq, qb, (uint64_t)D * 2, pr.n_pad, pr.BH, 128, 128) ||
+      !make_map(&tk, kb, (uint64_t)D * 2, pr.n_pad, pr.BH, 128, 128) ||
+      !make_map(&tv, vb, (uint64_t)pr.n_pad * 2, D, pr.BH, 128, D))
+    return cudaErrorUnknown;
+  Attn4Args a{};
+  a.q_g = (const float*)(quant + ql.q_scale);
+  a.k_g = (const float*)(quant + ql.k_scale);
+  a.v_means = (const __nv_bfloat16*)(quant + ql.v_means);
+  a.o = (__nv_bfloat16*)o;
+  a.status = (uint32_t*)(work + wl.status);
+  a.N = pr.N; a.n_pad = pr.n_pad; a.nb = pr.nb;
+  a.sl = pr.softmax_scale * 1.4426950408889634f;
+  const size_t smem = 1024 + 2 * (D / 64) * 128 * 128 + 2 * D * 128 + D * 4 + 64;
+  cudaError_t e = cudaFuncSetAttribute(attn_fwd_serial4_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return e;
+  attn_fwd_serial4_kernel<D><<<dim3(pr.nb, pr.BH), 128, smem, s>>>(tq, tk, tv, a);
+  count_launches(4);
+  return cudaGetLastError();
+}
+
 }  // namespace
 
 cudaError_t launch_attn_fwd(const Problem& pr, const QuantLayout& ql, const WorkLayout& wl,
                             const uint8_t* quant, void* o, uint8_t* work, cudaStream_t stream) {
   cudaError_t e = cudaMemsetAsync(work + wl.status, 0, 4, stream);
   if (e != cudaSuccess) return e;
-  if (pr.bits != 8) return cudaErrorNotSupported;
+  if (pr.bits == 4) return pr.d == 128 ? run4<128>(pr, ql, wl, quant, o, work, stream) : run4<64>(pr, ql, wl, quant, o, work, stream);
   return pr.d == 128 ? run8<128>(pr, ql, wl, quant, o, work, stream) : run8<64>(pr, ql, wl, quant, o, work, stream);
 }
 

@@ -41,6 +41,7 @@ struct WorkLayout {
   size_t amax;       // uint32 [BH][d] residual amax bits (8-bit V) then [2][BH] Q/K head amax (4-bit)
   size_t amax_bytes;
   size_t mu_mma;     // fp32 [BH][nb][d][8]: block means as the B operand of the mean-restoration MMA
+  size_t expand;     // bf16 [3][BH][N_pad][d]: NVFP4 operands expanded for the 4-bit attention (0 bytes at 8 bits)
   size_t total;
   int rope_off[3];   // entry offset of each axis table
   int rope_entries;

@@ -28,11 +28,8 @@ def test_fullsize_sampled_parity(name, bits, perm_kind):
     p = Params.make(w.B, w.H, w.N, w.d, w.grid, bits=bits)
     quant, work = alloc_buffers(p)
     o = torch.empty(w.B, w.H, w.N, w.d, dtype=torch.bfloat16, device="cuda")
-    if bits == 8:
-        vc.vc_attn(p, q, k, v, perm, o, quant, work)
-        vc.vc_poll_status(work)
-    else:
-        vc.vc_prep(p, q, k, v, perm, quant, work)       # the 4-bit attention kernel is not built yet
+    vc.vc_attn(p, q, k, v, perm, o, quant, work)
+    vc.vc_poll_status(work)
     torch.cuda.synchronize()
     got = Hh.gpu_sections(p, quant)
     nb = (w.N + 127) // 128
@@ -41,8 +38,7 @@ def test_fullsize_sampled_parity(name, bits, perm_kind):
     for (b, h) in [(0, 0), (w.B - 1, w.H - 1)]:
         ref, cfg = Hh.oracle_prep(p, q, k, v, perm, b, h)
         stats = Hh.check_prep_head(p, got, b * w.H + h, ref, what=f"{name} b{b} h{h}")
-        if bits == 8:
-            o_ref = OA.emulate_head(ref, cfg, rows=rows)
-            vmax = float(v[b, h].float().abs().max())
-            m = Hh.check_output(o[b, h].float().cpu().numpy()[rows], o_ref, vmax)
-            print(name, bits, (b, h), stats, m)
+        o_ref = OA.emulate_head(ref, cfg, rows=rows)
+        vmax = float(v[b, h].float().abs().max())
+        m = Hh.check_output(o[b, h].float().cpu().numpy()[rows], o_ref, vmax)
+        print(name, bits, (b, h), stats, m)

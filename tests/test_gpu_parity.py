@@ -128,6 +128,26 @@ def test_vc_attn_end_to_end_config1(perm_kind):
         assert m0["max_err_over_vmax"] < m1["max_err_over_vmax"] + 1e-2, (m0, m1)
 
 
+@pytest.mark.parametrize("perm_kind", ["identity", "random"])
+@pytest.mark.parametrize("case", SMALL, ids=[c[0] for c in SMALL])
+def test_vc_attn_4bit_end_to_end(case, perm_kind):
+    """4-bit path (NVFP4 Q, K, residual and P): vc_attn against the oracle's emulation."""
+    _, B, H, N, d, grid = case
+    q, k, v = _inputs(B, H, N, d, grid, seed=31)
+    perm = None if perm_kind == "identity" else vc_inputs.random_perm(B, H, N, 8).cuda()
+    p = Params.make(B, H, N, d, grid, bits=4)
+    quant, work = alloc_buffers(p)
+    o = torch.empty(B, H, N, d, dtype=torch.bfloat16, device="cuda")
+    vc.vc_attn(p, q, k, v, perm, o, quant, work)
+    vc.vc_poll_status(work)
+    vmax = float(v.float().abs().max())
+    for b in range(B):
+        for h in range(H):
+            bundle, cfg = Hh.oracle_prep(p, q, k, v, perm, b, h)
+            ref = OA.emulate_head(bundle, cfg)
+            Hh.check_output(o[b, h].float().cpu().numpy(), ref, vmax)
+
+
 def test_bad_arguments_are_rejected_on_the_host():
     p = Params.make(1, 1, 128, 128, (2, 8, 8))
     quant, work = alloc_buffers(p)
