@@ -1,0 +1,99 @@
+"""Edge and degenerate cases of the CUDA path against the oracle: the shortest sequences,
+stage switches end to end, non-default softmax scale and ExpCast offset, and inputs that make
+a scale degenerate (all-zero V, constant K, constant V)."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2609_15810_b200 as vc
+import vc_inputs
+from paper_2609_15810_b200.binding import Params, alloc_buffers
+from oracle import attention as OA
+from oracle import compare as CMP
+
+import helpers as Hh
+
+pytestmark = pytest.mark.gpu
+
+
+def _run(p, q, k, v, perm, softmax_scale=None, beta=None, p_format=None):
+    quant, work = alloc_buffers(p)
+    o = torch.empty(p.B, p.H, p.N, p.d, dtype=torch.bfloat16, device="cuda")
+    vc.vc_attn(p, q, k, v, perm, o, quant, work)
+    vc.vc_poll_status(work)
+    vmax = max(float(v.float().abs().max()), 1e-6)
+    worst = None
+    for b in range(p.B):
+        for h in range(p.H):
+            bundle, cfg = Hh.oracle_prep(p, q, k, v, perm, b, h)
+            kw = {}
+            if softmax_scale is not None:
+                kw["softmax_scale"] = softmax_scale
+            if beta is not None:
+                kw["beta"] = beta
+            if p_format is not None:
+                kw["p_format"] = p_format
+            ref = OA.emulate_head(bundle, cfg, **kw)
+            got = o[b, h].float().cpu().numpy()
+            assert np.isfinite(got).all()
+            m = CMP.output_metrics(got, ref, vmax)
+            assert m["max_err_over_vmax"] <= 2e-2, m
+            if np.linalg.norm(ref) > 1e-6:
+                assert m["cos"] >= 0.999, m
+            worst = m
+    return worst
+
+
+@pytest.mark.parametrize("bits", [8, 4])
+@pytest.mark.parametrize("N,grid", [(1, (1, 1, 1)), (2, (1, 1, 2)), (17, (1, 1, 17)), (127, (1, 1, 127))])
+def test_shortest_sequences(N, grid, bits):
+    w = vc_inputs.Workload("t", 1, 2, N, 128, grid, (8,), 41, "gauss")
+    q, k, v = [t.cuda() for t in vc_inputs.make_qkv(w)]
+    _run(Params.make(1, 2, N, 128, grid, bits=bits), q, k, v, None)
+
+
+@pytest.mark.parametrize("flags", [0, vc.VC_FLAG_ROPE, vc.VC_FLAG_HADAMARD | vc.VC_FLAG_K_SMOOTH, vc.VC_FLAG_V_SMOOTH,
+                                   vc.VC_FLAG_ALL & ~vc.VC_FLAG_V_SMOOTH])
+def test_stage_switches_end_to_end(flags):
+    w = vc_inputs.Workload("t", 1, 2, 600, 128, (6, 10, 10), (8,), 42, "gauss")
+    q, k, v = [t.cuda() for t in vc_inputs.make_qkv(w)]
+    perm = vc_inputs.random_perm(1, 2, 600, 9).cuda()
+    _run(Params.make(1, 2, 600, 128, (6, 10, 10), bits=8, flags=flags), q, k, v, perm)
+
+
+def test_softmax_scale_beta_and_exp_then_cast():
+    w = vc_inputs.Workload("t", 1, 1, 512, 64, (8, 8, 8), (8,), 43, "gauss")
+    q, k, v = [t.cuda() for t in vc_inputs.make_qkv(w)]
+    _run(Params.make(1, 1, 512, 64, (8, 8, 8), bits=8, softmax_scale=0.05, beta=-0.2), q, k, v, None,
+         softmax_scale=0.05, beta=-0.2)
+    _run(Params.make(1, 1, 512, 64, (8, 8, 8), bits=8, p_format=vc.VC_P_EXP_E4M3, softmax_scale=0.2), q, k, v, None,
+         softmax_scale=0.2, p_format=OA.P_EXP_E4M3)
+
+
+@pytest.mark.parametrize("bits", [8, 4])
+def test_degenerate_scales(bits):
+    w = vc_inputs.Workload("t", 1, 1, 384, 128, (6, 8, 8), (8,), 44, "gauss")
+    q, k, v = [t.cuda() for t in vc_inputs.make_qkv(w)]
+    p = Params.make(1, 1, 384, 128, (6, 8, 8), bits=bits)
+    _run(p, q, k, torch.zeros_like(v), None)                                   # all-zero V: every scale degenerate
+    _run(p, q, k, torch.full_like(v, 1.5), None)                               # constant V: zero residual, mean only
+    pk = Params.make(1, 1, 384, 128, (6, 8, 8), bits=bits, flags=vc.VC_FLAG_ALL & ~vc.VC_FLAG_ROPE)
+    _run(pk, q, torch.full_like(k, 0.75), v, None)                             # constant K: centered keys vanish
+    _run(p, torch.zeros_like(q), k, v, None)                                   # zero Q: uniform attention
+
+
+def test_strided_inputs_through_vc_attn():
+    B, H, N, d, grid = 1, 3, 300, 128, (3, 10, 10)
+    w = vc_inputs.Workload("t", B, H, N, d, grid, (8,), 45, "gauss")
+    q, k, v = [t.cuda() for t in vc_inputs.make_qkv(w)]
+    qs, ks, vs = [t.permute(0, 2, 1, 3).contiguous() for t in (q, k, v)]       # [B, N, H, d] storage
+    ps = Params.make(B, H, N, d, grid, bits=8, stride_b=N * H * d, stride_h=d, stride_n=H * d)
+    p0 = Params.make(B, H, N, d, grid, bits=8)
+    outs = []
+    for p, (a, b, c) in ((ps, (qs, ks, vs)), (p0, (q, k, v))):
+        quant, work = alloc_buffers(p)
+        o = torch.empty(B, H, N, d, dtype=torch.bfloat16, device="cuda")
+        vc.vc_attn(p, a, b, c, None, o, quant, work)
+        vc.vc_poll_status(work)
+        outs.append(o)
+    assert torch.equal(outs[0], outs[1])
