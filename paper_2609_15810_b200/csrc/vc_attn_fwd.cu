@@ -423,9 +423,11 @@ attn_fwd_2q_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
     unsigned char* p_row = sP + t * kPBytes + (row >> 3) * 1024 + (row & 7) * 128;
     const float sq = qblk < nb ? a.q_scale[(size_t)bh * nb + qblk] : 1.0f;
     float m_run = -INFINITY;
+    float sk_next = __ldg(&a.k_scale[(size_t)bh * nb]);   // fetched one tile ahead: an L2 round trip
     for (int j = 0; j < nb; ++j) {
       const int ph = j & 1;
-      const float cs = (sq * __ldg(&a.k_scale[(size_t)bh * nb + j])) * a.sl;
+      const float cs = (sq * sk_next) * a.sl;             // code units -> log2 domain
+      if (j + 1 < nb) sk_next = __ldg(&a.k_scale[(size_t)bh * nb + j + 1]);
       if (!warp_wait2(&sh->s_full[t], ph, sh, a.status, 30)) break;
       tc_fence_after();
       uint32_t s0[32], s1[32], s2[32], s3[32];
