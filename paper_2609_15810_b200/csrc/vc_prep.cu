@@ -9,8 +9,8 @@
 //       gather -> residual -> codes written channel-major, block means beside them
 //
 // The two global reductions (K channel mean over all tokens, per-channel amax of the V
-// residual over all tokens) force a statistics launch before the quantizing launch; heads
-// are processed in groups so that the second read of K and V can hit L2.
+// residual over all tokens) force a statistics launch before the quantizing launches; heads
+// can be processed in groups so that the second read of K and V may hit L2.
 #include <cuda_bf16.h>
 #include <cuda_fp4.h>
 #include <cuda_fp8.h>
@@ -36,7 +36,7 @@ struct PrepArgs {
   const __nv_bfloat16 *q, *k, *v;
   const int32_t* perm;
   int64_t stride_b, stride_h, stride_n;
-  int H, N, n_pad, nb, bh0, flags, rope_in_smem;
+  int H, N, n_pad, nb, bh0, flags, rope_in_smem, rope_default;
   uint8_t *q_codes, *k_codes, *v_codes, *q_micro, *k_micro, *v_micro;
   float *q_scale, *k_scale, *v_scale, *k_mean;
   __nv_bfloat16* v_means;
@@ -289,6 +289,185 @@ __device__ __forceinline__ void qk_body(const PrepArgs& a, unsigned char* smem) 
 }
 
 // ---------------------------------------------------------------------------------------
+// Q / K body, one query/key row per thread (128 threads, one 128-row block per CTA).  All D
+// channels of a row sit in the registers of one thread, so the Hadamard rotation is D/2 * log2 D
+// register butterflies with no shuffle at all (a warp shuffle costs a full issue slot per 32
+// values, which made the lane-per-8-channels layout issue-bound), RoPE pairs and NVFP4 groups are
+// thread-local, and a row's codes leave as 16-byte stores.  Used for the amax and quantizing
+// stages; the column sums of K need the transposed ownership and keep the layout above.
+constexpr int kRowThreads = 128;
+
+template <int D> struct RopeSplit;          // pair boundaries of the default channel split
+template <> struct RopeSplit<128> { static constexpr int p1 = 22, p2 = 43; };   // 44 / 42 / 42
+template <> struct RopeSplit<64> { static constexpr int p1 = 12, p2 = 22; };    // 24 / 20 / 20
+
+template <int D, int TENSOR /*0 = Q, 1 = K*/, int STAGE>
+__device__ __forceinline__ void qk_row_body(const PrepArgs& a, unsigned char* smem) {
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int blk = blockIdx.x, bh = a.bh0 + blockIdx.y;
+  const int b = bh / a.H, h = bh - b * a.H;
+  const __nv_bfloat16* base = (TENSOR == 0 ? a.q : a.k) + b * a.stride_b + h * a.stride_h;
+  const bool do_rope = a.flags & VC_FLAG_ROPE;
+  const bool do_had = a.flags & VC_FLAG_HADAMARD;
+  const bool gather = TENSOR == 1 && a.perm != nullptr && STAGE >= kStageQuant8;
+  float* red = reinterpret_cast<float*>(smem);                   // [4] warp maxima
+  float* kmean_s = reinterpret_cast<float*>(smem + 64);          // [D]
+  float2* tab_s = reinterpret_cast<float2*>(smem + 64 + D * 4);
+
+  const int t = blk * kBlock + tid;
+  const bool valid = t < a.N;
+  int src = valid ? t : 0;
+  if (gather && valid) src = __ldg(&a.perm[(size_t)bh * a.N + t]);
+  uint4 raw[D / 8];
+#pragma unroll
+  for (int i = 0; i < D / 8; ++i) {
+    raw[i] = make_uint4(0, 0, 0, 0);
+    if (valid) raw[i] = __ldg(reinterpret_cast<const uint4*>(base + (int64_t)src * a.stride_n + 8 * i));
+  }
+  // tables -> shared memory while the row is in flight
+  const float2* tab = a.rope;
+  if (do_rope && a.rope_in_smem) {
+    for (int e = tid; e < a.rd.entries; e += kRowThreads) tab_s[e] = __ldg(&a.rope[e]);
+    tab = tab_s;
+  }
+  const bool center = TENSOR == 1 && (a.flags & VC_FLAG_K_SMOOTH);
+  if (center) {
+    for (int c = tid; c < D; c += kRowThreads) kmean_s[c] = a.k_mean[(size_t)bh * D + c];
+  }
+  __syncthreads();
+
+  float x[D];
+#pragma unroll
+  for (int i = 0; i < D / 8; ++i) {
+    const unsigned int w[4] = {raw[i].x, raw[i].y, raw[i].z, raw[i].w};
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      x[8 * i + 2 * j] = __uint_as_float(w[j] << 16);
+      x[8 * i + 2 * j + 1] = __uint_as_float(w[j] & 0xffff0000u);
+    }
+  }
+  if (do_rope && valid) {
+    const unsigned int q1 = div40((unsigned)src, a.rd.mul_w);
+    const int tx = src - q1 * a.rd.grid_w;
+    const int tt = div40(q1, a.rd.mul_h);
+    const int ty = q1 - tt * a.rd.grid_h;
+    // entry of pair p of axis ax: off[ax] + pos[ax] * pairs[ax] + (p - pair_start[ax])
+    const int e0 = a.rd.off[0] + tt * a.rd.pairs[0] - a.rd.pair_start[0];
+    const int e1 = a.rd.off[1] + ty * a.rd.pairs[1] - a.rd.pair_start[1];
+    const int e2 = a.rd.off[2] + tx * a.rd.pairs[2] - a.rd.pair_start[2];
+    if (a.rope_default) {                       // compile-time pair boundaries: one load per pair
+#pragma unroll
+      for (int p = 0; p < D / 2; ++p) {
+        const int e = p < RopeSplit<D>::p1 ? e0 : (p < RopeSplit<D>::p2 ? e1 : e2);
+        const float2 cs = tab[e + p];
+        const float x0 = x[2 * p], x1 = x[2 * p + 1];
+        x[2 * p] = x0 * cs.x - x1 * cs.y;
+        x[2 * p + 1] = x0 * cs.y + x1 * cs.x;
+      }
+    } else {
+#pragma unroll
+      for (int p = 0; p < D / 2; ++p) {
+        const int e = p < a.rd.pair_start[1] ? e0 : (p < a.rd.pair_start[2] ? e1 : e2);
+        const float2 cs = tab[e + p];
+        const float x0 = x[2 * p], x1 = x[2 * p + 1];
+        x[2 * p] = x0 * cs.x - x1 * cs.y;
+        x[2 * p + 1] = x0 * cs.y + x1 * cs.x;
+      }
+    }
+  }
+  if (center && valid) {
+#pragma unroll
+    for (int c4 = 0; c4 < D / 4; ++c4) {
+      const float4 m = reinterpret_cast<const float4*>(kmean_s)[c4];
+      x[4 * c4] -= m.x; x[4 * c4 + 1] -= m.y; x[4 * c4 + 2] -= m.z; x[4 * c4 + 3] -= m.w;
+    }
+  }
+  if (do_had) {
+#pragma unroll
+    for (int sft = 1; sft < D; sft <<= 1) {
+#pragma unroll
+      for (int c = 0; c < D; ++c) {
+        if (!(c & sft)) {
+          const float u = x[c], v = x[c | sft];
+          x[c] = u + v;
+          x[c | sft] = u - v;
+        }
+      }
+    }
+  }
+  const float rs = do_had ? (D == 128 ? 0.08838834764831845f : 0.125f) : 1.0f;   // 1/sqrt(D)
+
+  float amax = 0.f;
+  if constexpr (STAGE != kStageQuant4) {
+#pragma unroll
+    for (int c = 0; c < D; ++c) amax = fmaxf(amax, fabsf(x[c]));
+    amax = warp_max(amax * rs);                 // max and the (positive) scale commute exactly
+    if (lane == 0) red[warp] = amax;
+    __syncthreads();
+    amax = fmaxf(fmaxf(red[0], red[1]), fmaxf(red[2], red[3]));
+  }
+  if constexpr (STAGE == kStageAmax) {
+    if (tid == 0) atomicMax(&a.qk_amax[TENSOR * a.BH + bh], __float_as_uint(amax));
+    return;
+  }
+  const size_t row_g = (size_t)bh * a.n_pad + (size_t)blk * kBlock + tid;
+
+  if constexpr (STAGE == kStageQuant8) {
+    const float inv = amax > 0.f ? 448.0f / amax : 0.f;
+    if (tid == 0) (TENSOR == 0 ? a.q_scale : a.k_scale)[(size_t)bh * a.nb + blk] = amax > 0.f ? amax / 448.0f : 1.0f;
+    uint4* dst = reinterpret_cast<uint4*>((TENSOR == 0 ? a.q_codes : a.k_codes) + row_g * D);
+#pragma unroll
+    for (int i = 0; i < D / 16; ++i) {
+      unsigned int w[4];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const int c = 16 * i + 4 * j;
+        const unsigned int lo = __nv_cvt_float2_to_fp8x2(make_float2((x[c] * rs) * inv, (x[c + 1] * rs) * inv), __NV_SATFINITE, __NV_E4M3);
+        const unsigned int hi = __nv_cvt_float2_to_fp8x2(make_float2((x[c + 2] * rs) * inv, (x[c + 3] * rs) * inv), __NV_SATFINITE, __NV_E4M3);
+        w[j] = lo | (hi << 16);
+      }
+      dst[i] = make_uint4(w[0], w[1], w[2], w[3]);
+    }
+  }
+
+  if constexpr (STAGE == kStageQuant4) {
+    // NVFP4: outer scale g per (b, h), microscale per token per 16 channels
+    const float g = (TENSOR == 0 ? a.q_scale : a.k_scale)[bh];
+    const float inv6 = 1.0f / (6.0f * g);
+    unsigned int codes[D / 8], micro[D / 64];
+#pragma unroll
+    for (int i = 0; i < D / 64; ++i) micro[i] = 0;
+#pragma unroll
+    for (int gq = 0; gq < D / 16; ++gq) {
+      float m = 0.f;
+#pragma unroll
+      for (int c = 0; c < 16; ++c) { x[16 * gq + c] *= rs; m = fmaxf(m, fabsf(x[16 * gq + c])); }
+      const unsigned int sb = __nv_cvt_float_to_fp8(m * inv6, __NV_SATFINITE, __NV_E4M3);
+      const float sdec = e4m3_to_float(sb);
+      const float rcp = sdec > 0.f ? 1.0f / (g * sdec) : 0.f;
+      micro[gq / 4] |= sb << (8 * (gq & 3));
+#pragma unroll
+      for (int wi = 0; wi < 2; ++wi) {
+        unsigned int word = 0;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const int c = 16 * gq + 8 * wi + 2 * j;
+          const unsigned int two = __nv_cvt_float2_to_fp4x2(make_float2(x[c] * rcp, x[c + 1] * rcp), __NV_E2M1, cudaRoundNearest);
+          word |= (two & 0xffu) << (8 * j);
+        }
+        codes[2 * gq + wi] = sdec > 0.f ? word : 0u;
+      }
+    }
+    uint4* dst = reinterpret_cast<uint4*>((TENSOR == 0 ? a.q_codes : a.k_codes) + row_g * (D / 2));
+#pragma unroll
+    for (int i = 0; i < D / 32; ++i) dst[i] = make_uint4(codes[4 * i], codes[4 * i + 1], codes[4 * i + 2], codes[4 * i + 3]);
+    unsigned int* mdst = reinterpret_cast<unsigned int*>((TENSOR == 0 ? a.q_micro : a.k_micro) + row_g * (D / 16));
+#pragma unroll
+    for (int i = 0; i < D / 64; ++i) mdst[i] = micro[i];
+  }
+}
+
+// ---------------------------------------------------------------------------------------
 // V body.  The gathered 128 x D block is staged in shared memory with coalesced 16-byte
 // loads; a thread then owns one channel pair and 128 / (256 / (D/2)) consecutive tokens,
 // so block means and the channel-major (token-contiguous) code rows need no transposition.
@@ -463,17 +642,14 @@ __device__ __forceinline__ void v_body(const PrepArgs& a, unsigned char* smem) {
 }
 
 // ---------------------------------------------------------------------------------------
-// Launch 1: statistics.  z = 0: K column sums; z = 1: V block means + residual amax;
-// z = 2 (4-bit): head amax of the rotated Q.
-template <int D, int BITS>
+// Launch 1: statistics.  z = 0: K column sums; z = 1: V block means + residual amax.
+template <int D>
 __global__ void __launch_bounds__(kThreads, 2) prep_stats_kernel(const PrepArgs a) {
   extern __shared__ __align__(16) unsigned char smem[];
   if (blockIdx.z == 0) {
     if (a.flags & VC_FLAG_K_SMOOTH) qk_body<D, 1, kStageColSum>(a, smem);
-  } else if (blockIdx.z == 1) {
-    v_body<D, kVStats>(a, smem);
   } else {
-    if constexpr (BITS == 4) qk_body<D, 0, kStageAmax>(a, smem);
+    v_body<D, kVStats>(a, smem);
   }
 }
 
@@ -504,37 +680,50 @@ __global__ void prep_finalize_kernel(const PrepArgs a, int which) {
   }
 }
 
-// Launch 3 (4-bit only): head amax of the centered, rotated K.
-template <int D>
-__global__ void __launch_bounds__(kThreads) prep_kamax_kernel(const PrepArgs a) {
+// 4-bit only: head amax of the rotated Q (tensor 0) or of the centered, rotated K (tensor 1).
+template <int D, int TENSOR>
+__global__ void __launch_bounds__(kRowThreads, 2) prep_amax_kernel(const PrepArgs a) {
   extern __shared__ __align__(16) unsigned char smem[];
-  qk_body<D, 1, kStageAmax>(a, smem);
+  qk_row_body<D, TENSOR, kStageAmax>(a, smem);
 }
 
-// Launch 4: quantization.  z = 0: Q; z = 1: K; z = 2: V.
+// Launch 3: quantization of Q (z = 0) and K (z = 1), one row per thread.
 template <int D, int BITS>
-__global__ void __launch_bounds__(kThreads, 2) prep_quant_kernel(const PrepArgs a) {
+__global__ void __launch_bounds__(kRowThreads, 3) prep_quant_qk_kernel(const PrepArgs a) {
   extern __shared__ __align__(16) unsigned char smem[];
   if (blockIdx.z == 0) {
-    qk_body<D, 0, BITS == 8 ? kStageQuant8 : kStageQuant4>(a, smem);
-  } else if (blockIdx.z == 1) {
-    qk_body<D, 1, BITS == 8 ? kStageQuant8 : kStageQuant4>(a, smem);
+    qk_row_body<D, 0, BITS == 8 ? kStageQuant8 : kStageQuant4>(a, smem);
   } else {
-    v_body<D, BITS == 8 ? kVQuant8 : kVQuant4>(a, smem);
+    qk_row_body<D, 1, BITS == 8 ? kStageQuant8 : kStageQuant4>(a, smem);
   }
+}
+
+// Launch 4: quantization of the V residual.
+template <int D, int BITS>
+__global__ void __launch_bounds__(kThreads, 2) prep_quant_v_kernel(const PrepArgs a) {
+  extern __shared__ __align__(16) unsigned char smem[];
+  v_body<D, BITS == 8 ? kVQuant8 : kVQuant4>(a, smem);
+}
+
+template <typename K>
+cudaError_t allow_smem(K kernel, size_t bytes) {
+  return bytes > 48 * 1024 ? cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) : cudaSuccess;
 }
 
 template <int D, int BITS>
 cudaError_t run(const Problem& pr, PrepArgs a, const WorkLayout& wl, uint8_t* work, cudaStream_t s) {
-  const size_t rope_bytes = (size_t)a.rd.entries * 8;
-  const size_t qk_smem = 8 * D * 4 + ((a.flags & VC_FLAG_ROPE) && a.rope_in_smem ? rope_bytes : 0);
+  const size_t rope_bytes = ((a.flags & VC_FLAG_ROPE) && a.rope_in_smem) ? (size_t)a.rd.entries * 8 : 0;
+  const size_t lane_smem = 8 * D * 4 + rope_bytes;                      // qk_body (column sums)
   const size_t v_smem = (size_t)kBlock * D * 2 + (kThreads / (D / 2)) * D * 4;
-  const size_t smem = qk_smem > v_smem ? qk_smem : v_smem;
+  const size_t stats_smem = lane_smem > v_smem ? lane_smem : v_smem;
+  const size_t row_smem = 64 + D * 4 + rope_bytes;                      // qk_row_body
   cudaError_t e;
-  if (smem > 48 * 1024) {
-    if ((e = cudaFuncSetAttribute(prep_stats_kernel<D, BITS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
-    if ((e = cudaFuncSetAttribute(prep_quant_kernel<D, BITS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
-    if ((e = cudaFuncSetAttribute(prep_kamax_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
+  if ((e = allow_smem(prep_stats_kernel<D>, stats_smem)) != cudaSuccess) return e;
+  if ((e = allow_smem(prep_quant_qk_kernel<D, BITS>, row_smem)) != cudaSuccess) return e;
+  if ((e = allow_smem(prep_quant_v_kernel<D, BITS>, v_smem)) != cudaSuccess) return e;
+  if (BITS == 4) {
+    if ((e = allow_smem(prep_amax_kernel<D, 0>, row_smem)) != cudaSuccess) return e;
+    if ((e = allow_smem(prep_amax_kernel<D, 1>, row_smem)) != cudaSuccess) return e;
   }
   if ((e = cudaMemsetAsync(work + wl.status, 0, 4, s)) != cudaSuccess) return e;
   if ((e = cudaMemsetAsync(work + wl.amax, 0, wl.amax_bytes, s)) != cudaSuccess) return e;
@@ -548,16 +737,18 @@ cudaError_t run(const Problem& pr, PrepArgs a, const WorkLayout& wl, uint8_t* wo
   for (int bh0 = 0; bh0 < pr.BH; bh0 += group) {
     const int nh = pr.BH - bh0 < group ? pr.BH - bh0 : group;
     a.bh0 = bh0;
-    prep_stats_kernel<D, BITS><<<dim3(pr.nb, nh, BITS == 4 ? 3 : 2), kThreads, smem, s>>>(a);
+    prep_stats_kernel<D><<<dim3(pr.nb, nh, 2), kThreads, stats_smem, s>>>(a);
+    if (BITS == 4) { prep_amax_kernel<D, 0><<<dim3(pr.nb, nh), kRowThreads, row_smem, s>>>(a); count_launches(1); }
     prep_finalize_kernel<D, BITS><<<nh, D, 0, s>>>(a, 0);
     count_launches(2);
     if (BITS == 4) {
-      prep_kamax_kernel<D><<<dim3(pr.nb, nh, 1), kThreads, smem, s>>>(a);
+      prep_amax_kernel<D, 1><<<dim3(pr.nb, nh), kRowThreads, row_smem, s>>>(a);
       prep_finalize_kernel<D, BITS><<<nh, 32, 0, s>>>(a, 1);
       count_launches(2);
     }
-    prep_quant_kernel<D, BITS><<<dim3(pr.nb, nh, 3), kThreads, smem, s>>>(a);
-    count_launches(1);
+    prep_quant_qk_kernel<D, BITS><<<dim3(pr.nb, nh, 2), kRowThreads, row_smem, s>>>(a);
+    prep_quant_v_kernel<D, BITS><<<dim3(pr.nb, nh), kThreads, v_smem, s>>>(a);
+    count_launches(2);
   }
   return cudaGetLastError();
 }
@@ -595,6 +786,10 @@ cudaError_t launch_prep(const Problem& pr, const QuantLayout& ql, const WorkLayo
   a.rd.mul_w = ((1ull << 40) + pr.grid_w - 1) / pr.grid_w;
   a.rd.mul_h = ((1ull << 40) + pr.grid_h - 1) / pr.grid_h;
   a.rope_in_smem = (size_t)wl.rope_entries * 8 <= 96 * 1024;
+  {
+    const int sdef = 2 * (pr.d / 6);
+    a.rope_default = pr.rope_dim[0] == pr.d - 2 * sdef && pr.rope_dim[1] == sdef && pr.rope_dim[2] == sdef;
+  }
   if (pr.d == 128) return pr.bits == 8 ? run<128, 8>(pr, a, wl, work, stream) : run<128, 4>(pr, a, wl, work, stream);
   return pr.bits == 8 ? run<64, 8>(pr, a, wl, work, stream) : run<64, 4>(pr, a, wl, work, stream);
 }
