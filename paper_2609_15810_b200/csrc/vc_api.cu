@@ -110,7 +110,9 @@ WorkLayout work_layout(const Problem& pr) {
   W.amax_bytes = BH * d * 4 + 2 * BH * 4;
   W.amax = place(W.amax_bytes);
   W.mu_mma = place(BH * nb * d * 32);
-  W.expand = place(pr.bits == 4 ? 3 * BH * (size_t)pr.n_pad * d * 2 : 0);
+  W.sf_q = place(pr.bits == 4 ? BH * nb * (d / 64) * 512 : 0);
+  W.sf_kv = place(pr.bits == 4 ? BH * nb * (d / 64 + 2) * 512 : 0);
+  W.expand = place(pr.bits == 4 && pr.kernel_variant == 1 ? 3 * BH * (size_t)pr.n_pad * d * 2 : 0);
   W.total = off;
   return W;
 }

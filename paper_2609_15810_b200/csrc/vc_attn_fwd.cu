@@ -16,13 +16,13 @@
 
 #include "vc_internal.h"
 #include "vc_sm100.cuh"
+#include "vc_attn_shared.cuh"
 
 namespace vc {
 namespace {
 
 using namespace sm100;
-
-constexpr uint32_t kErrTimeout = 0x100;
+using namespace attn;
 
 struct AttnArgs {
   const float *q_scale, *k_scale, *v_scale;
@@ -242,34 +242,6 @@ attn_fwd_serial_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
 //                 row maximum moved, hands (r_hi, r_lo) alpha_j to the mean MMA, writes the output
 //
 // Tensor memory: S (128 columns) | A_0 (d + 16) | A_1 (d + 16).
-constexpr int kStages2 = 4;
-constexpr uint32_t kWaitLimit2 = 1u << 18;   // x up to 4 us per try: about one second
-
-struct FaSmem {
-  uint64_t q_full, kv_full[kStages2], kv_empty[kStages2];
-  uint64_t s_full[2], s_free[2], o_done[2], fin_full[2], o_final[2];
-  // alpha and codes+correction hand-offs can run one key tile ahead of their consumer, so they
-  // alternate between two barriers (a parity wait aliases after two phases)
-  uint64_t a_full[2][2], pc_full[2][2];
-  float alpha[2][128];
-  uint32_t tmem_base;
-  volatile int abort;
-};
-
-__device__ __forceinline__ bool wait2(uint64_t* bar, uint32_t parity, FaSmem* sh, uint32_t* status, uint32_t code) {
-  if (mbar_try_wait(bar, parity)) return true;
-  for (uint32_t i = 0; i < kWaitLimit2; ++i) {
-    if (mbar_try_wait_hint(bar, parity, 4000u)) return true;
-    if ((i & 63u) == 63u && sh->abort) return false;
-  }
-  sh->abort = 1;
-  atomicExch(status, kErrTimeout | code);
-  return false;
-}
-__device__ __forceinline__ bool warp_wait2(uint64_t* bar, uint32_t parity, FaSmem* sh, uint32_t* status, uint32_t code) {
-  return __all_sync(0xffffffffu, wait2(bar, parity, sh, status, code));
-}
-
 template <int D, bool EXPCAST>
 __global__ void __launch_bounds__(640, 1)
 attn_fwd_2q_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
@@ -582,19 +554,6 @@ attn_fwd_2q_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
   if (warp == 2) tmem_dealloc<kTmemCols>(tmem);
 }
 
-// Block means as the B operand of the per-tile mean-restoration MMA: per (b, h, key tile) a
-// [d][8] fp32 tile with entry [c][0] = [c][1] = mu~[c] (for r_hi and r_lo) and zeros elsewhere.
-template <int D>
-__global__ void means_tile_layout_kernel(const __nv_bfloat16* __restrict__ means, float* __restrict__ out, size_t n) {
-  const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;   // (bh * nb + tile) * D + c
-  if (i >= n) return;
-  const float v = __bfloat162float(means[i]);
-  float4* dst = reinterpret_cast<float4*>(out + i * 8);
-  dst[0] = make_float4(v, v, 0.f, 0.f);
-  dst[1] = make_float4(0.f, 0.f, 0.f, 0.f);
-}
-
-
 // ---------------------------------------------------------------------------------------
 // 4-bit path (NVFP4 Q, K, R and P; App. A "Scope of ExpCast-FP8", App. B).
 //
@@ -811,36 +770,6 @@ attn_fwd_serial4_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
 }
 
 // ---------------------------------------------------------------------------------------
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiledFn encode_fn() {
-  static EncodeTiledFn fn = nullptr;   // resolved once; the driver entry point never changes
-  if (!fn) {
-    void* p = nullptr;
-    cudaDriverEntryPointQueryResult qres;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
-        qres == cudaDriverEntryPointSuccess)
-      fn = reinterpret_cast<EncodeTiledFn>(p);
-  }
-  return fn;
-}
-
-// 3-D byte tensor [dim2][dim1][dim0], box {box0, box1, 1}, swizzle chosen by the box width.
-bool make_map(CUtensorMap* m, const void* base, uint64_t dim0, uint64_t dim1, uint64_t dim2, uint32_t box0, uint32_t box1) {
-  EncodeTiledFn fn = encode_fn();
-  if (!fn) return false;
-  const cuuint64_t dims[3] = {dim0, dim1, dim2};
-  const cuuint64_t strides[2] = {dim0, dim0 * dim1};
-  const cuuint32_t box[3] = {box0, box1, 1};
-  const cuuint32_t estr[3] = {1, 1, 1};
-  const CUtensorMapSwizzle sw = box0 == 128 ? CU_TENSOR_MAP_SWIZZLE_128B : (box0 == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B);
-  return fn(m, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, const_cast<void*>(base), dims, strides, box, estr,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, sw, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
 template <int D>
 cudaError_t run8(const Problem& pr, const QuantLayout& ql, const WorkLayout& wl, const uint8_t* quant,
                  void* o, uint8_t* work, cudaStream_t s) {
@@ -926,6 +855,7 @@ cudaError_t launch_attn_fwd(const Problem& pr, const QuantLayout& ql, const Work
                             const uint8_t* quant, void* o, uint8_t* work, cudaStream_t stream) {
   cudaError_t e = cudaMemsetAsync(work + wl.status, 0, 4, stream);
   if (e != cudaSuccess) return e;
+  if (pr.bits == 4 && pr.kernel_variant == 0) return launch_attn_fwd4(pr, ql, wl, quant, o, work, stream);
   if (pr.bits == 4) return pr.d == 128 ? run4<128>(pr, ql, wl, quant, o, work, stream) : run4<64>(pr, ql, wl, quant, o, work, stream);
   return pr.d == 128 ? run8<128>(pr, ql, wl, quant, o, work, stream) : run8<64>(pr, ql, wl, quant, o, work, stream);
 }

@@ -41,7 +41,9 @@ struct WorkLayout {
   size_t amax;       // uint32 [BH][d] residual amax bits (8-bit V) then [2][BH] Q/K head amax (4-bit)
   size_t amax_bytes;
   size_t mu_mma;     // fp32 [BH][nb][d][8]: block means as the B operand of the mean-restoration MMA
-  size_t expand;     // bf16 [3][BH][N_pad][d]: NVFP4 operands expanded for the 4-bit attention (0 bytes at 8 bits)
+  size_t sf_q;       // bytes [BH][nb][d/64][512]: Q^ NVFP4 factors in MMA chunk order (4 bits)
+  size_t sf_kv;      // bytes [BH][nb][d/64 + 2][512]: K^ and R^ factors per key tile (4 bits)
+  size_t expand;     // bf16 [3][BH][N_pad][d]: NVFP4 operands expanded to bf16, serial 4-bit kernel only
   size_t total;
   int rope_off[3];   // entry offset of each axis table
   int rope_entries;
@@ -57,6 +59,9 @@ cudaError_t launch_prep(const Problem& pr, const QuantLayout& ql, const WorkLayo
                         uint8_t* quant, uint8_t* work, cudaStream_t stream);
 cudaError_t launch_attn_fwd(const Problem& pr, const QuantLayout& ql, const WorkLayout& wl,
                             const uint8_t* quant, void* o, uint8_t* work, cudaStream_t stream);
+
+cudaError_t launch_attn_fwd4(const Problem& pr, const QuantLayout& ql, const WorkLayout& wl,
+                             const uint8_t* quant, void* o, uint8_t* work, cudaStream_t stream);
 
 void count_launches(int n);
 
