@@ -2,25 +2,28 @@
 // App. B): every operand is read as bf16 with 16-byte vector loads and leaves as low-bit
 // codes plus scales; no rotated / permuted / centered high-precision tensor reaches HBM.
 //
-//   Q : RoPE -> Hadamard (registers + warp shuffles) -> per-128-row scale -> codes
+//   Q : RoPE -> Hadamard (in registers, one row per thread) -> per-128-row scale -> codes
 //   K : RoPE -> column sums (stats launch) ... gather by pi -> RoPE at the source position
 //       -> subtract channel mean -> Hadamard -> scale -> codes
 //   V : gather by pi -> block mean (Eq. 4) and residual amax (stats launch) ...
 //       gather -> residual -> codes written channel-major, block means beside them
 //
 // The two global reductions (K channel mean over all tokens, per-channel amax of the V
-// residual over all tokens) force a statistics launch before the quantizing launches; heads
-// can be processed in groups so that the second read of K and V may hit L2.
+// residual over all tokens) force statistics launches before the quantizing launches; heads
+// can be processed in groups so that the second read of K and V may hit L2.  All passes are
+// persistent kernels that prefetch the next row blocks with cp.async while they transform
+// the current one.
 #include <cuda_bf16.h>
 #include <cuda_fp4.h>
 #include <cuda_fp8.h>
 
 #include "vc_internal.h"
+#include "vc_sm100.cuh"
 
 namespace vc {
 namespace {
 
-constexpr int kThreads = 256;
+using namespace sm100;
 
 struct RopeDesc {
   int pair_start[3];   // first channel pair of each axis
@@ -78,263 +81,151 @@ __global__ void rope_table_kernel(float2* tab, RopeDesc rd, double theta) {
 }
 
 // ---------------------------------------------------------------------------------------
-// Q / K body.  A CTA owns one block of 128 rows; a lane owns 8 consecutive channels of
-// D/16 consecutive rows, so RoPE pairs and 3 Hadamard stages stay in registers and the
-// remaining log2(D/8) stages are xor-shuffles inside the D/8 lanes that share a row.
-enum { kStageColSum = 0, kStageAmax = 1, kStageQuant8 = 2, kStageQuant4 = 3 };
+// Persistent, pipelined passes.  Every pass is a loop over work items (tensor, head, block of
+// 128 rows); a CTA takes items blockIdx.x, blockIdx.x + gridDim.x, ...  The 16-byte chunks of
+// the NEXT items are already on their way into a ring of shared-memory stages (cp.async, no
+// registers held for bytes in flight) while the current item is transformed, so the load
+// latency of a block hides behind the arithmetic of the blocks before it.  For Q and K a
+// thread fetches exactly the chunks it will read itself, so those passes need no barrier for
+// the data at all; V is staged as a tile because its codes leave channel-major.
+// (One bulk-async copy per gathered row was tried instead of cp.async: 128 small copies per
+// block kept the copy engine, not HBM, busy.)
+constexpr int kThreads = 256;      // threads of the column-sum and V passes
+constexpr int kRowThreads = 128;   // threads of the row-per-thread Q/K pass
 
-template <int D, int TENSOR /*0 = Q, 1 = K*/, int STAGE>
-__device__ __forceinline__ void qk_body(const PrepArgs& a, unsigned char* smem) {
+template <int D> struct Geo {
+  static constexpr int pitch = 2 * D + 16;          // row pitch of the thread-per-row layout
+  static constexpr int stage_bytes = kBlock * pitch;
+};
+
+__device__ __forceinline__ void cp_async16(void* dst, const void* src) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_u32(dst)), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
+struct Item {
+  int z, bh, blk;
+};
+// items are numbered block-fastest, then head, then tensor
+__device__ __forceinline__ Item decode_item(int item, int nb, int nh, int bh0) {
+  Item it;
+  it.blk = item % nb;
+  const int r = item / nb;
+  it.bh = bh0 + r % nh;
+  it.z = r / nh;
+  return it;
+}
+
+// Token position -> (t, y, x) of the grid.
+__device__ __forceinline__ void grid_pos(const RopeDesc& rd, int src, int& tt, int& ty, int& tx) {
+  const unsigned int q1 = div40((unsigned)src, rd.mul_w);
+  tx = src - q1 * rd.grid_w;
+  tt = div40(q1, rd.mul_h);
+  ty = q1 - tt * rd.grid_h;
+}
+
+// ---------------------------------------------------------------------------------------
+// K column sums after RoPE (the channel mean of Sec. 3.4 is taken after the rotation).  A lane
+// owns 8 consecutive channels of D/16 rows, so a column's partial sums meet by xor-shuffles.
+template <int D>
+__device__ __forceinline__ void k_colsum_item(const PrepArgs& a, const unsigned char* stage, float* red, const float2* tab,
+                                              int bh, int blk) {
   constexpr int LPR = D / 8;         // lanes per row
   constexpr int RPL = LPR / 2;       // rows per lane (a warp covers 16 rows)
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int lr = lane % LPR, hb = lane / LPR;
-  const int blk = blockIdx.x, bh = a.bh0 + blockIdx.y;
-  const int b = bh / a.H, h = bh - b * a.H;
-  const __nv_bfloat16* base = (TENSOR == 0 ? a.q : a.k) + b * a.stride_b + h * a.stride_h;
   const bool do_rope = a.flags & VC_FLAG_ROPE;
-  const bool do_had = (a.flags & VC_FLAG_HADAMARD) && STAGE != kStageColSum;
-  const bool gather = TENSOR == 1 && a.perm != nullptr && STAGE >= kStageQuant8;
-
-  float* red = reinterpret_cast<float*>(smem);            // [8][D] floats of scratch
-  // per-lane constants of the 4 channel pairs it owns
   int p_axis[4], p_idx[4];
 #pragma unroll
   for (int j = 0; j < 4; ++j) {
-    int p = 4 * lr + j;
-    int ax = p >= a.rd.pair_start[2] ? 2 : (p >= a.rd.pair_start[1] ? 1 : 0);
+    const int p = 4 * lr + j;
+    const int ax = p >= a.rd.pair_start[2] ? 2 : (p >= a.rd.pair_start[1] ? 1 : 0);
     p_axis[j] = ax;
     p_idx[j] = a.rd.off[ax] + (p - a.rd.pair_start[ax]);
   }
-  float kmean[8];
+  float s[8];
 #pragma unroll
-  for (int c = 0; c < 8; ++c) kmean[c] = 0.f;
-  if (TENSOR == 1 && STAGE != kStageColSum && (a.flags & VC_FLAG_K_SMOOTH)) {
-#pragma unroll
-    for (int c = 0; c < 8; ++c) kmean[c] = a.k_mean[(size_t)bh * D + 8 * lr + c];
-  }
-
-  // all row loads of the thread are issued before any arithmetic: bytes in flight, not
-  // instruction count, set the speed of this pass
-  int srcs[RPL];
+  for (int c = 0; c < 8; ++c) s[c] = 0.f;
 #pragma unroll
   for (int i = 0; i < RPL; ++i) {
-    const int t = blk * kBlock + 16 * warp + RPL * hb + i;
-    srcs[i] = t < a.N ? t : -1;
-    if (gather && t < a.N) srcs[i] = __ldg(&a.perm[(size_t)bh * a.N + t]);
-  }
-  uint4 raws[RPL];
-#pragma unroll
-  for (int i = 0; i < RPL; ++i) {
-    raws[i] = make_uint4(0, 0, 0, 0);
-    if (srcs[i] >= 0) raws[i] = __ldg(reinterpret_cast<const uint4*>(base + (int64_t)srcs[i] * a.stride_n + 8 * lr));
-  }
-  // RoPE table -> shared memory while the rows are in flight (read through L2 if it does not fit)
-  const float2* tab = a.rope;
-  if (do_rope && a.rope_in_smem) {
-    float2* st = reinterpret_cast<float2*>(smem + 8 * D * 4);
-    for (int e = tid; e < a.rd.entries; e += kThreads) st[e] = __ldg(&a.rope[e]);
-    tab = st;
-    __syncthreads();
-  }
-  float x[RPL][8];
-#pragma unroll
-  for (int i = 0; i < RPL; ++i) {
-    const bool valid = srcs[i] >= 0;
-    const int src = valid ? srcs[i] : 0;
-    const uint4 raw = raws[i];
+    const int row = 16 * warp + RPL * hb + i;
+    const int t = blk * kBlock + row;            // column sums need no gather: a sum over all rows
+    if (t >= a.N) continue;
+    const uint4 raw = *reinterpret_cast<const uint4*>(stage + (i * kThreads + tid) * 16);   // the chunk this thread fetched
     const unsigned int w[4] = {raw.x, raw.y, raw.z, raw.w};
+    float x[8];
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
-      x[i][2 * j] = __uint_as_float(w[j] << 16);
-      x[i][2 * j + 1] = __uint_as_float(w[j] & 0xffff0000u);
+      x[2 * j] = __uint_as_float(w[j] << 16);
+      x[2 * j + 1] = __uint_as_float(w[j] & 0xffff0000u);
     }
-    if (do_rope && valid) {
-      const unsigned int q1 = div40((unsigned)src, a.rd.mul_w);
-      const unsigned int tx = src - q1 * a.rd.grid_w;
-      const unsigned int tt = div40(q1, a.rd.mul_h);
-      const unsigned int ty = q1 - tt * a.rd.grid_h;
-      const unsigned int pos[3] = {tt, ty, tx};
+    if (do_rope) {
+      int pos[3];
+      grid_pos(a.rd, t, pos[0], pos[1], pos[2]);
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
         const int ax = p_axis[j];
-        const float2 cs = tab[p_idx[j] + (int)pos[ax] * a.rd.pairs[ax]];
-        const float x0 = x[i][2 * j], x1 = x[i][2 * j + 1];
-        x[i][2 * j] = x0 * cs.x - x1 * cs.y;
-        x[i][2 * j + 1] = x0 * cs.y + x1 * cs.x;
+        const float2 cs = tab[p_idx[j] + pos[ax] * a.rd.pairs[ax]];
+        const float x0 = x[2 * j], x1 = x[2 * j + 1];
+        x[2 * j] = x0 * cs.x - x1 * cs.y;
+        x[2 * j + 1] = x0 * cs.y + x1 * cs.x;
       }
     }
-    if (TENSOR == 1 && STAGE != kStageColSum && valid) {
 #pragma unroll
-      for (int c = 0; c < 8; ++c) x[i][c] -= kmean[c];
-    }
-    if (do_had) {
-      // in-register stages (channel bits 0..2)
-#pragma unroll
-      for (int s = 1; s < 8; s <<= 1) {
-#pragma unroll
-        for (int c = 0; c < 8; ++c) {
-          if (!(c & s)) {
-            const float u = x[i][c], v = x[i][c | s];
-            x[i][c] = u + v;
-            x[i][c | s] = u - v;
-          }
-        }
-      }
-      // cross-lane stages (channel bits 3..)
-#pragma unroll
-      for (int s = 1; s < LPR; s <<= 1) {
-        const bool upper = lr & s;
-#pragma unroll
-        for (int c = 0; c < 8; ++c) {
-          const float other = __shfl_xor_sync(0xffffffffu, x[i][c], s);
-          x[i][c] = upper ? other - x[i][c] : x[i][c] + other;
-        }
-      }
-      const float rs = D == 128 ? 0.08838834764831845f : 0.125f;   // 1/sqrt(D)
-#pragma unroll
-      for (int c = 0; c < 8; ++c) x[i][c] *= rs;
-    }
+    for (int c = 0; c < 8; ++c) s[c] += x[c];
   }
-
-  if constexpr (STAGE == kStageColSum) {
-    float s[8];
 #pragma unroll
-    for (int c = 0; c < 8; ++c) {
-      s[c] = 0.f;
+  for (int c = 0; c < 8; ++c) {
 #pragma unroll
-      for (int i = 0; i < RPL; ++i) s[c] += x[i][c];
-#pragma unroll
-      for (int m = LPR; m < 32; m <<= 1) s[c] += __shfl_xor_sync(0xffffffffu, s[c], m);
-    }
-    if (hb == 0) {
-#pragma unroll
-      for (int c = 0; c < 8; ++c) red[warp * D + 8 * lr + c] = s[c];
-    }
-    __syncthreads();
-    if (tid < D) {
-      float t = 0.f;
-#pragma unroll
-      for (int w8 = 0; w8 < 8; ++w8) t += red[w8 * D + tid];
-      a.k_part[((size_t)bh * a.nb + blk) * D + tid] = t;
-    }
-    return;
+    for (int m = LPR; m < 32; m <<= 1) s[c] += __shfl_xor_sync(0xffffffffu, s[c], m);
   }
-
-  // amax of the block (and of the head for the 4-bit outer scale)
-  float amax = 0.f;
-  if constexpr (STAGE != kStageQuant4) {
+  __syncthreads();                           // the previous item's reads of `red` are done
+  if (hb == 0) {
 #pragma unroll
-    for (int i = 0; i < RPL; ++i)
-#pragma unroll
-      for (int c = 0; c < 8; ++c) amax = fmaxf(amax, fabsf(x[i][c]));
-    amax = warp_max(amax);
-    __syncthreads();
-    if (lane == 0) red[warp] = amax;
-    __syncthreads();
-    amax = red[0];
-#pragma unroll
-    for (int w8 = 1; w8 < 8; ++w8) amax = fmaxf(amax, red[w8]);
+    for (int c = 0; c < 8; ++c) red[warp * D + 8 * lr + c] = s[c];
   }
-  if constexpr (STAGE == kStageAmax) {
-    if (tid == 0) atomicMax(&a.qk_amax[TENSOR * a.BH + bh], __float_as_uint(amax));
-    return;
-  }
-
-  if constexpr (STAGE == kStageQuant8) {
-    const float inv = amax > 0.f ? 448.0f / amax : 0.f;
-    if (tid == 0) (TENSOR == 0 ? a.q_scale : a.k_scale)[(size_t)bh * a.nb + blk] = amax > 0.f ? amax / 448.0f : 1.0f;
-    uint8_t* dst = (TENSOR == 0 ? a.q_codes : a.k_codes) + ((size_t)bh * a.n_pad + (size_t)blk * kBlock) * D;
+  __syncthreads();
+  if (tid < D) {
+    float t = 0.f;
 #pragma unroll
-    for (int i = 0; i < RPL; ++i) {
-      const int row = 16 * warp + RPL * hb + i;
-      unsigned int w[2];
-#pragma unroll
-      for (int j = 0; j < 2; ++j) {
-        const unsigned int lo = __nv_cvt_float2_to_fp8x2(make_float2(x[i][4 * j] * inv, x[i][4 * j + 1] * inv), __NV_SATFINITE, __NV_E4M3);
-        const unsigned int hi = __nv_cvt_float2_to_fp8x2(make_float2(x[i][4 * j + 2] * inv, x[i][4 * j + 3] * inv), __NV_SATFINITE, __NV_E4M3);
-        w[j] = lo | (hi << 16);
-      }
-      *reinterpret_cast<uint2*>(dst + (size_t)row * D + 8 * lr) = make_uint2(w[0], w[1]);
-    }
-  }
-
-  if constexpr (STAGE == kStageQuant4) {
-    // NVFP4: outer scale g per (b, h), microscale per token per 16 channels (= 2 lanes)
-    const float g = (TENSOR == 0 ? a.q_scale : a.k_scale)[bh];
-    const float inv6 = 1.0f / (6.0f * g);
-    uint8_t* dst = (TENSOR == 0 ? a.q_codes : a.k_codes) + ((size_t)bh * a.n_pad + (size_t)blk * kBlock) * (D / 2);
-    uint8_t* mdst = (TENSOR == 0 ? a.q_micro : a.k_micro) + ((size_t)bh * a.n_pad + (size_t)blk * kBlock) * (D / 16);
-#pragma unroll
-    for (int i = 0; i < RPL; ++i) {
-      const int row = 16 * warp + RPL * hb + i;
-      float m = 0.f;
-#pragma unroll
-      for (int c = 0; c < 8; ++c) m = fmaxf(m, fabsf(x[i][c]));
-      m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 1));
-      const unsigned int sb = __nv_cvt_float_to_fp8(m * inv6, __NV_SATFINITE, __NV_E4M3);
-      const float sdec = e4m3_to_float(sb);
-      const float rcp = sdec > 0.f ? 1.0f / (g * sdec) : 0.f;
-      unsigned int packed = 0;
-#pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        const unsigned int two = __nv_cvt_float2_to_fp4x2(make_float2(x[i][2 * j] * rcp, x[i][2 * j + 1] * rcp), __NV_E2M1, cudaRoundNearest);
-        packed |= (two & 0xffu) << (8 * j);
-      }
-      if (!(sdec > 0.f)) packed = 0;
-      *reinterpret_cast<unsigned int*>(dst + (size_t)row * (D / 2) + 4 * lr) = packed;
-      if (!(lr & 1)) mdst[(size_t)row * (D / 16) + (lr >> 1)] = (uint8_t)sb;
-    }
+    for (int w8 = 0; w8 < 8; ++w8) t += red[w8 * D + tid];
+    a.k_part[((size_t)bh * a.nb + blk) * D + tid] = t;
   }
 }
 
 // ---------------------------------------------------------------------------------------
-// Q / K body, one query/key row per thread (128 threads, one 128-row block per CTA).  All D
-// channels of a row sit in the registers of one thread, so the Hadamard rotation is D/2 * log2 D
-// register butterflies with no shuffle at all (a warp shuffle costs a full issue slot per 32
-// values, which made the lane-per-8-channels layout issue-bound), RoPE pairs and NVFP4 groups are
-// thread-local, and a row's codes leave as 16-byte stores.  Used for the amax and quantizing
-// stages; the column sums of K need the transposed ownership and keep the layout above.
-constexpr int kRowThreads = 128;
+// Q / K, one row per thread.  All D channels of a row sit in the registers of one thread, so
+// the Hadamard rotation is D/2 * log2 D register butterflies with no shuffle, RoPE pairs and
+// NVFP4 groups are thread-local, and a row's codes leave as 16-byte stores.
+enum { kStageAmax = 1, kStageQuant8 = 2, kStageQuant4 = 3 };
 
 template <int D> struct RopeSplit;          // pair boundaries of the default channel split
 template <> struct RopeSplit<128> { static constexpr int p1 = 22, p2 = 43; };   // 44 / 42 / 42
 template <> struct RopeSplit<64> { static constexpr int p1 = 12, p2 = 22; };    // 24 / 20 / 20
 
+// Reads the thread's row out of the stage, releases the stage, then transforms the row.
+// `red` is [2][4] floats and `kmean_s` [D] floats of compute-warp scratch.
 template <int D, int TENSOR /*0 = Q, 1 = K*/, int STAGE>
-__device__ __forceinline__ void qk_row_body(const PrepArgs& a, unsigned char* smem) {
+__device__ __forceinline__ void qk_row_item(const PrepArgs& a, const unsigned char* stage, float* red, float* kmean_s,
+                                            const float2* tab, int bh, int blk, int iter, bool new_head, int src_row) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int blk = blockIdx.x, bh = a.bh0 + blockIdx.y;
-  const int b = bh / a.H, h = bh - b * a.H;
-  const __nv_bfloat16* base = (TENSOR == 0 ? a.q : a.k) + b * a.stride_b + h * a.stride_h;
   const bool do_rope = a.flags & VC_FLAG_ROPE;
   const bool do_had = a.flags & VC_FLAG_HADAMARD;
-  const bool gather = TENSOR == 1 && a.perm != nullptr && STAGE >= kStageQuant8;
-  float* red = reinterpret_cast<float*>(smem);                   // [4] warp maxima
-  float* kmean_s = reinterpret_cast<float*>(smem + 64);          // [D]
-  float2* tab_s = reinterpret_cast<float2*>(smem + 64 + D * 4);
-
-  const int t = blk * kBlock + tid;
-  const bool valid = t < a.N;
-  int src = valid ? t : 0;
-  if (gather && valid) src = __ldg(&a.perm[(size_t)bh * a.N + t]);
+  const bool center = TENSOR == 1 && (a.flags & VC_FLAG_K_SMOOTH);
+  const bool valid = src_row >= 0;               // src_row: the input row behind this thread's row
+  const int src = valid ? src_row : 0;           // (RoPE acts at the source position)
   uint4 raw[D / 8];
 #pragma unroll
   for (int i = 0; i < D / 8; ++i) {
     raw[i] = make_uint4(0, 0, 0, 0);
-    if (valid) raw[i] = __ldg(reinterpret_cast<const uint4*>(base + (int64_t)src * a.stride_n + 8 * i));
+    if (valid) raw[i] = *reinterpret_cast<const uint4*>(stage + tid * Geo<D>::pitch + 16 * i);
   }
-  // tables -> shared memory while the row is in flight
-  const float2* tab = a.rope;
-  if (do_rope && a.rope_in_smem) {
-    for (int e = tid; e < a.rd.entries; e += kRowThreads) tab_s[e] = __ldg(&a.rope[e]);
-    tab = tab_s;
-  }
-  const bool center = TENSOR == 1 && (a.flags & VC_FLAG_K_SMOOTH);
-  if (center) {
+  if (center && new_head) {
+    __syncthreads();                               // everyone is done with the previous head's mean
     for (int c = tid; c < D; c += kRowThreads) kmean_s[c] = a.k_mean[(size_t)bh * D + c];
+    __syncthreads();
   }
-  __syncthreads();
 
   float x[D];
 #pragma unroll
@@ -347,10 +238,8 @@ __device__ __forceinline__ void qk_row_body(const PrepArgs& a, unsigned char* sm
     }
   }
   if (do_rope && valid) {
-    const unsigned int q1 = div40((unsigned)src, a.rd.mul_w);
-    const int tx = src - q1 * a.rd.grid_w;
-    const int tt = div40(q1, a.rd.mul_h);
-    const int ty = q1 - tt * a.rd.grid_h;
+    int tt, ty, tx;
+    grid_pos(a.rd, src, tt, ty, tx);
     // entry of pair p of axis ax: off[ax] + pos[ax] * pairs[ax] + (p - pair_start[ax])
     const int e0 = a.rd.off[0] + tt * a.rd.pairs[0] - a.rd.pair_start[0];
     const int e1 = a.rd.off[1] + ty * a.rd.pairs[1] - a.rd.pair_start[1];
@@ -399,12 +288,17 @@ __device__ __forceinline__ void qk_row_body(const PrepArgs& a, unsigned char* sm
 
   float amax = 0.f;
   if constexpr (STAGE != kStageQuant4) {
+    float m0 = 0.f, m1 = 0.f;
 #pragma unroll
-    for (int c = 0; c < D; ++c) amax = fmaxf(amax, fabsf(x[c]));
-    amax = warp_max(amax * rs);                 // max and the (positive) scale commute exactly
-    if (lane == 0) red[warp] = amax;
+    for (int c = 0; c < D; c += 4) {
+      m0 = max3(m0, fabsf(x[c]), fabsf(x[c + 1]));
+      m1 = max3(m1, fabsf(x[c + 2]), fabsf(x[c + 3]));
+    }
+    amax = warp_max(fmaxf(m0, m1) * rs);        // max and the (positive) scale commute exactly
+    float* rbuf = red + 4 * (iter & 1);         // alternate buffers: one barrier per item suffices
+    if (lane == 0) rbuf[warp] = amax;
     __syncthreads();
-    amax = fmaxf(fmaxf(red[0], red[1]), fmaxf(red[2], red[3]));
+    amax = fmaxf(fmaxf(rbuf[0], rbuf[1]), fmaxf(rbuf[2], rbuf[3]));
   }
   if constexpr (STAGE == kStageAmax) {
     if (tid == 0) atomicMax(&a.qk_amax[TENSOR * a.BH + bh], __float_as_uint(amax));
@@ -468,53 +362,24 @@ __device__ __forceinline__ void qk_row_body(const PrepArgs& a, unsigned char* sm
 }
 
 // ---------------------------------------------------------------------------------------
-// V body.  The gathered 128 x D block is staged in shared memory with coalesced 16-byte
-// loads; a thread then owns one channel pair and 128 / (256 / (D/2)) consecutive tokens,
-// so block means and the channel-major (token-contiguous) code rows need no transposition.
+// V.  A thread owns one channel pair and 128 / (256 / (D/2)) consecutive tokens of the gathered
+// block, so block means and the channel-major (token-contiguous) code rows need no transposition.
 enum { kVStats = 0, kVQuant8 = 1, kVQuant4 = 2 };
 
 template <int D, int STAGE>
-__device__ __forceinline__ void v_body(const PrepArgs& a, unsigned char* smem) {
-  constexpr int LPR = D / 8;
+__device__ __forceinline__ void v_item(const PrepArgs& a, const unsigned char* stage, float* red, int bh, int blk,
+                                       float2 mu_in, float2 am_in) {
   constexpr int CP = D / 2;             // channel pairs
   constexpr int TG = kThreads / CP;     // token groups
   constexpr int TPG = kBlock / TG;      // tokens per thread
   const int tid = threadIdx.x;
-  const int blk = blockIdx.x, bh = a.bh0 + blockIdx.y;
-  const int b = bh / a.H, h = bh - b * a.H;
-  const __nv_bfloat16* base = a.v + b * a.stride_b + h * a.stride_h;
-  uint4* tile4 = reinterpret_cast<uint4*>(smem);                       // [128][D] bf16
-  float* red = reinterpret_cast<float*>(smem + kBlock * D * 2);        // [TG][D]
-
-  {
-    constexpr int NL = kBlock * LPR / kThreads;   // 16-byte chunks per thread
-    int srcs[NL];
-#pragma unroll
-    for (int i = 0; i < NL; ++i) {
-      const int row = (tid + i * kThreads) / LPR;
-      const int t = blk * kBlock + row;
-      srcs[i] = t < a.N ? (a.perm ? __ldg(&a.perm[(size_t)bh * a.N + t]) : t) : -1;
-    }
-    uint4 vals[NL];
-#pragma unroll
-    for (int i = 0; i < NL; ++i) {
-      const int idx = tid + i * kThreads;
-      const int ch = idx % LPR;
-      vals[i] = make_uint4(0, 0, 0, 0);
-      if (srcs[i] >= 0) vals[i] = __ldg(reinterpret_cast<const uint4*>(base + (int64_t)srcs[i] * a.stride_n + 8 * ch));
-    }
-#pragma unroll
-    for (int i = 0; i < NL; ++i) tile4[tid + i * kThreads] = vals[i];
-  }
-  __syncthreads();
-
   const int cp = tid % CP, tg = tid / CP;
   const int n_valid = min(kBlock, a.N - blk * kBlock);
-  const unsigned int* tile32 = reinterpret_cast<const unsigned int*>(smem);
   float v0[TPG], v1[TPG];
 #pragma unroll
   for (int i = 0; i < TPG; ++i) {
-    const unsigned int w = tile32[(tg * TPG + i) * CP + cp];
+    const int row = tg * TPG + i;
+    const unsigned int w = row < n_valid ? *reinterpret_cast<const unsigned int*>(stage + row * (2 * D) + 4 * cp) : 0u;
     v0[i] = __uint_as_float(w << 16);
     v1[i] = __uint_as_float(w & 0xffff0000u);
   }
@@ -523,6 +388,7 @@ __device__ __forceinline__ void v_body(const PrepArgs& a, unsigned char* smem) {
   float mu0 = 0.f, mu1 = 0.f;
 
   if constexpr (STAGE == kVStats) {
+    __syncthreads();                         // the previous item's reads of `red` are done
     if (smooth) {
       float s0 = 0.f, s1 = 0.f;
 #pragma unroll
@@ -558,8 +424,8 @@ __device__ __forceinline__ void v_body(const PrepArgs& a, unsigned char* smem) {
     return;
   }
 
-  mu0 = a.v_mu[mu_at];
-  mu1 = a.v_mu[mu_at + 1];
+  mu0 = mu_in.x;
+  mu1 = mu_in.y;
   float r0[TPG], r1[TPG];
 #pragma unroll
   for (int i = 0; i < TPG; ++i) {
@@ -570,8 +436,7 @@ __device__ __forceinline__ void v_body(const PrepArgs& a, unsigned char* smem) {
   const size_t tok0 = (size_t)blk * kBlock + tg * TPG;
 
   if constexpr (STAGE == kVQuant8) {
-    const float am0 = __uint_as_float(a.v_amax[(size_t)bh * D + 2 * cp]);
-    const float am1 = __uint_as_float(a.v_amax[(size_t)bh * D + 2 * cp + 1]);
+    const float am0 = am_in.x, am1 = am_in.y;
     const float inv0 = am0 > 0.f ? 448.0f / am0 : 0.f, inv1 = am1 > 0.f ? 448.0f / am1 : 0.f;
     unsigned int w0[TPG / 4], w1[TPG / 4];
 #pragma unroll
@@ -642,14 +507,109 @@ __device__ __forceinline__ void v_body(const PrepArgs& a, unsigned char* smem) {
 }
 
 // ---------------------------------------------------------------------------------------
-// Launch 1: statistics.  z = 0: K column sums; z = 1: V block means + residual amax.
+// RoPE table -> shared memory (when it fits), once per CTA.
+__device__ __forceinline__ const float2* stage_rope_table(const PrepArgs& a, unsigned char* at) {
+  const float2* tab = a.rope;
+  if ((a.flags & VC_FLAG_ROPE) && a.rope_in_smem) {
+    float2* tab_s = reinterpret_cast<float2*>(at);
+    for (int e = threadIdx.x; e < a.rd.entries; e += blockDim.x) tab_s[e] = __ldg(&a.rope[e]);
+    tab = tab_s;
+  }
+  __syncthreads();
+  return tab;
+}
+
+// Launch 1a: column sums of RoPE(K) per block (the channel mean is taken after the rotation).
+// Shared memory: [2 stages x 32 KB][red: 8 D floats][RoPE table].
 template <int D>
-__global__ void __launch_bounds__(kThreads, 2) prep_stats_kernel(const PrepArgs a) {
-  extern __shared__ __align__(16) unsigned char smem[];
-  if (blockIdx.z == 0) {
-    if (a.flags & VC_FLAG_K_SMOOTH) qk_body<D, 1, kStageColSum>(a, smem);
-  } else {
-    v_body<D, kVStats>(a, smem);
+__global__ void __launch_bounds__(kThreads, 2) prep_kcolsum_kernel(const PrepArgs a, int n_items, int nh) {
+  constexpr int LPR = D / 8, RPL = LPR / 2, kStage = kThreads * RPL * 16;
+  extern __shared__ __align__(128) unsigned char smem[];
+  float* red = reinterpret_cast<float*>(smem + 2 * kStage);
+  const float2* tab = stage_rope_table(a, smem + 2 * kStage + 8 * D * 4);
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int lr = lane % LPR, hb = lane / LPR;
+  auto issue = [&](int item, int st) {
+    if (item < n_items) {
+      const Item w = decode_item(item, a.nb, nh, a.bh0);
+      const int b = w.bh / a.H, h = w.bh - b * a.H;
+      const __nv_bfloat16* base = a.k + b * a.stride_b + h * a.stride_h + 8 * lr;
+#pragma unroll
+      for (int i = 0; i < RPL; ++i) {
+        const int t = w.blk * kBlock + 16 * warp + RPL * hb + i;
+        if (t < a.N) cp_async16(smem + st * kStage + (i * kThreads + tid) * 16, base + (int64_t)t * a.stride_n);
+      }
+    }
+    cp_async_commit();
+  };
+  issue(blockIdx.x, 0);
+  int i = 0;
+  for (int item = blockIdx.x; item < n_items; item += gridDim.x, ++i) {
+    issue(item + gridDim.x, (i + 1) & 1);
+    cp_async_wait<1>();                       // this thread's chunks of item i have landed
+    const Item w = decode_item(item, a.nb, nh, a.bh0);
+    k_colsum_item<D>(a, smem + (i & 1) * kStage, red, tab, w.bh, w.blk);
+  }
+}
+
+// V pass: STAGE = block means + residual amax (launch 1b) or quantization of the residual.
+// Shared memory: [3 stages x (128 x 2 D)][red: 8 D floats].
+template <int D, int STAGE>
+__global__ void __launch_bounds__(kThreads, 2) prep_v_kernel(const PrepArgs a, int n_items, int nh) {
+  constexpr int LPR = D / 8, kStage = kBlock * 2 * D, NL = kBlock * LPR / kThreads;
+  extern __shared__ __align__(128) unsigned char smem[];
+  float* red = reinterpret_cast<float*>(smem + 3 * kStage);
+  const int tid = threadIdx.x;
+  auto fetch = [&](int item, int (&src)[NL]) {          // source rows of the chunks this thread copies
+#pragma unroll
+    for (int c = 0; c < NL; ++c) src[c] = -1;
+    if (item >= n_items) return;
+    const Item w = decode_item(item, a.nb, nh, a.bh0);
+#pragma unroll
+    for (int c = 0; c < NL; ++c) {
+      const int t = w.blk * kBlock + (tid + c * kThreads) / LPR;
+      if (t < a.N) src[c] = a.perm ? __ldg(&a.perm[(size_t)w.bh * a.N + t]) : t;
+    }
+  };
+  auto issue = [&](int item, int st, const int (&src)[NL]) {
+    if (item < n_items) {
+      const Item w = decode_item(item, a.nb, nh, a.bh0);
+      const int b = w.bh / a.H, h = w.bh - b * a.H;
+      const __nv_bfloat16* base = a.v + b * a.stride_b + h * a.stride_h + 8 * (tid % LPR);
+#pragma unroll
+      for (int c = 0; c < NL; ++c)
+        if (src[c] >= 0) cp_async16(smem + st * kStage + (tid + c * kThreads) * 16, base + (int64_t)src[c] * a.stride_n);
+    }
+    cp_async_commit();
+  };
+  // per-item scalars of the quantizing stage, fetched one item ahead
+  const int cp = tid % (D / 2);
+  auto fetch_mu = [&](int item) -> float2 {
+    if (STAGE == kVStats || item >= n_items) return make_float2(0.f, 0.f);
+    const Item w = decode_item(item, a.nb, nh, a.bh0);
+    return *reinterpret_cast<const float2*>(a.v_mu + ((size_t)w.bh * a.nb + w.blk) * D + 2 * cp);
+  };
+  int src[NL];
+  fetch(blockIdx.x, src);
+  issue(blockIdx.x, 0, src);
+  fetch(blockIdx.x + gridDim.x, src);
+  issue(blockIdx.x + gridDim.x, 1, src);
+  fetch(blockIdx.x + 2 * gridDim.x, src);
+  float2 mu = fetch_mu(blockIdx.x), am = make_float2(0.f, 0.f);
+  int i = 0, last_bh = -1;
+  for (int item = blockIdx.x; item < n_items; item += gridDim.x, ++i) {
+    cp_async_wait<1>();                       // my chunks of item i have landed ...
+    __syncthreads();                          // ... and everyone's; all are done with item i-1
+    issue(item + 2 * gridDim.x, (i + 2) % 3, src);
+    fetch(item + 3 * gridDim.x, src);
+    const float2 mu_next = fetch_mu(item + gridDim.x);
+    const Item w = decode_item(item, a.nb, nh, a.bh0);
+    if (STAGE == kVQuant8 && w.bh != last_bh) {
+      am = make_float2(__uint_as_float(a.v_amax[(size_t)w.bh * D + 2 * cp]), __uint_as_float(a.v_amax[(size_t)w.bh * D + 2 * cp + 1]));
+      last_bh = w.bh;
+    }
+    v_item<D, STAGE>(a, smem + (i % 3) * kStage, red, w.bh, w.blk, mu, am);
+    mu = mu_next;
   }
 }
 
@@ -680,29 +640,54 @@ __global__ void prep_finalize_kernel(const PrepArgs a, int which) {
   }
 }
 
-// 4-bit only: head amax of the rotated Q (tensor 0) or of the centered, rotated K (tensor 1).
-template <int D, int TENSOR>
-__global__ void __launch_bounds__(kRowThreads, 2) prep_amax_kernel(const PrepArgs a) {
-  extern __shared__ __align__(16) unsigned char smem[];
-  qk_row_body<D, TENSOR, kStageAmax>(a, smem);
-}
-
-// Launch 3: quantization of Q (z = 0) and K (z = 1), one row per thread.
-template <int D, int BITS>
-__global__ void __launch_bounds__(kRowThreads, 3) prep_quant_qk_kernel(const PrepArgs a) {
-  extern __shared__ __align__(16) unsigned char smem[];
-  if (blockIdx.z == 0) {
-    qk_row_body<D, 0, BITS == 8 ? kStageQuant8 : kStageQuant4>(a, smem);
-  } else {
-    qk_row_body<D, 1, BITS == 8 ? kStageQuant8 : kStageQuant4>(a, smem);
+// Q/K pass, one row per thread: STAGE = amax (4-bit head amax of tensor z0), or quantization
+// of Q (z = 0) and K (z = 1).  Shared memory: [2 stages x 128 x pitch][scratch][RoPE table].
+template <int D, int STAGE>
+__global__ void __launch_bounds__(kRowThreads, 2) prep_qk_kernel(const PrepArgs a, int n_items, int nh, int z0) {
+  extern __shared__ __align__(128) unsigned char smem[];
+  float* red = reinterpret_cast<float*>(smem + 2 * Geo<D>::stage_bytes);      // [2][4]
+  float* kmean_s = red + 16;                                                  // [D]
+  const float2* tab = stage_rope_table(a, smem + 2 * Geo<D>::stage_bytes + 64 + D * 4);
+  const int tid = threadIdx.x;
+  auto fetch = [&](int item) -> int {        // input row behind my row of the item, -1 if none
+    if (item >= n_items) return -1;
+    const Item w = decode_item(item, a.nb, nh, a.bh0);
+    const int t = w.blk * kBlock + tid;
+    if (t >= a.N) return -1;
+    // the head amax is a maximum over all rows: that stage reads the rows in place
+    const bool gather = (w.z + z0) == 1 && a.perm != nullptr && STAGE != kStageAmax;
+    return gather ? __ldg(&a.perm[(size_t)w.bh * a.N + t]) : t;
+  };
+  auto issue = [&](int item, int st, int src) {
+    if (src >= 0) {
+      const Item w = decode_item(item, a.nb, nh, a.bh0);
+      const int b = w.bh / a.H, h = w.bh - b * a.H;
+      const __nv_bfloat16* row = ((w.z + z0) == 0 ? a.q : a.k) + b * a.stride_b + h * a.stride_h + (int64_t)src * a.stride_n;
+      unsigned char* dst = smem + st * Geo<D>::stage_bytes + tid * Geo<D>::pitch;
+#pragma unroll
+      for (int c = 0; c < D / 8; ++c) cp_async16(dst + 16 * c, row + 8 * c);
+    }
+    cp_async_commit();
+  };
+  int s0 = fetch(blockIdx.x);
+  issue(blockIdx.x, 0, s0);
+  int s1 = fetch(blockIdx.x + gridDim.x);
+  int i = 0, last_bh = -1;
+  for (int item = blockIdx.x; item < n_items; item += gridDim.x, ++i) {
+    issue(item + gridDim.x, (i + 1) & 1, s1);
+    const int s2 = fetch(item + 2 * gridDim.x);
+    cp_async_wait<1>();                       // my row of item i has landed
+    const Item w = decode_item(item, a.nb, nh, a.bh0);
+    const unsigned char* stage = smem + (i & 1) * Geo<D>::stage_bytes;
+    if (w.z + z0 == 0) {
+      qk_row_item<D, 0, STAGE>(a, stage, red, kmean_s, tab, w.bh, w.blk, i, false, s0);
+    } else {
+      qk_row_item<D, 1, STAGE>(a, stage, red, kmean_s, tab, w.bh, w.blk, i, w.bh != last_bh, s0);
+      last_bh = w.bh;
+    }
+    s0 = s1;
+    s1 = s2;
   }
-}
-
-// Launch 4: quantization of the V residual.
-template <int D, int BITS>
-__global__ void __launch_bounds__(kThreads, 2) prep_quant_v_kernel(const PrepArgs a) {
-  extern __shared__ __align__(16) unsigned char smem[];
-  v_body<D, BITS == 8 ? kVQuant8 : kVQuant4>(a, smem);
 }
 
 template <typename K>
@@ -710,21 +695,31 @@ cudaError_t allow_smem(K kernel, size_t bytes) {
   return bytes > 48 * 1024 ? cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) : cudaSuccess;
 }
 
+int persistent_grid(int n_items, int per_sm = 2) {
+  static int sms = 0;
+  if (!sms) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
+      sms = 148;
+  }
+  const int g = per_sm * sms;
+  return n_items < g ? n_items : g;
+}
+
 template <int D, int BITS>
 cudaError_t run(const Problem& pr, PrepArgs a, const WorkLayout& wl, uint8_t* work, cudaStream_t s) {
   const size_t rope_bytes = ((a.flags & VC_FLAG_ROPE) && a.rope_in_smem) ? (size_t)a.rd.entries * 8 : 0;
-  const size_t lane_smem = 8 * D * 4 + rope_bytes;                      // qk_body (column sums)
-  const size_t v_smem = (size_t)kBlock * D * 2 + (kThreads / (D / 2)) * D * 4;
-  const size_t stats_smem = lane_smem > v_smem ? lane_smem : v_smem;
-  const size_t row_smem = 64 + D * 4 + rope_bytes;                      // qk_row_body
+  const size_t colsum_smem = 2 * (size_t)kThreads * (D / 16) * 16 + 8 * D * 4 + rope_bytes;
+  const size_t row_smem = 2 * (size_t)Geo<D>::stage_bytes + 64 + D * 4 + rope_bytes;
+  const size_t v_smem = 3 * (size_t)kBlock * 2 * D + 8 * D * 4;
+  constexpr int kQuant = BITS == 8 ? kStageQuant8 : kStageQuant4;
+  constexpr int kVQuant = BITS == 8 ? kVQuant8 : kVQuant4;
   cudaError_t e;
-  if ((e = allow_smem(prep_stats_kernel<D>, stats_smem)) != cudaSuccess) return e;
-  if ((e = allow_smem(prep_quant_qk_kernel<D, BITS>, row_smem)) != cudaSuccess) return e;
-  if ((e = allow_smem(prep_quant_v_kernel<D, BITS>, v_smem)) != cudaSuccess) return e;
-  if (BITS == 4) {
-    if ((e = allow_smem(prep_amax_kernel<D, 0>, row_smem)) != cudaSuccess) return e;
-    if ((e = allow_smem(prep_amax_kernel<D, 1>, row_smem)) != cudaSuccess) return e;
-  }
+  if ((e = allow_smem(prep_kcolsum_kernel<D>, colsum_smem)) != cudaSuccess) return e;
+  if ((e = allow_smem(prep_v_kernel<D, kVStats>, v_smem)) != cudaSuccess) return e;
+  if ((e = allow_smem(prep_v_kernel<D, kVQuant>, v_smem)) != cudaSuccess) return e;
+  if ((e = allow_smem(prep_qk_kernel<D, kQuant>, row_smem)) != cudaSuccess) return e;
+  if (BITS == 4 && (e = allow_smem(prep_qk_kernel<D, kStageAmax>, row_smem)) != cudaSuccess) return e;
   if ((e = cudaMemsetAsync(work + wl.status, 0, 4, s)) != cudaSuccess) return e;
   if ((e = cudaMemsetAsync(work + wl.amax, 0, wl.amax_bytes, s)) != cudaSuccess) return e;
   if (a.flags & VC_FLAG_ROPE) {
@@ -736,18 +731,23 @@ cudaError_t run(const Problem& pr, PrepArgs a, const WorkLayout& wl, uint8_t* wo
   if (group > 32768) group = 32768;
   for (int bh0 = 0; bh0 < pr.BH; bh0 += group) {
     const int nh = pr.BH - bh0 < group ? pr.BH - bh0 : group;
+    const int per = pr.nb * nh;
     a.bh0 = bh0;
-    prep_stats_kernel<D><<<dim3(pr.nb, nh, 2), kThreads, stats_smem, s>>>(a);
-    if (BITS == 4) { prep_amax_kernel<D, 0><<<dim3(pr.nb, nh), kRowThreads, row_smem, s>>>(a); count_launches(1); }
+    if (a.flags & VC_FLAG_K_SMOOTH) {
+      prep_kcolsum_kernel<D><<<persistent_grid(per), kThreads, colsum_smem, s>>>(a, per, nh);
+      count_launches(1);
+    }
+    prep_v_kernel<D, kVStats><<<persistent_grid(per), kThreads, v_smem, s>>>(a, per, nh);
+    if (BITS == 4) { prep_qk_kernel<D, kStageAmax><<<persistent_grid(per), kRowThreads, row_smem, s>>>(a, per, nh, 0); count_launches(1); }
     prep_finalize_kernel<D, BITS><<<nh, D, 0, s>>>(a, 0);
     count_launches(2);
     if (BITS == 4) {
-      prep_amax_kernel<D, 1><<<dim3(pr.nb, nh), kRowThreads, row_smem, s>>>(a);
+      prep_qk_kernel<D, kStageAmax><<<persistent_grid(per), kRowThreads, row_smem, s>>>(a, per, nh, 1);
       prep_finalize_kernel<D, BITS><<<nh, 32, 0, s>>>(a, 1);
       count_launches(2);
     }
-    prep_quant_qk_kernel<D, BITS><<<dim3(pr.nb, nh, 2), kRowThreads, row_smem, s>>>(a);
-    prep_quant_v_kernel<D, BITS><<<dim3(pr.nb, nh), kThreads, v_smem, s>>>(a);
+    prep_qk_kernel<D, kQuant><<<persistent_grid(2 * per), kRowThreads, row_smem, s>>>(a, 2 * per, nh, 0);
+    prep_v_kernel<D, kVQuant><<<persistent_grid(per), kThreads, v_smem, s>>>(a, per, nh);
     count_launches(2);
   }
   return cudaGetLastError();

@@ -128,14 +128,16 @@ def test_vc_attn_end_to_end_config1(perm_kind):
         assert m0["max_err_over_vmax"] < m1["max_err_over_vmax"] + 1e-2, (m0, m1)
 
 
+@pytest.mark.parametrize("variant", [0, 1], ids=["block_scaled_fp4", "serial_bf16"])
 @pytest.mark.parametrize("perm_kind", ["identity", "random"])
 @pytest.mark.parametrize("case", SMALL, ids=[c[0] for c in SMALL])
-def test_vc_attn_4bit_end_to_end(case, perm_kind):
-    """4-bit path (NVFP4 Q, K, residual and P): vc_attn against the oracle's emulation."""
+def test_vc_attn_4bit_end_to_end(case, perm_kind, variant):
+    """4-bit path (NVFP4 Q, K, residual and P): vc_attn against the oracle's emulation, for the
+    block-scaled FP4 kernel (default) and the serial kernel that expands the operands to bf16."""
     _, B, H, N, d, grid = case
     q, k, v = _inputs(B, H, N, d, grid, seed=31)
     perm = None if perm_kind == "identity" else vc_inputs.random_perm(B, H, N, 8).cuda()
-    p = Params.make(B, H, N, d, grid, bits=4)
+    p = Params.make(B, H, N, d, grid, bits=4, kernel_variant=variant)
     quant, work = alloc_buffers(p)
     o = torch.empty(B, H, N, d, dtype=torch.bfloat16, device="cuda")
     vc.vc_attn(p, q, k, v, perm, o, quant, work)
