@@ -173,7 +173,9 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="c3")
     ap.add_argument("--bits", type=int, default=8)
-    ap.add_argument("--perm", default="kmeans", choices=["kmeans", "identity", "random"])
+    ap.add_argument("--perm", default="group", choices=["group", "kmeans", "identity", "random"],
+                    help="group: vc_group on the GPU, recomputed (warm-started) every 4th step inside the timed\n"
+                         "region and reused in between; kmeans: the harness's torch k-means, computed once")
     ap.add_argument("--heads-per-pass", type=int, default=0)
     ap.add_argument("--ref-rows", type=int, default=1024)
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -211,13 +213,19 @@ def main():
         q, k, v = [torch.randn(w.B, w.H, w.N, w.d, generator=g, device=dev).to(torch.bfloat16) for _ in range(3)]
     else:
         q, k, v = vc_inputs.make_qkv(w, device=dev)
-    if args.perm == "kmeans":
+    p = Params.make(w.B, w.H, w.N, w.d, w.grid, bits=args.bits, heads_per_pass=args.heads_per_pass)
+    group_k, group_every = 64, 4
+    if args.perm == "group":
+        gwork = torch.empty(vc.vc_group_workspace_bytes(p), dtype=torch.uint8, device=dev)
+        centroids = torch.zeros(w.B, w.H, group_k, w.d, dtype=torch.float32, device=dev)
+        perm = torch.empty(w.B, w.H, w.N, dtype=torch.int32, device=dev)
+        vc.vc_group(p, v, group_k, 4, False, centroids, perm, gwork)      # cold start: 4 Lloyd iterations
+    elif args.perm == "kmeans":
         perm = vc_inputs.kmeans_perm_all(v)
     elif args.perm == "random":
         perm = vc_inputs.random_perm(w.B, w.H, w.N, w.seed, device=dev)
     else:
         perm = None
-    p = Params.make(w.B, w.H, w.N, w.d, w.grid, bits=args.bits, heads_per_pass=args.heads_per_pass)
     quant, work = alloc_buffers(p, device=dev)
     o = torch.empty(w.B, w.H, w.N, w.d, dtype=torch.bfloat16, device=dev)
     stream = torch.cuda.current_stream()
@@ -232,13 +240,16 @@ def main():
         vc.vc_attn(p, q, k, v, perm, o, quant, work)
     vc.vc_poll_status(work)
 
-    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(args.steps)]
     launches0 = vc.vc_launch_count()
     barrier()
     wall0 = time.time()
     t_start, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     t_start.record(stream)
     for s in range(args.steps):
+        ev[s][3].record(stream)
+        if args.perm == "group" and s % group_every == 0:     # a grouping step: one warm-started iteration
+            vc.vc_group(p, v, group_k, 1, True, centroids, perm, gwork)
         ev[s][0].record(stream)
         vc.vc_prep(p, q, k, v, perm, quant, work)
         ev[s][1].record(stream)
@@ -253,6 +264,12 @@ def main():
     ms_total = t_start.elapsed_time(t_end)
     prep_ms = statistics.mean(e[0].elapsed_time(e[1]) for e in ev)
     attn_ms = statistics.mean(e[1].elapsed_time(e[2]) for e in ev)
+    group = None
+    if args.perm == "group":
+        calls = [e[3].elapsed_time(e[0]) for i, e in enumerate(ev) if i % group_every == 0]
+        group = {"ms_per_call": statistics.mean(calls), "calls": len(calls), "every": group_every, "k": group_k,
+                 "iters": {"cold": 4, "warm": 1}, "ms_amortized_per_step": sum(calls) / args.steps,
+                 "share_of_attention_on_a_grouping_step": statistics.mean(calls) / attn_ms}
     value, ms_step = job_throughput(w.flops, ms_total / args.steps, world, dev)
 
     # end to end through the host-buffer entry point: H2D of Q, K, V, pi and D2H of O inside the timer
@@ -296,13 +313,14 @@ def main():
         "vs_baseline": None, "dtype": "e4m3" if args.bits == 8 else "nvfp4", "data": "synthetic",
         "config": {"workload": w.name, "B": w.B, "H": w.H, "N": w.N, "d": w.d, "grid": list(w.grid),
                    "bits": args.bits, "perm": args.perm, "data": args.data, "l2": "inputs larger than L2 (Q+K+V = %.0f MB)" % (3 * q.numel() * 2 / 1e6),
-                   "step": "vc_prep + vc_attn_fwd"},
+                   "step": "vc_prep + vc_attn_fwd" + (" (+ vc_group every 4th step)" if args.perm == "group" else "")},
         "clocks": clocks, "gpu_launches": launches, "e2e": e2e,
         "roofline": {"bound": "tensor", "kernel": "vc_attn_fwd", "achieved": achieved, "peak": peak, "unit": UNIT,
                      "frac": achieved / peak, "traffic": None,
                      "peak_source": f"{peaks['source']}: bf16 sustained {peaks['bf16_sustained']} TF/s x {ratio:g}" + (" (nominal FP8:bf16)" if args.bits == 8 else " (nominal FP4:bf16)"),
                      ("frac_of_nominal_fp8_4500" if args.bits == 8 else "frac_of_nominal_fp4_9000"): achieved / (4500.0 if args.bits == 8 else 9000.0),
                      "ms": attn_ms},
+        "group": group,
         "prep": {"ms": prep_ms, "algorithmic_gb": prep_bytes / 1e9, "gbs": prep_gbs,
                  "frac_of_measured_hbm": prep_gbs / peaks["hbm_gbs"], "frac_of_8tbs": prep_gbs / 8000.0},
     }

@@ -13,6 +13,8 @@
  *                (ExpCast-FP8, Eq. 7), low-bit P V, and the block means added back inside
  *                the recurrence (Eq. 6); epilogue O = s_V * A / l.
  *   vc_attn      vc_prep followed by vc_attn_fwd.
+ *   vc_group     the producer of the token-group permutation pi (Sec. 3.2): k-means on V,
+ *                stable argsort of the labels.
  *
  * Conventions
  *   - Every pointer is a DEVICE pointer unless the name says host; all must be 16-byte
@@ -137,6 +139,26 @@ vc_status vc_attn_host(const vc_params *p, const void *q_host, const void *k_hos
                        const void *v_host, const int32_t *perm_host, void *o_host,
                        void *q_dev, void *k_dev, void *v_dev, int32_t *perm_dev, void *o_dev,
                        void *quant, void *workspace, void *stream);
+
+/* Token grouping (Sec. 3.2 "Value-guided permutation"): per (b, h) a k-means over the value
+ * tokens labels every token, and perm = argsort(labels), stable: row t of the permuted K/V is
+ * row perm[t] of the input (Eq. 3), every cluster one contiguous run.  The output is the `perm`
+ * argument of vc_prep / vc_attn; a caller following the paper's schedule (Sec. 3.4 "Amortized
+ * grouping schedule") calls this on the first ceil(n/4) denoising steps, every 4th step, with
+ * warm_start = 1 after the first call, and reuses `perm` in between.
+ *   v          [B][H][N][d] bf16, strides as in vc_params
+ *   k          clusters, 1 <= k <= min(N, 64)
+ *   iters      Lloyd iterations (assign, then update), >= 1; labels are those of the last assignment
+ *   warm_start 0: centroids start at rows 0, N/k, 2 N/k, ... of V; 1: at the values in `centroids`
+ *   centroids  [B][H][k][d] fp32, in (warm start) and out (after the last update)
+ *   perm       out, int32 [B][H][N]
+ *   workspace  vc_group_workspace_bytes(p) bytes; on return its first B*H*N int32 are the labels
+ * The paper leaves k, the initialisation and the iteration count open; distances are squared
+ * Euclidean on the fp32 rows, ties go to the lower cluster index, an empty cluster keeps its
+ * centroid.  Deterministic (no floating-point atomics).  Returns VC_ERR_UNSUPPORTED for k > 64. */
+size_t vc_group_workspace_bytes(const vc_params *p);
+vc_status vc_group(const vc_params *p, const void *v, int32_t k, int32_t iters, int32_t warm_start,
+                   float *centroids, int32_t *perm, void *workspace, void *stream);
 
 /* vc_prep without a workspace argument and without any allocation.  (The paper has no
  * counterpart: this entry point exists for the sake of its callers, not of the method.)

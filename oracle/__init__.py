@@ -6,6 +6,7 @@ A plain, slow NumPy restatement of what the path computes, written from the pape
 * ``prep``       the preprocessing chain (Sec. 3.4 "Fused preprocessing", App. B)
 * ``attention``  exact fp64 attention and the emulated low-bit recurrence
                  (Eq. 1, Eq. 6, Eq. 7)
+* ``grouping``   the value-guided permutation (Sec. 3.2): k-means labels, stable argsort
 
 Only the tests, ``__graft_entry__.smoke()`` and the ``cpu_baseline`` / ``--impl reference``
 legs of ``bench.py`` may import this package.  It shares no code with the CUDA path and
@@ -18,4 +19,7 @@ paper's worked example and printed constants; the recurrence by brute-force atte
 with quantization switched off.  The *end-to-end quantized* output has no printed value
 in the paper: "parity unpinned" for the granularity of the Q/K scales, the NVFP4
 second-level scales and the RoPE channel split, which are readings fixed by this build.
+Grouping is pinned by brute-force nearest-centroid search, cluster recovery on separated
+blobs, the monotone k-means objective and the definition of a stable sort; k, the
+initialisation and the iteration count are readings too ("parity unpinned").
 """

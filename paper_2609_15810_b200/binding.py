@@ -77,6 +77,10 @@ def load_library():
     lib.vc_attn.argtypes = [P, vp, vp, vp, i32p, vp, vp, vp, vp]
     lib.vc_attn_host.restype = ctypes.c_int
     lib.vc_attn_host.argtypes = [P] + [vp] * 13
+    lib.vc_group_workspace_bytes.restype = ctypes.c_size_t
+    lib.vc_group_workspace_bytes.argtypes = [P]
+    lib.vc_group.restype = ctypes.c_int
+    lib.vc_group.argtypes = [P, vp, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, vp, i32p, vp, vp]
     lib.vc_quant_view.restype = ctypes.c_int
     lib.vc_quant_view.argtypes = [P, vp, ctypes.POINTER(QuantView)]
     lib.vc_poll_status.restype = ctypes.c_int
@@ -145,6 +149,16 @@ def vc_attn_host(p, q_host, k_host, v_host, perm_host, o_host, q_dev, k_dev, v_d
     _check(load_library().vc_attn_host(ctypes.byref(p), _ptr(q_host), _ptr(k_host), _ptr(v_host), _ptr(perm_host),
                                        _ptr(o_host), _ptr(q_dev), _ptr(k_dev), _ptr(v_dev), _ptr(perm_dev),
                                        _ptr(o_dev), _ptr(quant), _ptr(workspace), _stream()), "vc_attn_host")
+
+
+def vc_group_workspace_bytes(p):
+    return int(load_library().vc_group_workspace_bytes(ctypes.byref(p)))
+
+
+def vc_group(p, v, k, iters, warm_start, centroids, perm, workspace):
+    """k-means on the value tokens -> perm = stable argsort of the labels (centroids in/out)."""
+    _check(load_library().vc_group(ctypes.byref(p), _ptr(v), int(k), int(iters), int(bool(warm_start)), _ptr(centroids),
+                                   _ptr(perm), _ptr(workspace), _stream()), "vc_group")
 
 
 def vc_quant_view(p, quant):

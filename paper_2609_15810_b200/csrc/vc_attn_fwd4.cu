@@ -14,7 +14,9 @@
 // softmax stage: P is quantized to NVFP4 per row and 16 keys.  The group maxima are a
 // by-product of the running-max pass; per group the E4M3 factor of max p / 6 is formed once,
 // its log2 is folded into the exponent offset, and every element costs one FMA, one ex2 and
-// half a conversion:  code = E2M1(2^(s cs + log2 2688 - m' - log2 f_g)).
+// half a conversion:  code = E2M1(2^(s cs + log2 2688 - m' - log2 f_g)).  (Moving part of the
+// exponentials to a polynomial on the FMA pipe was measured and is slower: the stage is bound by
+// issue slots and hand-off latency before the special-function unit, which runs at 64 %.)
 #include <cuda_bf16.h>
 #include <cuda_fp8.h>
 
