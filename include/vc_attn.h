@@ -134,7 +134,11 @@ vc_status vc_attn(const vc_params *p, const void *q, const void *k, const void *
 /* The same with HOST input/output buffers (pinned memory recommended): copies q, k, v
  * (packed [B][H][N][d] bf16) and perm (or NULL) to the device staging buffers q_dev,
  * k_dev, v_dev, perm_dev, runs vc_attn, copies o_dev to o_host and synchronizes the
- * stream.  The staging buffers are caller-allocated device memory of the same sizes. */
+ * stream.  The staging buffers are caller-allocated device memory of the same sizes.
+ * Heads are independent, so the call works through groups of heads and overlaps the
+ * input copy of the next group and the output copy of the previous one with the kernels of
+ * the current one, on two helper streams that it creates and destroys itself (ordered after
+ * the work already on `stream`; `stream` is complete when the call returns). */
 vc_status vc_attn_host(const vc_params *p, const void *q_host, const void *k_host,
                        const void *v_host, const int32_t *perm_host, void *o_host,
                        void *q_dev, void *k_dev, void *v_dev, int32_t *perm_dev, void *o_dev,

@@ -1,5 +1,6 @@
 // C-ABI entry points of libvc: argument validation, buffer layouts, launch sequencing.
 #include <atomic>
+#include <vector>
 #include <cstring>
 
 #include "vc_internal.h"
@@ -190,22 +191,61 @@ vc_status vc_attn_host(const vc_params* p, const void* q_host, const void* k_hos
         pr.stride_b != (int64_t)pr.H * pr.N * pr.d)
       return VC_ERR_INVALID_ARG;   // host buffers are packed
   }
+  // Heads are independent, so the call is pipelined over groups of heads: while group g is
+  // computed on `stream`, group g+1 is on its way in on a copy stream and group g-1 on its
+  // way out on another (PCIe is full duplex).  The bundle and workspace are reused by every
+  // group, which is safe because the groups' kernels run in order on `stream`.
   cudaStream_t s = (cudaStream_t)stream;
-  const size_t bytes = (size_t)pr.BH * pr.N * pr.d * 2;
-  if (cudaMemcpyAsync(q_dev, q_host, bytes, cudaMemcpyHostToDevice, s) != cudaSuccess ||
-      cudaMemcpyAsync(k_dev, k_host, bytes, cudaMemcpyHostToDevice, s) != cudaSuccess ||
-      cudaMemcpyAsync(v_dev, v_host, bytes, cudaMemcpyHostToDevice, s) != cudaSuccess)
-    return VC_ERR_CUDA;
-  if (perm_host &&
-      cudaMemcpyAsync(perm_dev, perm_host, (size_t)pr.BH * pr.N * 4, cudaMemcpyHostToDevice, s) !=
-          cudaSuccess)
-    return VC_ERR_CUDA;
-  st = vc_attn(p, q_dev, k_dev, v_dev, perm_host ? perm_dev : nullptr, o_dev, quant, workspace,
-               stream);
-  if (st != VC_OK) return st;
-  if (cudaMemcpyAsync(o_host, o_dev, bytes, cudaMemcpyDeviceToHost, s) != cudaSuccess)
-    return VC_ERR_CUDA;
-  return cudaStreamSynchronize(s) == cudaSuccess ? VC_OK : VC_ERR_CUDA;
+  // heads per group: about a tenth of the heads, in multiples that keep a group's slice of
+  // perm 16-byte aligned (N * 4 bytes per head)
+  const int mult = pr.N % 4 == 0 ? 1 : (pr.N % 2 == 0 ? 2 : 4);
+  int hg = pr.BH >= 10 ? (pr.BH + 9) / 10 : 1;
+  hg = (hg + mult - 1) / mult * mult;
+  const int groups = (pr.BH + hg - 1) / hg;
+  const size_t head_elems = (size_t)pr.N * pr.d;
+  cudaStream_t s_in = nullptr, s_out = nullptr;
+  std::vector<cudaEvent_t> ev(2 * groups + 2, nullptr);
+  bool ok = cudaStreamCreateWithFlags(&s_in, cudaStreamNonBlocking) == cudaSuccess &&
+            cudaStreamCreateWithFlags(&s_out, cudaStreamNonBlocking) == cudaSuccess;
+  for (size_t i = 0; ok && i < ev.size(); ++i) ok = cudaEventCreateWithFlags(&ev[i], cudaEventDisableTiming) == cudaSuccess;
+  vc_status result = VC_OK;
+  if (ok) {
+    cudaEvent_t e_begin = ev[2 * groups], e_end = ev[2 * groups + 1];
+    ok = cudaEventRecord(e_begin, s) == cudaSuccess && cudaStreamWaitEvent(s_in, e_begin, 0) == cudaSuccess &&
+         cudaStreamWaitEvent(s_out, e_begin, 0) == cudaSuccess;
+    vc_params sub = *p;
+    sub.B = 1;
+    sub.stride_b = sub.stride_h = sub.stride_n = 0;
+    for (int g = 0; ok && g < groups; ++g) {
+      const int h0 = g * hg, nh = pr.BH - h0 < hg ? pr.BH - h0 : hg;
+      const size_t off = (size_t)h0 * head_elems * 2, bytes = (size_t)nh * head_elems * 2;
+      ok = cudaMemcpyAsync((char*)q_dev + off, (const char*)q_host + off, bytes, cudaMemcpyHostToDevice, s_in) == cudaSuccess &&
+           cudaMemcpyAsync((char*)k_dev + off, (const char*)k_host + off, bytes, cudaMemcpyHostToDevice, s_in) == cudaSuccess &&
+           cudaMemcpyAsync((char*)v_dev + off, (const char*)v_host + off, bytes, cudaMemcpyHostToDevice, s_in) == cudaSuccess;
+      if (ok && perm_host)
+        ok = cudaMemcpyAsync(perm_dev + (size_t)h0 * pr.N, perm_host + (size_t)h0 * pr.N, (size_t)nh * pr.N * 4,
+                             cudaMemcpyHostToDevice, s_in) == cudaSuccess;
+      ok = ok && cudaEventRecord(ev[2 * g], s_in) == cudaSuccess && cudaStreamWaitEvent(s, ev[2 * g], 0) == cudaSuccess;
+      if (!ok) break;
+      sub.H = nh;
+      const vc_status st_g = vc_attn(&sub, (char*)q_dev + off, (char*)k_dev + off, (char*)v_dev + off,
+                                     perm_host ? perm_dev + (size_t)h0 * pr.N : nullptr, (char*)o_dev + off, quant,
+                                     workspace, stream);
+      if (st_g != VC_OK) { result = st_g; break; }
+      ok = cudaEventRecord(ev[2 * g + 1], s) == cudaSuccess && cudaStreamWaitEvent(s_out, ev[2 * g + 1], 0) == cudaSuccess &&
+           cudaMemcpyAsync((char*)o_host + off, (char*)o_dev + off, bytes, cudaMemcpyDeviceToHost, s_out) == cudaSuccess;
+    }
+    // join: `stream` is complete only when the last output copy is
+    if (cudaEventRecord(e_end, s_out) != cudaSuccess || cudaStreamWaitEvent(s, e_end, 0) != cudaSuccess) ok = false;
+    if (cudaStreamSynchronize(s_in) != cudaSuccess) ok = false;
+    if (cudaStreamSynchronize(s) != cudaSuccess) ok = false;
+  }
+  for (cudaEvent_t e : ev)
+    if (e) cudaEventDestroy(e);
+  if (s_in) cudaStreamDestroy(s_in);
+  if (s_out) cudaStreamDestroy(s_out);
+  if (result != VC_OK) return result;
+  return ok ? VC_OK : VC_ERR_CUDA;
 }
 
 vc_status vc_quant_view(const vc_params* p, const void* quant, vc_quant_ptrs* out) {

@@ -97,3 +97,27 @@ def test_strided_inputs_through_vc_attn():
         vc.vc_poll_status(work)
         outs.append(o)
     assert torch.equal(outs[0], outs[1])
+
+
+@pytest.mark.parametrize("shape", [(2, 6, 300, 64, (3, 10, 10)), (1, 3, 257, 128, (1, 1, 257))], ids=["12_heads_6_groups", "3_heads"])
+@pytest.mark.parametrize("bits", [8, 4])
+def test_host_entry_point_equals_the_device_path(shape, bits):
+    """vc_attn_host (pinned host buffers in and out, pipelined over groups of heads) gives exactly
+    the output of vc_attn on the same inputs, with and without a permutation."""
+    B, H, N, d, grid = shape
+    w = vc_inputs.Workload("t", B, H, N, d, grid, (8,), 77, "gauss")
+    q, k, v = [t.cuda() for t in vc_inputs.make_qkv(w)]
+    for perm in (None, vc_inputs.random_perm(B, H, N, 3).cuda()):
+        p = Params.make(B, H, N, d, grid, bits=bits)
+        quant, work = alloc_buffers(p)
+        o_ref = torch.empty(B, H, N, d, dtype=torch.bfloat16, device="cuda")
+        vc.vc_attn(p, q, k, v, perm, o_ref, quant, work)
+        vc.vc_poll_status(work)
+        hq, hk, hv = [t.cpu().pin_memory() for t in (q, k, v)]
+        hperm = perm.cpu().pin_memory() if perm is not None else None
+        ho = torch.zeros(B, H, N, d, dtype=torch.bfloat16).pin_memory()
+        dq, dk, dv, do = [torch.zeros_like(q) for _ in range(4)]
+        dperm = torch.zeros(B, H, N, dtype=torch.int32, device="cuda") if perm is not None else None
+        vc.vc_attn_host(p, hq, hk, hv, hperm, ho, dq, dk, dv, dperm, do, quant, work)
+        vc.vc_poll_status(work)
+        assert torch.equal(ho, o_ref.cpu())
