@@ -303,6 +303,11 @@ def main():
     ratio = 2.0 if args.bits == 8 else 4.0   # nominal dense FP8 : bf16 = 2, FP4 : bf16 = 4
     peak = peaks["bf16_sustained"] * ratio
     achieved = w.flops / (attn_ms * 1e-3) / 1e12
+    # DRAM traffic of one attention launch: measured once under ncu on a smaller case of the same
+    # kernel (the headline launch is too long to capture) and proportional to B*H*N (codes in,
+    # bf16 out; key/value re-reads are L2 hits)
+    per_ht = {8: 323.9e6, 4: 220.6e6}[args.bits] / (32 * 16384) * (w.d / 128.0)
+    traffic = per_ht * w.B * w.H * w.N
     n_pad = 128 * ((w.N + 127) // 128)
     prep_bytes = w.B * w.H * (3 * w.N * w.d * 2 + 2 * w.N * 4 + 3 * n_pad * w.d * (1 if args.bits == 8 else 0.5625)
                               + (2 * (n_pad // 128) * 4 + w.d * 4) + (n_pad // 128) * w.d * 2)
@@ -316,7 +321,9 @@ def main():
                    "step": "vc_prep + vc_attn_fwd" + (" (+ vc_group every 4th step)" if args.perm == "group" else "")},
         "clocks": clocks, "gpu_launches": launches, "e2e": e2e,
         "roofline": {"bound": "tensor", "kernel": "vc_attn_fwd", "achieved": achieved, "peak": peak, "unit": UNIT,
-                     "frac": achieved / peak, "traffic": None,
+                     "frac": achieved / peak, "traffic": traffic,
+                     "traffic_source": "ncu dram__bytes_read+write of this kernel on B2 H16 N16384 d128 "
+                                       "(profiles/), scaled by head-tokens: %.0f B per (head, token)" % per_ht,
                      "peak_source": f"{peaks['source']}: bf16 sustained {peaks['bf16_sustained']} TF/s x {ratio:g}" + (" (nominal FP8:bf16)" if args.bits == 8 else " (nominal FP4:bf16)"),
                      ("frac_of_nominal_fp8_4500" if args.bits == 8 else "frac_of_nominal_fp4_9000"): achieved / (4500.0 if args.bits == 8 else 9000.0),
                      "ms": attn_ms},

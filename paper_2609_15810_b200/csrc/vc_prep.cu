@@ -128,22 +128,33 @@ __device__ __forceinline__ void grid_pos(const RopeDesc& rd, int src, int& tt, i
 // ---------------------------------------------------------------------------------------
 // K column sums after RoPE (the channel mean of Sec. 3.4 is taken after the rotation).  A lane
 // owns 8 consecutive channels of D/16 rows, so a column's partial sums meet by xor-shuffles.
+struct PairSlots {          // the 4 channel pairs a lane owns: axis and table slot of each
+  int axis[4], idx[4], stride[4];
+};
+__device__ __forceinline__ PairSlots pair_slots(const RopeDesc& rd, int first_pair) {
+  PairSlots ps;
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    const int p = first_pair + j;
+    const int ax = p >= rd.pair_start[2] ? 2 : (p >= rd.pair_start[1] ? 1 : 0);
+    ps.axis[j] = ax;
+    ps.idx[j] = rd.off[ax] + (p - rd.pair_start[ax]);
+    ps.stride[j] = rd.pairs[ax];
+  }
+  return ps;
+}
+
 template <int D>
 __device__ __forceinline__ void k_colsum_item(const PrepArgs& a, const unsigned char* stage, float* red, const float2* tab,
-                                              int bh, int blk) {
+                                              const PairSlots& ps, int bh, int blk) {
   constexpr int LPR = D / 8;         // lanes per row
   constexpr int RPL = LPR / 2;       // rows per lane (a warp covers 16 rows)
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int lr = lane % LPR, hb = lane / LPR;
   const bool do_rope = a.flags & VC_FLAG_ROPE;
-  int p_axis[4], p_idx[4];
-#pragma unroll
-  for (int j = 0; j < 4; ++j) {
-    const int p = 4 * lr + j;
-    const int ax = p >= a.rd.pair_start[2] ? 2 : (p >= a.rd.pair_start[1] ? 1 : 0);
-    p_axis[j] = ax;
-    p_idx[j] = a.rd.off[ax] + (p - a.rd.pair_start[ax]);
-  }
+  // grid position of the lane's first row; the following rows advance x with carry
+  int tt, ty, tx;
+  grid_pos(a.rd, blk * kBlock + 16 * warp + RPL * hb, tt, ty, tx);
   float s[8];
 #pragma unroll
   for (int c = 0; c < 8; ++c) s[c] = 0.f;
@@ -151,7 +162,7 @@ __device__ __forceinline__ void k_colsum_item(const PrepArgs& a, const unsigned 
   for (int i = 0; i < RPL; ++i) {
     const int row = 16 * warp + RPL * hb + i;
     const int t = blk * kBlock + row;            // column sums need no gather: a sum over all rows
-    if (t >= a.N) continue;
+    if (t >= a.N) break;                         // rows of a lane ascend: the rest is padding too
     const uint4 raw = *reinterpret_cast<const uint4*>(stage + (i * kThreads + tid) * 16);   // the chunk this thread fetched
     const unsigned int w[4] = {raw.x, raw.y, raw.z, raw.w};
     float x[8];
@@ -161,16 +172,15 @@ __device__ __forceinline__ void k_colsum_item(const PrepArgs& a, const unsigned 
       x[2 * j + 1] = __uint_as_float(w[j] & 0xffff0000u);
     }
     if (do_rope) {
-      int pos[3];
-      grid_pos(a.rd, t, pos[0], pos[1], pos[2]);
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
-        const int ax = p_axis[j];
-        const float2 cs = tab[p_idx[j] + pos[ax] * a.rd.pairs[ax]];
+        const int pos = ps.axis[j] == 0 ? tt : (ps.axis[j] == 1 ? ty : tx);
+        const float2 cs = tab[ps.idx[j] + pos * ps.stride[j]];
         const float x0 = x[2 * j], x1 = x[2 * j + 1];
         x[2 * j] = x0 * cs.x - x1 * cs.y;
         x[2 * j + 1] = x0 * cs.y + x1 * cs.x;
       }
+      if (++tx == a.rd.grid_w) { tx = 0; if (++ty == a.rd.grid_h) { ty = 0; ++tt; } }
     }
 #pragma unroll
     for (int c = 0; c < 8; ++c) s[c] += x[c];
@@ -529,6 +539,7 @@ __global__ void __launch_bounds__(kThreads, 2) prep_kcolsum_kernel(const PrepArg
   const float2* tab = stage_rope_table(a, smem + 2 * kStage + 8 * D * 4);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int lr = lane % LPR, hb = lane / LPR;
+  const PairSlots ps = pair_slots(a.rd, 4 * lr);
   auto issue = [&](int item, int st) {
     if (item < n_items) {
       const Item w = decode_item(item, a.nb, nh, a.bh0);
@@ -548,7 +559,7 @@ __global__ void __launch_bounds__(kThreads, 2) prep_kcolsum_kernel(const PrepArg
     issue(item + gridDim.x, (i + 1) & 1);
     cp_async_wait<1>();                       // this thread's chunks of item i have landed
     const Item w = decode_item(item, a.nb, nh, a.bh0);
-    k_colsum_item<D>(a, smem + (i & 1) * kStage, red, tab, w.bh, w.blk);
+    k_colsum_item<D>(a, smem + (i & 1) * kStage, red, tab, ps, w.bh, w.blk);
   }
 }
 
@@ -560,20 +571,22 @@ __global__ void __launch_bounds__(kThreads, 2) prep_v_kernel(const PrepArgs a, i
   extern __shared__ __align__(128) unsigned char smem[];
   float* red = reinterpret_cast<float*>(smem + 3 * kStage);
   const int tid = threadIdx.x;
-  auto fetch = [&](int item, int (&src)[NL]) {          // source rows of the chunks this thread copies
+  // items i .. i+3 of this CTA, decoded once each (the divisions are not free at 64 elements per thread)
+  Item q0 = decode_item(blockIdx.x, a.nb, nh, a.bh0), q1 = decode_item(blockIdx.x + gridDim.x, a.nb, nh, a.bh0),
+       q2 = decode_item(blockIdx.x + 2 * gridDim.x, a.nb, nh, a.bh0), q3 = decode_item(blockIdx.x + 3 * gridDim.x, a.nb, nh, a.bh0);
+  auto fetch = [&](int item, const Item& w, int (&src)[NL]) {          // source rows of the chunks this thread copies
 #pragma unroll
     for (int c = 0; c < NL; ++c) src[c] = -1;
     if (item >= n_items) return;
-    const Item w = decode_item(item, a.nb, nh, a.bh0);
+    const int32_t* prow = a.perm + (size_t)w.bh * a.N;
 #pragma unroll
     for (int c = 0; c < NL; ++c) {
       const int t = w.blk * kBlock + (tid + c * kThreads) / LPR;
-      if (t < a.N) src[c] = a.perm ? __ldg(&a.perm[(size_t)w.bh * a.N + t]) : t;
+      if (t < a.N) src[c] = a.perm ? __ldg(prow + t) : t;
     }
   };
-  auto issue = [&](int item, int st, const int (&src)[NL]) {
+  auto issue = [&](int item, const Item& w, int st, const int (&src)[NL]) {
     if (item < n_items) {
-      const Item w = decode_item(item, a.nb, nh, a.bh0);
       const int b = w.bh / a.H, h = w.bh - b * a.H;
       const __nv_bfloat16* base = a.v + b * a.stride_b + h * a.stride_h + 8 * (tid % LPR);
 #pragma unroll
@@ -584,32 +597,32 @@ __global__ void __launch_bounds__(kThreads, 2) prep_v_kernel(const PrepArgs a, i
   };
   // per-item scalars of the quantizing stage, fetched one item ahead
   const int cp = tid % (D / 2);
-  auto fetch_mu = [&](int item) -> float2 {
+  auto fetch_mu = [&](int item, const Item& w) -> float2 {
     if (STAGE == kVStats || item >= n_items) return make_float2(0.f, 0.f);
-    const Item w = decode_item(item, a.nb, nh, a.bh0);
     return *reinterpret_cast<const float2*>(a.v_mu + ((size_t)w.bh * a.nb + w.blk) * D + 2 * cp);
   };
   int src[NL];
-  fetch(blockIdx.x, src);
-  issue(blockIdx.x, 0, src);
-  fetch(blockIdx.x + gridDim.x, src);
-  issue(blockIdx.x + gridDim.x, 1, src);
-  fetch(blockIdx.x + 2 * gridDim.x, src);
-  float2 mu = fetch_mu(blockIdx.x), am = make_float2(0.f, 0.f);
+  fetch(blockIdx.x, q0, src);
+  issue(blockIdx.x, q0, 0, src);
+  fetch(blockIdx.x + gridDim.x, q1, src);
+  issue(blockIdx.x + gridDim.x, q1, 1, src);
+  fetch(blockIdx.x + 2 * gridDim.x, q2, src);
+  float2 mu = fetch_mu(blockIdx.x, q0), am = make_float2(0.f, 0.f);
   int i = 0, last_bh = -1;
   for (int item = blockIdx.x; item < n_items; item += gridDim.x, ++i) {
     cp_async_wait<1>();                       // my chunks of item i have landed ...
     __syncthreads();                          // ... and everyone's; all are done with item i-1
-    issue(item + 2 * gridDim.x, (i + 2) % 3, src);
-    fetch(item + 3 * gridDim.x, src);
-    const float2 mu_next = fetch_mu(item + gridDim.x);
-    const Item w = decode_item(item, a.nb, nh, a.bh0);
-    if (STAGE == kVQuant8 && w.bh != last_bh) {
-      am = make_float2(__uint_as_float(a.v_amax[(size_t)w.bh * D + 2 * cp]), __uint_as_float(a.v_amax[(size_t)w.bh * D + 2 * cp + 1]));
-      last_bh = w.bh;
+    issue(item + 2 * gridDim.x, q2, (i + 2) % 3, src);
+    fetch(item + 3 * gridDim.x, q3, src);
+    const float2 mu_next = fetch_mu(item + gridDim.x, q1);
+    if (STAGE == kVQuant8 && q0.bh != last_bh) {
+      am = make_float2(__uint_as_float(a.v_amax[(size_t)q0.bh * D + 2 * cp]), __uint_as_float(a.v_amax[(size_t)q0.bh * D + 2 * cp + 1]));
+      last_bh = q0.bh;
     }
-    v_item<D, STAGE>(a, smem + (i % 3) * kStage, red, w.bh, w.blk, mu, am);
+    v_item<D, STAGE>(a, smem + (i % 3) * kStage, red, q0.bh, q0.blk, mu, am);
     mu = mu_next;
+    q0 = q1; q1 = q2; q2 = q3;
+    q3 = decode_item(item + 4 * gridDim.x, a.nb, nh, a.bh0);
   }
 }
 
