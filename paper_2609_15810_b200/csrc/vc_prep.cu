@@ -217,8 +217,9 @@ template <> struct RopeSplit<64> { static constexpr int p1 = 12, p2 = 22; };    
 // Reads the thread's row out of the stage, releases the stage, then transforms the row.
 // `red` is [2][4] floats and `kmean_s` [D] floats of compute-warp scratch.
 template <int D, int TENSOR /*0 = Q, 1 = K*/, int STAGE>
-__device__ __forceinline__ void qk_row_item(const PrepArgs& a, const unsigned char* stage, float* red, float* kmean_s,
-                                            const float2* tab, int bh, int blk, int iter, bool new_head, int src_row) {
+__device__ __forceinline__ void qk_row_item(const PrepArgs& a, const unsigned char* stage, unsigned char* out_tile, float* red,
+                                            float* kmean_s, const float2* tab, int bh, int blk, int iter, bool new_head,
+                                            int src_row) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const bool do_rope = a.flags & VC_FLAG_ROPE;
   const bool do_had = a.flags & VC_FLAG_HADAMARD;
@@ -319,7 +320,10 @@ __device__ __forceinline__ void qk_row_item(const PrepArgs& a, const unsigned ch
   if constexpr (STAGE == kStageQuant8) {
     const float inv = amax > 0.f ? 448.0f / amax : 0.f;
     if (tid == 0) (TENSOR == 0 ? a.q_scale : a.k_scale)[(size_t)bh * a.nb + blk] = amax > 0.f ? amax / 448.0f : 1.0f;
-    uint4* dst = reinterpret_cast<uint4*>((TENSOR == 0 ? a.q_codes : a.k_codes) + row_g * D);
+    // codes go to the swizzled output tile; the CTA copies it out with coalesced stores
+    constexpr int CPR = D / 16;
+    uint4* dst = reinterpret_cast<uint4*>(out_tile + tid * D);
+    const int sw = (tid / (8 / CPR)) & (CPR - 1);
 #pragma unroll
     for (int i = 0; i < D / 16; ++i) {
       unsigned int w[4];
@@ -330,7 +334,7 @@ __device__ __forceinline__ void qk_row_item(const PrepArgs& a, const unsigned ch
         const unsigned int hi = __nv_cvt_float2_to_fp8x2(make_float2((x[c + 2] * rs) * inv, (x[c + 3] * rs) * inv), __NV_SATFINITE, __NV_E4M3);
         w[j] = lo | (hi << 16);
       }
-      dst[i] = make_uint4(w[0], w[1], w[2], w[3]);
+      dst[i ^ sw] = make_uint4(w[0], w[1], w[2], w[3]);
     }
   }
 
@@ -362,9 +366,11 @@ __device__ __forceinline__ void qk_row_item(const PrepArgs& a, const unsigned ch
         codes[2 * gq + wi] = sdec > 0.f ? word : 0u;
       }
     }
-    uint4* dst = reinterpret_cast<uint4*>((TENSOR == 0 ? a.q_codes : a.k_codes) + row_g * (D / 2));
+    constexpr int CPR = D / 32;
+    uint4* dst = reinterpret_cast<uint4*>(out_tile + tid * (D / 2));
+    const int sw = (tid / (8 / CPR)) & (CPR - 1);
 #pragma unroll
-    for (int i = 0; i < D / 32; ++i) dst[i] = make_uint4(codes[4 * i], codes[4 * i + 1], codes[4 * i + 2], codes[4 * i + 3]);
+    for (int i = 0; i < D / 32; ++i) dst[i ^ sw] = make_uint4(codes[4 * i], codes[4 * i + 1], codes[4 * i + 2], codes[4 * i + 3]);
     unsigned int* mdst = reinterpret_cast<unsigned int*>((TENSOR == 0 ? a.q_micro : a.k_micro) + row_g * (D / 16));
 #pragma unroll
     for (int i = 0; i < D / 64; ++i) mdst[i] = micro[i];
@@ -654,13 +660,21 @@ __global__ void prep_finalize_kernel(const PrepArgs a, int which) {
 }
 
 // Q/K pass, one row per thread: STAGE = amax (4-bit head amax of tensor z0), or quantization
-// of Q (z = 0) and K (z = 1).  Shared memory: [2 stages x 128 x pitch][scratch][RoPE table].
+// of Q (z = 0) and K (z = 1).  Loads and stores are coalesced: the CTA copies the next block in
+// with consecutive lanes on consecutive 16-byte chunks (two rows per warp instruction, the source
+// rows taken from a small ring of permutation slices in shared memory), a thread then reads its
+// row from the padded tile; codes leave through a swizzled tile in the same way.
+// Shared memory: [2 stages x 128 x pitch][out tile 128 x D][src ring 3 x 128][scratch][RoPE table].
 template <int D, int STAGE>
 __global__ void __launch_bounds__(kRowThreads, 2) prep_qk_kernel(const PrepArgs a, int n_items, int nh, int z0) {
+  constexpr int kRowBytes = STAGE == kStageQuant4 ? D / 2 : D;      // code bytes per row
+  constexpr int CPR = kRowBytes / 16;                                // 16-byte chunks per code row
   extern __shared__ __align__(128) unsigned char smem[];
-  float* red = reinterpret_cast<float*>(smem + 2 * Geo<D>::stage_bytes);      // [2][4]
-  float* kmean_s = red + 16;                                                  // [D]
-  const float2* tab = stage_rope_table(a, smem + 2 * Geo<D>::stage_bytes + 64 + D * 4);
+  unsigned char* out_tile = smem + 2 * Geo<D>::stage_bytes;
+  int* src_ring = reinterpret_cast<int*>(out_tile + kBlock * D);     // [3][128]
+  float* red = reinterpret_cast<float*>(src_ring + 3 * kBlock);      // [2][4]
+  float* kmean_s = red + 16;                                         // [D]
+  const float2* tab = stage_rope_table(a, reinterpret_cast<unsigned char*>(kmean_s + D));
   const int tid = threadIdx.x;
   auto fetch = [&](int item) -> int {        // input row behind my row of the item, -1 if none
     if (item >= n_items) return -1;
@@ -671,35 +685,53 @@ __global__ void __launch_bounds__(kRowThreads, 2) prep_qk_kernel(const PrepArgs 
     const bool gather = (w.z + z0) == 1 && a.perm != nullptr && STAGE != kStageAmax;
     return gather ? __ldg(&a.perm[(size_t)w.bh * a.N + t]) : t;
   };
-  auto issue = [&](int item, int st, int src) {
-    if (src >= 0) {
+  auto issue = [&](int item, int st, const int* src) {
+    if (item < n_items) {
       const Item w = decode_item(item, a.nb, nh, a.bh0);
       const int b = w.bh / a.H, h = w.bh - b * a.H;
-      const __nv_bfloat16* row = ((w.z + z0) == 0 ? a.q : a.k) + b * a.stride_b + h * a.stride_h + (int64_t)src * a.stride_n;
-      unsigned char* dst = smem + st * Geo<D>::stage_bytes + tid * Geo<D>::pitch;
+      const __nv_bfloat16* base = ((w.z + z0) == 0 ? a.q : a.k) + b * a.stride_b + h * a.stride_h + 8 * (tid % (D / 8));
+      unsigned char* dst = smem + st * Geo<D>::stage_bytes + 16 * (tid % (D / 8));
 #pragma unroll
-      for (int c = 0; c < D / 8; ++c) cp_async16(dst + 16 * c, row + 8 * c);
+      for (int c = 0; c < D / 8; ++c) {
+        const int row = (c * kRowThreads + tid) / (D / 8);
+        const int sr = src[row];
+        if (sr >= 0) cp_async16(dst + row * Geo<D>::pitch, base + (int64_t)sr * a.stride_n);
+      }
     }
     cp_async_commit();
   };
-  int s0 = fetch(blockIdx.x);
-  issue(blockIdx.x, 0, s0);
-  int s1 = fetch(blockIdx.x + gridDim.x);
+  src_ring[tid] = fetch(blockIdx.x);
+  src_ring[kBlock + tid] = fetch(blockIdx.x + gridDim.x);
+  int nxt = fetch(blockIdx.x + 2 * gridDim.x);
+  __syncthreads();
+  issue(blockIdx.x, 0, src_ring);
   int i = 0, last_bh = -1;
   for (int item = blockIdx.x; item < n_items; item += gridDim.x, ++i) {
-    issue(item + gridDim.x, (i + 1) & 1, s1);
-    const int s2 = fetch(item + 2 * gridDim.x);
-    cp_async_wait<1>();                       // my row of item i has landed
+    cp_async_wait<0>();                       // my chunks of item i have landed ...
+    __syncthreads();                          // ... and everyone's; item i-1 is finished everywhere
+    src_ring[((i + 2) % 3) * kBlock + tid] = nxt;
+    nxt = fetch(item + 3 * gridDim.x);
+    issue(item + gridDim.x, (i + 1) & 1, src_ring + ((i + 1) % 3) * kBlock);
     const Item w = decode_item(item, a.nb, nh, a.bh0);
     const unsigned char* stage = smem + (i & 1) * Geo<D>::stage_bytes;
+    const int s0 = src_ring[(i % 3) * kBlock + tid];
     if (w.z + z0 == 0) {
-      qk_row_item<D, 0, STAGE>(a, stage, red, kmean_s, tab, w.bh, w.blk, i, false, s0);
+      qk_row_item<D, 0, STAGE>(a, stage, out_tile, red, kmean_s, tab, w.bh, w.blk, i, false, s0);
     } else {
-      qk_row_item<D, 1, STAGE>(a, stage, red, kmean_s, tab, w.bh, w.blk, i, w.bh != last_bh, s0);
+      qk_row_item<D, 1, STAGE>(a, stage, out_tile, red, kmean_s, tab, w.bh, w.blk, i, w.bh != last_bh, s0);
       last_bh = w.bh;
     }
-    s0 = s1;
-    s1 = s2;
+    if constexpr (STAGE != kStageAmax) {
+      __syncthreads();                        // the code tile is complete
+      uint8_t* gdst = (w.z + z0 == 0 ? a.q_codes : a.k_codes) + ((size_t)w.bh * a.n_pad + (size_t)w.blk * kBlock) * kRowBytes;
+#pragma unroll
+      for (int c = 0; c < CPR; ++c) {
+        const int idx = c * kRowThreads + tid, row = idx / CPR, chunk = idx % CPR;
+        const int sw = (row / (8 / CPR)) & (CPR - 1);
+        const uint4 v = *reinterpret_cast<const uint4*>(out_tile + row * kRowBytes + ((chunk ^ sw) << 4));
+        *reinterpret_cast<uint4*>(gdst + (size_t)idx * 16) = v;
+      }
+    }
   }
 }
 
@@ -723,7 +755,7 @@ template <int D, int BITS>
 cudaError_t run(const Problem& pr, PrepArgs a, const WorkLayout& wl, uint8_t* work, cudaStream_t s) {
   const size_t rope_bytes = ((a.flags & VC_FLAG_ROPE) && a.rope_in_smem) ? (size_t)a.rd.entries * 8 : 0;
   const size_t colsum_smem = 2 * (size_t)kThreads * (D / 16) * 16 + 8 * D * 4 + rope_bytes;
-  const size_t row_smem = 2 * (size_t)Geo<D>::stage_bytes + 64 + D * 4 + rope_bytes;
+  const size_t row_smem = 2 * (size_t)Geo<D>::stage_bytes + (size_t)kBlock * D + 3 * kBlock * 4 + 64 + D * 4 + rope_bytes;
   const size_t v_smem = 3 * (size_t)kBlock * 2 * D + 8 * D * 4;
   constexpr int kQuant = BITS == 8 ? kStageQuant8 : kStageQuant4;
   constexpr int kVQuant = BITS == 8 ? kVQuant8 : kVQuant4;
