@@ -318,21 +318,27 @@ attn4_fwd_2q_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       sh->alpha[t][row] = ex2_approx(m_run - m_new);      // alpha; 0 on the first tile
       mbar_arrive(&sh->a_full[t][j & 1]);
       m_run = m_new;
-      // the previous code tile must have been consumed before it is overwritten
-      if (j > 0 && !warp_wait2(&sh->o_done[t], (j - 1) & 1, sh, a.status, 31)) break;
-
-      // p = 2^(s cs - m') * 2688: the row maximum maps to 6 * 448, so the largest factor is 448
+      // p = 2^(s cs - m') * 2688: the row maximum maps to 6 * 448, so the largest factor is 448.
+      // Per 16-key group: factor = E4M3(max p / 6); element / factor = 2^(s cs + c0 - log2 factor),
+      // a zero factor zeroes the group.  The eight factor chains run before the wait below: they
+      // do not touch the code tile.
       const float c0 = 11.39231742277876f - m_new;        // log2(2688) - m'
       uint32_t sfw[2] = {0u, 0u};
-      auto quant16 = [&](const uint32_t (&sv)[32], int half, int g) -> uint2 {   // keys 16 g .. 16 g + 15
+      float off[8];
+#pragma unroll
+      for (int g = 0; g < 8; ++g) {
         const float pmax = ex2_approx(fmaf(mx[g], cs, c0));
         const uint32_t sb = (uint32_t)__nv_cvt_float_to_fp8(pmax * (1.0f / 6.0f), __NV_SATFINITE, __NV_E4M3);
         sfw[g >> 2] |= sb << (8 * (g & 3));
-        // element / factor = 2^(s cs + c0 - log2 factor); a zero factor zeroes the group
-        const float off = sb ? c0 - lg2_approx(decode_ue4m3(sb)) : -INFINITY;
+        off[g] = sb ? c0 - lg2_approx(decode_ue4m3(sb)) : -INFINITY;
+      }
+      // the previous code tile must have been consumed before it is overwritten
+      if (j > 0 && !warp_wait2(&sh->o_done[t], (j - 1) & 1, sh, a.status, 31)) break;
+
+      auto quant16 = [&](const uint32_t (&sv)[32], int half, int g) -> uint2 {   // keys 16 g .. 16 g + 15
         float v[16];
 #pragma unroll
-        for (int i = 0; i < 16; ++i) v[i] = ex2_approx(fmaf(__uint_as_float(sv[16 * half + i]), cs, off));
+        for (int i = 0; i < 16; ++i) v[i] = ex2_approx(fmaf(__uint_as_float(sv[16 * half + i]), cs, off[g]));
         return make_uint2(cvt_e2m1x8(v[0], v[1], v[2], v[3], v[4], v[5], v[6], v[7]),
                           cvt_e2m1x8(v[8], v[9], v[10], v[11], v[12], v[13], v[14], v[15]));
       };
