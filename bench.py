@@ -177,6 +177,7 @@ def main():
                     help="group: vc_group on the GPU, recomputed (warm-started) every 4th step inside the timed\n"
                          "region and reused in between; kmeans: the harness's torch k-means, computed once")
     ap.add_argument("--heads-per-pass", type=int, default=0)
+    ap.add_argument("--variant", type=int, default=0, help="attention kernel (vc_params.kernel_variant)")
     ap.add_argument("--ref-rows", type=int, default=1024)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
@@ -213,7 +214,8 @@ def main():
         q, k, v = [torch.randn(w.B, w.H, w.N, w.d, generator=g, device=dev).to(torch.bfloat16) for _ in range(3)]
     else:
         q, k, v = vc_inputs.make_qkv(w, device=dev)
-    p = Params.make(w.B, w.H, w.N, w.d, w.grid, bits=args.bits, heads_per_pass=args.heads_per_pass)
+    p = Params.make(w.B, w.H, w.N, w.d, w.grid, bits=args.bits, heads_per_pass=args.heads_per_pass,
+                    kernel_variant=args.variant)
     group_k, group_every = 64, 4
     if args.perm == "group":
         gwork = torch.empty(vc.vc_group_workspace_bytes(p), dtype=torch.uint8, device=dev)

@@ -24,15 +24,6 @@ namespace {
 using namespace sm100;
 using namespace attn;
 
-struct AttnArgs {
-  const float *q_scale, *k_scale, *v_scale;
-  const __nv_bfloat16* v_means;
-  __nv_bfloat16* o;
-  uint32_t* status;
-  int N, n_pad, nb, p_format;
-  float sl;        // softmax_scale * log2(e)
-  float code_off;  // 120 + beta  (Eq. 7)
-};
 
 // Value of an ExpCast / E4M3 code in [0, 126] (non-negative): normals by placing the
 // exponent and mantissa fields into an fp32 pattern, subnormals (codes 1..7) as m * 2^-9.

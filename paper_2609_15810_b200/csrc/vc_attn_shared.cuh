@@ -15,6 +15,17 @@ using namespace sm100;
 
 constexpr uint32_t kErrTimeout = 0x100;
 
+// Arguments of the 8-bit attention kernels.
+struct AttnArgs {
+  const float *q_scale, *k_scale, *v_scale;
+  const __nv_bfloat16* v_means;
+  __nv_bfloat16* o;
+  uint32_t* status;
+  int N, n_pad, nb, p_format;
+  float sl;        // softmax_scale * log2(e)
+  float code_off;  // 120 + beta  (Eq. 7)
+};
+
 constexpr int kStages2 = 4;
 constexpr uint32_t kWaitLimit2 = 1u << 18;   // x up to 4 us per try: about one second
 

@@ -121,3 +121,31 @@ def test_host_entry_point_equals_the_device_path(shape, bits):
         vc.vc_attn_host(p, hq, hk, hv, hperm, ho, dq, dk, dv, dperm, do, quant, work)
         vc.vc_poll_status(work)
         assert torch.equal(ho, o_ref.cpu())
+
+
+@pytest.mark.parametrize("p_format", [vc.VC_P_EXPCAST_E4M3, vc.VC_P_EXP_E4M3], ids=["expcast", "exp_then_cast"])
+@pytest.mark.parametrize("shape", [(1, 2, 128, 128, (2, 8, 8)), (1, 2, 129, 128, (1, 3, 43)), (2, 1, 300, 64, (3, 10, 10)),
+                                   (1, 2, 1024, 128, (4, 16, 16)), (1, 1, 2000, 128, (5, 20, 20))],
+                         ids=["n128", "n129", "n300_d64", "n1024", "n2000"])
+def test_8bit_kernel_variants_agree(shape, p_format):
+    """The two 8-bit kernels (two query tiles per CTA, pipelined; one tile per CTA, serial) run the
+    same arithmetic per key tile: each matches the oracle's emulation."""
+    B, H, N, d, grid = shape
+    w = vc_inputs.Workload("t", B, H, N, d, grid, (8,), 91, "gauss")
+    q, k, v = [t.cuda() for t in vc_inputs.make_qkv(w)]
+    perm = vc_inputs.random_perm(B, H, N, 5).cuda()
+    outs = {}
+    for variant in (0, 1):
+        p = Params.make(B, H, N, d, grid, bits=8, p_format=p_format, kernel_variant=variant)
+        quant, work = alloc_buffers(p)
+        o = torch.zeros(B, H, N, d, dtype=torch.bfloat16, device="cuda")
+        vc.vc_attn(p, q, k, v, perm, o, quant, work)
+        vc.vc_poll_status(work)
+        outs[variant] = o
+    vmax = float(v.float().abs().max())
+    p = Params.make(B, H, N, d, grid, bits=8, p_format=p_format)
+    pf = {vc.VC_P_EXPCAST_E4M3: OA.P_EXPCAST, vc.VC_P_EXP_E4M3: OA.P_EXP_E4M3}[p_format]
+    bundle, cfg = Hh.oracle_prep(p, q, k, v, perm, 0, 0)
+    ref = OA.emulate_head(bundle, cfg, p_format=pf)
+    for variant in (0, 1):
+        Hh.check_output(outs[variant][0, 0].float().cpu().numpy(), ref, vmax)
