@@ -132,7 +132,10 @@ def emulate_head(bundle, cfg, p_format=None, softmax_scale=None, beta=C.EXPCAST_
         p_format = p_format or P_EXPCAST
         sq, sk = bundle["q_scale"], bundle["k_scale"]
         scale_fn = lambda bq, bk: np.float32(np.float32(sq[bq] * sk[bk]) * sl)
-        q_deq, k_deq = C.e4m3_decode(bundle["q_codes"]), C.e4m3_decode(bundle["k_codes"])
+        if cfg.qk_format == "int8":
+            q_deq, k_deq = bundle["q_codes"].astype(np.float64), bundle["k_codes"].astype(np.float64)
+        else:
+            q_deq, k_deq = C.e4m3_decode(bundle["q_codes"]), C.e4m3_decode(bundle["k_codes"])
     elif cfg.bits == 4:
         p_format = p_format or P_NVFP4
         scale_fn = float(np.float32(np.float32(bundle["q_g"] * bundle["k_g"]) * sl))

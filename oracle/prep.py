@@ -41,6 +41,7 @@ class PrepConfig:
     v_smooth: bool = True
     rope_dims: tuple = None          # channels per axis, sum == d
     rope_theta: float = 10000.0
+    qk_format: str = "e4m3"          # 8-bit Q/K codes: "e4m3", or "int8" (the INT8 Q K^T of Fig. 3)
 
     def __post_init__(self):
         if self.rope_dims is None:
@@ -136,6 +137,26 @@ def quantize_e4m3_blocks(x):
     return codes, scale.astype(np.float32), deq
 
 
+def quantize_int8_blocks(x):
+    """INT8 Q/K codes (Fig. 3: INT8 Q K^T, FP8 softmax output, FP8 P V).  The paper gives no
+    scale convention; taken here: symmetric, per block of 128 rows s = amax/127 (1 if amax = 0),
+    code = round-to-nearest-even(x * (127/amax)) clamped to [-127, 127].
+
+    x: [n_pad, d] fp32.  Returns (codes int8, scales fp32 [n_blocks], dequantized fp64).
+    """
+    n_pad, d = x.shape
+    xb = x.reshape(n_pad // BLOCK, BLOCK * d)
+    amax = np.max(np.abs(xb), axis=1).astype(np.float32)
+    f127 = np.float32(127.0)
+    with np.errstate(divide="ignore", invalid="ignore"):
+        scale = np.where(amax > 0, (amax / f127).astype(np.float32), np.float32(1.0))
+        inv = np.where(amax > 0, (f127 / amax).astype(np.float32), np.float32(0.0))
+    y = (xb * inv[:, None]).astype(np.float32)
+    codes = np.clip(np.rint(y.astype(np.float64)), -127, 127).astype(np.int8).reshape(n_pad, d)   # rint: ties to even
+    deq = codes.astype(np.float64) * np.repeat(scale.astype(np.float64), BLOCK)[:, None]
+    return codes, scale.astype(np.float32), deq
+
+
 # ----------------------------------------------------------------------------- operands
 def prep_q(q, cfg, cos=None, sin=None):
     """Q: RoPE, Hadamard, pad, quantize (App. B).  q: [N, d] fp32 holding bf16 values."""
@@ -172,7 +193,7 @@ def prep_k(k, perm, cfg, cos=None, sin=None):
 def _quantize_qk(x, cfg, name):
     out = {name + "_pre": x}                   # the high-precision operand, for diagnostics
     if cfg.bits == 8:
-        codes, scale, deq = quantize_e4m3_blocks(x)
+        codes, scale, deq = quantize_int8_blocks(x) if cfg.qk_format == "int8" else quantize_e4m3_blocks(x)
         out.update({name + "_codes": codes, name + "_scale": scale, name + "_deq": deq})
     elif cfg.bits == 4:
         amax = np.float32(np.max(np.abs(x)))

@@ -261,3 +261,27 @@ def test_inputs_are_reproducible_and_shaped():
     assert sorted(p[0, 1].tolist()) == list(range(1024))
     pk, _ = vc_inputs.kmeans_perm(a[2][0, 0], k=8)
     assert sorted(pk.tolist()) == list(range(1024))
+
+
+def test_int8_qk_codes_follow_their_definition():
+    """INT8 Q/K quantizer (Fig. 3): symmetric per-128-row scale amax/127, round to nearest even,
+    checked element by element with Python's own round() on a block with exact ties."""
+    from oracle import prep as OP
+    rng = np.random.default_rng(3)
+    x = rng.normal(size=(256, 16)).astype(np.float32)
+    x[0, 0] = 4.0                                  # amax of block 0 -> code 127
+    x[0, 1] = np.float32(4.0 * 2.5 / 127.0)        # lands (nearly) on a tie
+    codes, scale, deq = OP.quantize_int8_blocks(x)
+    assert codes.dtype == np.int8 and codes.min() >= -127 and codes.max() == 127
+    for blk in range(2):
+        amax = float(np.abs(x[128 * blk:128 * (blk + 1)]).max())
+        assert scale[blk] == np.float32(amax) / np.float32(127.0)
+        inv = np.float32(127.0) / np.float32(amax)
+        for r in range(128 * blk, 128 * blk + 128, 17):
+            for c in range(16):
+                y = float(np.float32(x[r, c] * inv))
+                assert codes[r, c] == max(-127, min(127, round(y)))      # Python rounds ties to even
+    assert np.abs(deq - x).max() <= 0.5 * float(scale.max()) * (1 + 1e-6)
+    z = np.zeros((128, 8), dtype=np.float32)
+    c0, s0, _ = OP.quantize_int8_blocks(z)
+    assert s0[0] == 1.0 and not c0.any()
