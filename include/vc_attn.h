@@ -65,7 +65,12 @@ enum {
   VC_FLAG_HADAMARD = 2,
   VC_FLAG_K_SMOOTH = 4,
   VC_FLAG_V_SMOOTH = 8,
-  VC_FLAG_ALL = 15
+  VC_FLAG_ALL = 15,
+  /* variant switch, not part of VC_FLAG_ALL: 8-bit Q^ and K^ as INT8 (symmetric, scale amax/127
+   * per 128 rows) and Q^ K^T as an integer product -- the arrangement the paper runs on B200
+   * (Fig. 3); default is FP8 E4M3 for both products (the paper's B300 arrangement, Sec. 4.5).
+   * bits = 8 and the pipelined kernel only. */
+  VC_FLAG_INT8_QK = 16
 };
 
 typedef struct {
@@ -88,7 +93,8 @@ typedef struct {
 } vc_params;
 
 /* Device pointers into the quantized bundle written by vc_prep (N_pad = 128*ceil(N/128),
- * nb = N_pad/128, BH = B*H).  8 bits: codes are E4M3 bytes.  4 bits: codes are E2M1
+ * nb = N_pad/128, BH = B*H).  8 bits: codes are E4M3 bytes (Q^, K^: two's-complement INT8
+ * bytes under VC_FLAG_INT8_QK).  4 bits: codes are E2M1
  * nibbles, two per byte, the even index in the low nibble; micro are unsigned E4M3 bytes.
  *   q_codes [BH][N_pad][d]      (4 bits: [BH][N_pad][d/2])   rows in query order
  *   k_codes [BH][N_pad][d]      (4 bits: [BH][N_pad][d/2])   rows in permuted order

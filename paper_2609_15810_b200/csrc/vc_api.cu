@@ -32,7 +32,7 @@ vc_status resolve(const vc_params* p, Problem* out) {
   if (pr.bits == 8 && pr.p_format == VC_P_NVFP4) return VC_ERR_UNSUPPORTED;
   if (pr.bits == 4 && pr.p_format != VC_P_NVFP4) return VC_ERR_UNSUPPORTED;
   pr.flags = p->flags;
-  if (pr.flags & ~VC_FLAG_ALL) return VC_ERR_INVALID_ARG;
+  if (pr.flags & ~(VC_FLAG_ALL | VC_FLAG_INT8_QK)) return VC_ERR_INVALID_ARG;
   pr.softmax_scale = p->softmax_scale != 0.f ? p->softmax_scale : 1.0f / sqrtf((float)pr.d);
   if (!(pr.softmax_scale > 0.f)) return VC_ERR_INVALID_ARG;
   pr.beta = p->beta != 0.f ? p->beta : -0.35f;
@@ -59,6 +59,7 @@ vc_status resolve(const vc_params* p, Problem* out) {
   pr.heads_per_pass = p->heads_per_pass > 0 ? p->heads_per_pass : 0;
   pr.kernel_variant = p->kernel_variant;
   if (pr.kernel_variant < 0 || pr.kernel_variant > 1) return VC_ERR_INVALID_ARG;
+  if ((pr.flags & VC_FLAG_INT8_QK) && (pr.bits != 8 || pr.kernel_variant != 0)) return VC_ERR_INVALID_ARG;
   *out = pr;
   return VC_OK;
 }

@@ -233,7 +233,7 @@ attn_fwd_serial_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
 //                 row maximum moved, hands (r_hi, r_lo) alpha_j to the mean MMA, writes the output
 //
 // Tensor memory: S (128 columns) | A_0 (d + 16) | A_1 (d + 16).
-template <int D, bool EXPCAST>
+template <int D, bool EXPCAST, bool INT8>
 __global__ void __launch_bounds__(640, 1)
 attn_fwd_2q_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                    const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_mu,
@@ -312,7 +312,7 @@ attn_fwd_2q_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
       // one has been read into registers.  (The whole warp runs the loop so that descriptors stay
       // in uniform registers; one elected lane issues.  A separate warp issues the A_t updates, so
       // that neither kind of MMA ever waits behind a barrier that only the other kind needs.)
-      const uint32_t idesc_qk = idesc_e4m3(128, 128);
+      const uint32_t idesc_qk = INT8 ? idesc_s8(128, 128) : idesc_e4m3(128, 128);
       const uint64_t dq0 = smem_desc_kmajor(smem_u32(sQ), D), dq1 = smem_desc_kmajor(smem_u32(sQ + kQBytes), D);
       bool ok = warp_wait2(&sh->q_full, 0, sh, a.status, 20);
       for (int j = 0; ok && j < nb; ++j) {
@@ -329,7 +329,10 @@ attn_fwd_2q_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
             tc_fence_after();
             const uint64_t dq = t == 0 ? dq0 : dq1;
 #pragma unroll
-            for (int k = 0; k < D / 32; ++k) mma_f8_ss(tmem, dq + 2 * k, dk + 2 * k, idesc_qk, k > 0);
+            for (int k = 0; k < D / 32; ++k) {
+              if constexpr (INT8) mma_s8_ss(tmem, dq + 2 * k, dk + 2 * k, idesc_qk, k > 0);
+              else mma_f8_ss(tmem, dq + 2 * k, dk + 2 * k, idesc_qk, k > 0);
+            }
             mma_commit(&sh->s_full[t]);
           }
           __syncwarp();
@@ -398,6 +401,18 @@ attn_fwd_2q_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
       tmem_wait_ld();
       tc_fence_before();
       mbar_arrive(&sh->s_free[t]);                        // the score buffer may be overwritten
+      if constexpr (INT8) {
+        // INT32 scores -> FP32, exactly: |s| <= 127 * 127 * 128 < 2^22, so the bits of 1.5 * 2^23 + s
+        // are an integer add away, and subtracting the constant is exact.  (The two extra
+        // instructions per score are what the E4M3 score product saves on this GPU.)
+#pragma unroll
+        for (int i = 0; i < 32; ++i) {
+          s0[i] = __float_as_uint(__uint_as_float(s0[i] + 0x4B400000u) - 12582912.0f);
+          s1[i] = __float_as_uint(__uint_as_float(s1[i] + 0x4B400000u) - 12582912.0f);
+          s2[i] = __float_as_uint(__uint_as_float(s2[i] + 0x4B400000u) - 12582912.0f);
+          s3[i] = __float_as_uint(__uint_as_float(s3[i] + 0x4B400000u) - 12582912.0f);
+        }
+      }
       const int nv = a.N - j * 128;                       // >= 128 except on the ragged last tile
       if (nv < 128) {                                     // padded keys never win the maximum
 #pragma unroll
@@ -795,13 +810,18 @@ cudaError_t run8(const Problem& pr, const QuantLayout& ql, const WorkLayout& wl,
     const size_t stage = 2 * 128 * D + 2048 + ((D * 32 + 1023) / 1024) * 1024;
     const size_t smem2 = 1024 + 2 * 128 * D + 2 * 128 * 128 + 2 * 128 * 32 + kStages2 * stage + sizeof(FaSmem);
     const dim3 grid((pr.nb + 1) / 2, pr.BH);
+    const bool int8 = pr.flags & VC_FLAG_INT8_QK;
+#define VC_LAUNCH_2Q(EC, I8)                                                                                             \
+  {                                                                                                                      \
+    if ((e = cudaFuncSetAttribute(attn_fwd_2q_kernel<D, EC, I8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem2)) != cudaSuccess) return e; \
+    attn_fwd_2q_kernel<D, EC, I8><<<grid, 640, smem2, s>>>(tq, tk, tv, tmt, a);                                           \
+  }
     if (pr.p_format == VC_P_EXPCAST_E4M3) {
-      if ((e = cudaFuncSetAttribute(attn_fwd_2q_kernel<D, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem2)) != cudaSuccess) return e;
-      attn_fwd_2q_kernel<D, true><<<grid, 640, smem2, s>>>(tq, tk, tv, tmt, a);
+      if (int8) VC_LAUNCH_2Q(true, true) else VC_LAUNCH_2Q(true, false)
     } else {
-      if ((e = cudaFuncSetAttribute(attn_fwd_2q_kernel<D, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem2)) != cudaSuccess) return e;
-      attn_fwd_2q_kernel<D, false><<<grid, 640, smem2, s>>>(tq, tk, tv, tmt, a);
+      if (int8) VC_LAUNCH_2Q(false, true) else VC_LAUNCH_2Q(false, false)
     }
+#undef VC_LAUNCH_2Q
     count_launches(2);
     return cudaGetLastError();
   }

@@ -318,8 +318,11 @@ __device__ __forceinline__ void qk_row_item(const PrepArgs& a, const unsigned ch
   const size_t row_g = (size_t)bh * a.n_pad + (size_t)blk * kBlock + tid;
 
   if constexpr (STAGE == kStageQuant8) {
-    const float inv = amax > 0.f ? 448.0f / amax : 0.f;
-    if (tid == 0) (TENSOR == 0 ? a.q_scale : a.k_scale)[(size_t)bh * a.nb + blk] = amax > 0.f ? amax / 448.0f : 1.0f;
+    // E4M3 codes (top value 448), or INT8 codes (top value 127; the INT8 Q K^T of Fig. 3)
+    const bool int8 = a.flags & VC_FLAG_INT8_QK;
+    const float top = int8 ? 127.0f : 448.0f;
+    const float inv = amax > 0.f ? top / amax : 0.f;
+    if (tid == 0) (TENSOR == 0 ? a.q_scale : a.k_scale)[(size_t)bh * a.nb + blk] = amax > 0.f ? amax / top : 1.0f;
     // codes go to the swizzled output tile; the CTA copies it out with coalesced stores
     constexpr int CPR = D / 16;
     uint4* dst = reinterpret_cast<uint4*>(out_tile + tid * D);
@@ -330,9 +333,17 @@ __device__ __forceinline__ void qk_row_item(const PrepArgs& a, const unsigned ch
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
         const int c = 16 * i + 4 * j;
-        const unsigned int lo = __nv_cvt_float2_to_fp8x2(make_float2((x[c] * rs) * inv, (x[c + 1] * rs) * inv), __NV_SATFINITE, __NV_E4M3);
-        const unsigned int hi = __nv_cvt_float2_to_fp8x2(make_float2((x[c + 2] * rs) * inv, (x[c + 3] * rs) * inv), __NV_SATFINITE, __NV_E4M3);
-        w[j] = lo | (hi << 16);
+        if (int8) {
+          // |y| <= 127: adding 1.5 * 2^23 rounds y to the nearest even integer into the low mantissa
+          // bits, two's complement for negative values; the low bytes are the codes
+          const unsigned int r0 = __float_as_uint(((x[c] * rs) * inv) + 12582912.0f), r1 = __float_as_uint(((x[c + 1] * rs) * inv) + 12582912.0f);
+          const unsigned int r2 = __float_as_uint(((x[c + 2] * rs) * inv) + 12582912.0f), r3 = __float_as_uint(((x[c + 3] * rs) * inv) + 12582912.0f);
+          w[j] = __byte_perm(__byte_perm(r0, r1, 0x0040), __byte_perm(r2, r3, 0x0040), 0x5410);
+        } else {
+          const unsigned int lo = __nv_cvt_float2_to_fp8x2(make_float2((x[c] * rs) * inv, (x[c + 1] * rs) * inv), __NV_SATFINITE, __NV_E4M3);
+          const unsigned int hi = __nv_cvt_float2_to_fp8x2(make_float2((x[c + 2] * rs) * inv, (x[c + 3] * rs) * inv), __NV_SATFINITE, __NV_E4M3);
+          w[j] = lo | (hi << 16);
+        }
       }
       dst[i ^ sw] = make_uint4(w[0], w[1], w[2], w[3]);
     }

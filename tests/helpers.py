@@ -16,7 +16,8 @@ def oracle_cfg(p, **kw):
                          rope=bool(p.flags & vc.VC_FLAG_ROPE), hadamard=bool(p.flags & vc.VC_FLAG_HADAMARD),
                          k_smooth=bool(p.flags & vc.VC_FLAG_K_SMOOTH), v_smooth=bool(p.flags & vc.VC_FLAG_V_SMOOTH),
                          rope_dims=dims if any(dims) else None,
-                         rope_theta=p.rope_theta if p.rope_theta else 10000.0, **kw)
+                         rope_theta=p.rope_theta if p.rope_theta else 10000.0,
+                         qk_format="int8" if (p.flags & vc.VC_FLAG_INT8_QK) else "e4m3", **kw)
 
 
 def oracle_prep(p, q, k, v, perm, b, h):
@@ -41,6 +42,8 @@ def gpu_sections(p, quant):
         out["v_codes"] = s("v_codes").numpy().reshape(BH, d, n_pad).transpose(0, 2, 1)
         out["q_scale"] = s("q_scale", torch.float32).numpy().reshape(BH, nb)
         out["k_scale"] = s("k_scale", torch.float32).numpy().reshape(BH, nb)
+        if p.flags & vc.VC_FLAG_INT8_QK:
+            out["q_codes"], out["k_codes"] = out["q_codes"].view(np.int8), out["k_codes"].view(np.int8)
     else:
         out["q_codes"] = CMP.unpack_nibbles(s("q_codes").numpy().reshape(BH, n_pad, d // 2))
         out["k_codes"] = CMP.unpack_nibbles(s("k_codes").numpy().reshape(BH, n_pad, d // 2))
@@ -88,7 +91,11 @@ def check_prep_head(p, got, bh, ref, what=""):
         for t in ("q", "k", "v"):
             stats[t + "_micro"] = CMP.assert_codes_close(got[t + "_micro"][bh], ref[t + "_micro"], 7, what=what + t + "_micro")
     for t in ("q", "k", "v"):
-        if p.bits == 8:
+        if p.bits == 8 and t != "v" and (p.flags & vc.VC_FLAG_INT8_QK):
+            diff = np.abs(got[t + "_codes"][bh].astype(np.int32) - ref[t + "_codes"].astype(np.int32))
+            assert diff.max() <= 1 and float(np.mean(diff != 0)) <= 1e-3, what + " " + t + "_codes (int8)"
+            stats[t] = float(np.mean(diff != 0))
+        elif p.bits == 8:
             stats[t] = CMP.assert_codes_close(got[t + "_codes"][bh], ref[t + "_codes"], mag, what=what + " " + t + "_codes")
         else:
             # elements under a differing microscale are compared after decoding

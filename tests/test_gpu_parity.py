@@ -165,3 +165,32 @@ def test_bad_arguments_are_rejected_on_the_host():
         assert vc.vc_quant_bytes(pb) == 0
         with pytest.raises(vc.VcError):
             vc.vc_prep(pb, x, x, x, None, quant, work)
+
+
+@pytest.mark.parametrize("perm_kind", ["identity", "random"])
+@pytest.mark.parametrize("case", SMALL, ids=[c[0] for c in SMALL])
+def test_int8_qk_variant(case, perm_kind):
+    """VC_FLAG_INT8_QK (the INT8 Q K^T arrangement of Fig. 3): the INT8 codes and scales of vc_prep
+    against the oracle, then vc_attn end to end against the oracle's emulation of that variant."""
+    _, B, H, N, d, grid = case
+    q, k, v = _inputs(B, H, N, d, grid, seed=41)
+    perm = None if perm_kind == "identity" else vc_inputs.random_perm(B, H, N, 9).cuda()
+    p = Params.make(B, H, N, d, grid, bits=8, flags=vc.VC_FLAG_ALL | vc.VC_FLAG_INT8_QK)
+    quant, work = Hh.run_prep(p, q, k, v, perm)
+    got = Hh.gpu_sections(p, quant)
+    o = torch.empty(B, H, N, d, dtype=torch.bfloat16, device="cuda")
+    vc.vc_attn(p, q, k, v, perm, o, quant, work)
+    vc.vc_poll_status(work)
+    vmax = float(v.float().abs().max())
+    for b in range(B):
+        for h in range(H):
+            bundle, cfg = Hh.oracle_prep(p, q, k, v, perm, b, h)
+            assert bundle["q_codes"].dtype == np.int8
+            Hh.check_prep_head(p, got, b * H + h, bundle, what=f"int8 head {b},{h}")
+            Hh.check_output(o[b, h].float().cpu().numpy(), OA.emulate_head(bundle, cfg), vmax)
+
+
+def test_int8_qk_is_rejected_where_it_does_not_apply():
+    for kw in (dict(bits=4), dict(bits=8, kernel_variant=1)):
+        p = Params.make(1, 1, 256, 128, (4, 8, 8), flags=vc.VC_FLAG_ALL | vc.VC_FLAG_INT8_QK, **kw)
+        assert vc.vc_quant_bytes(p) == 0
