@@ -208,7 +208,7 @@ __device__ __forceinline__ void k_colsum_item(const PrepArgs& a, const unsigned 
 // Q / K, one row per thread.  All D channels of a row sit in the registers of one thread, so
 // the Hadamard rotation is D/2 * log2 D register butterflies with no shuffle, RoPE pairs and
 // NVFP4 groups are thread-local, and a row's codes leave as 16-byte stores.
-enum { kStageAmax = 1, kStageQuant8 = 2, kStageQuant4 = 3 };
+enum { kStageAmax = 1, kStageQuant8 = 2, kStageQuant4 = 3, kStageQuant8I = 4 };   // 8I: INT8 codes (VC_FLAG_INT8_QK)
 
 template <int D> struct RopeSplit;          // pair boundaries of the default channel split
 template <> struct RopeSplit<128> { static constexpr int p1 = 22, p2 = 43; };   // 44 / 42 / 42
@@ -317,9 +317,9 @@ __device__ __forceinline__ void qk_row_item(const PrepArgs& a, const unsigned ch
   }
   const size_t row_g = (size_t)bh * a.n_pad + (size_t)blk * kBlock + tid;
 
-  if constexpr (STAGE == kStageQuant8) {
+  if constexpr (STAGE == kStageQuant8 || STAGE == kStageQuant8I) {
     // E4M3 codes (top value 448), or INT8 codes (top value 127; the INT8 Q K^T of Fig. 3)
-    const bool int8 = a.flags & VC_FLAG_INT8_QK;
+    constexpr bool int8 = STAGE == kStageQuant8I;
     const float top = int8 ? 127.0f : 448.0f;
     const float inv = amax > 0.f ? top / amax : 0.f;
     if (tid == 0) (TENSOR == 0 ? a.q_scale : a.k_scale)[(size_t)bh * a.nb + blk] = amax > 0.f ? amax / top : 1.0f;
@@ -333,7 +333,7 @@ __device__ __forceinline__ void qk_row_item(const PrepArgs& a, const unsigned ch
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
         const int c = 16 * i + 4 * j;
-        if (int8) {
+        if constexpr (int8) {
           // |y| <= 127: adding 1.5 * 2^23 rounds y to the nearest even integer into the low mantissa
           // bits, two's complement for negative values; the low bytes are the codes
           const unsigned int r0 = __float_as_uint(((x[c] * rs) * inv) + 12582912.0f), r1 = __float_as_uint(((x[c + 1] * rs) * inv) + 12582912.0f);
@@ -775,6 +775,7 @@ cudaError_t run(const Problem& pr, PrepArgs a, const WorkLayout& wl, uint8_t* wo
   if ((e = allow_smem(prep_v_kernel<D, kVStats>, v_smem)) != cudaSuccess) return e;
   if ((e = allow_smem(prep_v_kernel<D, kVQuant>, v_smem)) != cudaSuccess) return e;
   if ((e = allow_smem(prep_qk_kernel<D, kQuant>, row_smem)) != cudaSuccess) return e;
+  if (BITS == 8 && (e = allow_smem(prep_qk_kernel<D, kStageQuant8I>, row_smem)) != cudaSuccess) return e;
   if (BITS == 4 && (e = allow_smem(prep_qk_kernel<D, kStageAmax>, row_smem)) != cudaSuccess) return e;
   if ((e = cudaMemsetAsync(work + wl.status, 0, 4, s)) != cudaSuccess) return e;
   if ((e = cudaMemsetAsync(work + wl.amax, 0, wl.amax_bytes, s)) != cudaSuccess) return e;
@@ -802,7 +803,10 @@ cudaError_t run(const Problem& pr, PrepArgs a, const WorkLayout& wl, uint8_t* wo
       prep_finalize_kernel<D, BITS><<<nh, 32, 0, s>>>(a, 1);
       count_launches(2);
     }
-    prep_qk_kernel<D, kQuant><<<persistent_grid(2 * per), kRowThreads, row_smem, s>>>(a, 2 * per, nh, 0);
+    if (BITS == 8 && (a.flags & VC_FLAG_INT8_QK))
+      prep_qk_kernel<D, kStageQuant8I><<<persistent_grid(2 * per), kRowThreads, row_smem, s>>>(a, 2 * per, nh, 0);
+    else
+      prep_qk_kernel<D, kQuant><<<persistent_grid(2 * per), kRowThreads, row_smem, s>>>(a, 2 * per, nh, 0);
     prep_v_kernel<D, kVQuant><<<persistent_grid(per), kThreads, v_smem, s>>>(a, per, nh);
     count_launches(2);
   }
