@@ -17,15 +17,29 @@ import helpers as Hh
 pytestmark = pytest.mark.gpu
 
 CASES = [("c2", 8, "kmeans"), ("c3", 8, "kmeans"), ("c3", 4, "random"), ("c4", 4, "kmeans"),
-         ("c5_d64_n4096", 8, "random"), ("c5_d64_n4096", 4, "random"), ("c5_d128_n16384", 8, "kmeans")]
+         ("c5_d64_n4096", 8, "random"), ("c5_d64_n4096", 4, "random"), ("c5_d128_n16384", 8, "kmeans"),
+         ("c3", 8, "group"),          # the permutation from vc_group, as bench.py runs it
+         ("c2", 8, "kmeans-int8"),    # the INT8 Q K^T arrangement
+         ("c4_2heads", 8, "random")]  # the longest sequence (929 key tiles, an odd count) at 8 bits
+
+vc_inputs.WORKLOADS.setdefault("c4_2heads", vc_inputs.Workload("c4_2heads", 1, 2, 118800, 128, (33, 45, 80), (8,), 1044, "field", True))
 
 
-@pytest.mark.parametrize("name,bits,perm_kind", CASES, ids=[f"{c[0]}-{c[1]}bit" for c in CASES])
+@pytest.mark.parametrize("name,bits,perm_kind", CASES, ids=[f"{c[0]}-{c[1]}bit-{c[2]}" for c in CASES])
 def test_fullsize_sampled_parity(name, bits, perm_kind):
     w = vc_inputs.WORKLOADS[name]
     q, k, v = vc_inputs.make_qkv(w, device="cuda")
-    perm = vc_inputs.kmeans_perm_all(v, iters=2) if perm_kind == "kmeans" else vc_inputs.random_perm(w.B, w.H, w.N, w.seed, device="cuda")
-    p = Params.make(w.B, w.H, w.N, w.d, w.grid, bits=bits)
+    flags = vc.VC_FLAG_ALL | (vc.VC_FLAG_INT8_QK if perm_kind.endswith("int8") else 0)
+    p = Params.make(w.B, w.H, w.N, w.d, w.grid, bits=bits, flags=flags)
+    if perm_kind == "group":
+        gwork = torch.empty(vc.vc_group_workspace_bytes(p), dtype=torch.uint8, device="cuda")
+        cent = torch.zeros(w.B, w.H, 64, w.d, dtype=torch.float32, device="cuda")
+        perm = torch.empty(w.B, w.H, w.N, dtype=torch.int32, device="cuda")
+        vc.vc_group(p, v, 64, 2, False, cent, perm, gwork)
+    elif perm_kind.startswith("kmeans"):
+        perm = vc_inputs.kmeans_perm_all(v, iters=2)
+    else:
+        perm = vc_inputs.random_perm(w.B, w.H, w.N, w.seed, device="cuda")
     quant, work = alloc_buffers(p)
     o = torch.empty(w.B, w.H, w.N, w.d, dtype=torch.bfloat16, device="cuda")
     vc.vc_attn(p, q, k, v, perm, o, quant, work)
