@@ -7,6 +7,7 @@ A plain, slow NumPy restatement of what the path computes, written from the pape
 * ``attention``  exact fp64 attention and the emulated low-bit recurrence
                  (Eq. 1, Eq. 6, Eq. 7)
 * ``grouping``   the value-guided permutation (Sec. 3.2): k-means labels, stable argsort
+* ``analysis``   analogues of the paper's value-side analysis (token-order table, Eq. 2, Eq. 5)
 
 Only the tests, ``__graft_entry__.smoke()`` and the ``cpu_baseline`` / ``--impl reference``
 legs of ``bench.py`` may import this package.  It shares no code with the CUDA path and
