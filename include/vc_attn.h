@@ -170,6 +170,18 @@ size_t vc_group_workspace_bytes(const vc_params *p);
 vc_status vc_group(const vc_params *p, const void *v, int32_t k, int32_t iters, int32_t warm_start,
                    float *centroids, int32_t *perm, void *workspace, void *stream);
 
+/* Amortized grouping schedule (Sec. 3.4 "Amortized grouping schedule", App. A "Grouping
+ * schedule"): host logic keyed on the denoising step index alone.  Value grouping and demeaning
+ * run on the first ceil(n_steps / 4) steps; inside that window the permutation is recomputed on
+ * every `reuse`-th step (the paper uses 4) and reused in between; the remaining steps run the
+ * plain low-bit kernel on the permutation the window left behind.
+ *   VC_GROUP_RECOMPUTE  call vc_group (warm-started after step 0), then vc_attn with V smoothing
+ *   VC_GROUP_REUSE      vc_attn with V smoothing and the permutation at hand
+ *   VC_GROUP_FROZEN     past the window: the permutation at hand, flags without VC_FLAG_V_SMOOTH
+ * Returns -1 for step < 0, step >= n_steps or reuse < 1. */
+enum { VC_GROUP_RECOMPUTE = 0, VC_GROUP_REUSE = 1, VC_GROUP_FROZEN = 2 };
+int32_t vc_group_schedule(int32_t step, int32_t n_steps, int32_t reuse);
+
 /* vc_prep without a workspace argument and without any allocation.  (The paper has no
  * counterpart: this entry point exists for the sake of its callers, not of the method.)
  *

@@ -82,6 +82,8 @@ def load_library():
     lib.vc_group_workspace_bytes.argtypes = [P]
     lib.vc_group.restype = ctypes.c_int
     lib.vc_group.argtypes = [P, vp, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, vp, i32p, vp, vp]
+    lib.vc_group_schedule.restype = ctypes.c_int32
+    lib.vc_group_schedule.argtypes = [ctypes.c_int32, ctypes.c_int32, ctypes.c_int32]
     lib.vc_quant_view.restype = ctypes.c_int
     lib.vc_quant_view.argtypes = [P, vp, ctypes.POINTER(QuantView)]
     lib.vc_poll_status.restype = ctypes.c_int
@@ -160,6 +162,14 @@ def vc_group(p, v, k, iters, warm_start, centroids, perm, workspace):
     """k-means on the value tokens -> perm = stable argsort of the labels (centroids in/out)."""
     _check(load_library().vc_group(ctypes.byref(p), _ptr(v), int(k), int(iters), int(bool(warm_start)), _ptr(centroids),
                                    _ptr(perm), _ptr(workspace), _stream()), "vc_group")
+
+
+VC_GROUP_RECOMPUTE, VC_GROUP_REUSE, VC_GROUP_FROZEN = 0, 1, 2
+
+
+def vc_group_schedule(step, n_steps, reuse=4):
+    """What the step-indexed grouping schedule asks for at denoising step `step` of `n_steps`."""
+    return int(load_library().vc_group_schedule(int(step), int(n_steps), int(reuse)))
 
 
 def vc_quant_view(p, quant):

@@ -288,6 +288,13 @@ vc_status vc_poll_status(void* workspace, void* stream) {
   return VC_OK;
 }
 
+int32_t vc_group_schedule(int32_t step, int32_t n_steps, int32_t reuse) {
+  if (step < 0 || step >= n_steps || reuse < 1) return -1;
+  const int32_t window = (n_steps + 3) / 4;          // ceil(n / 4)
+  if (step >= window) return VC_GROUP_FROZEN;
+  return step % reuse == 0 ? VC_GROUP_RECOMPUTE : VC_GROUP_REUSE;
+}
+
 uint64_t vc_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 
 const char* vc_status_string(vc_status s) {

@@ -39,3 +39,17 @@ def test_sizes_and_argument_validation_without_a_gpu():
     assert vc.vc_status_string(0) == "ok" and "timed out" in vc.vc_status_string(5)
     assert ctypes.sizeof(Params) == 96
     assert vc.vc_launch_count() == 0
+
+
+def test_grouping_schedule_matches_the_papers_worked_examples():
+    """vc_group_schedule against the step lists the paper prints (tests/golden/grouping_schedule.txt)."""
+    for line in open(os.path.join(ROOT, "tests", "golden", "grouping_schedule.txt")):
+        if line.startswith("#") or not line.strip():
+            continue
+        n, steps, window = line.split()
+        n, window = int(n), int(window)
+        want = [int(s) for s in steps.split(",")]
+        kinds = [vc.vc_group_schedule(s, n, 4) for s in range(n)]
+        assert [s for s in range(n) if kinds[s] == vc.VC_GROUP_RECOMPUTE] == want
+        assert all(k == vc.VC_GROUP_FROZEN for k in kinds[window:]) and vc.VC_GROUP_FROZEN not in kinds[:window]
+    assert vc.vc_group_schedule(-1, 8, 4) == -1 and vc.vc_group_schedule(8, 8, 4) == -1 and vc.vc_group_schedule(0, 8, 0) == -1
