@@ -178,6 +178,9 @@ def main():
                          "region and reused in between; kmeans: the harness's torch k-means, computed once")
     ap.add_argument("--heads-per-pass", type=int, default=0)
     ap.add_argument("--variant", type=int, default=0, help="attention kernel (vc_params.kernel_variant)")
+    ap.add_argument("--p-format", default="default", choices=["default", "expcast", "exp", "exp_poly", "exp_mix"],
+                    help="8-bit probability format: ExpCast-FP8 (Eq. 7, the default) or exponentiate-then-cast with 2^u on the "
+                         "special-function unit (exp), on the FMA pipe (exp_poly), or one score in four there (exp_mix)")
     ap.add_argument("--int8-qk", action="store_true", help="8-bit Q/K as INT8 and an integer score product (Fig. 3)")
     ap.add_argument("--ref-rows", type=int, default=1024)
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -216,7 +219,8 @@ def main():
     else:
         q, k, v = vc_inputs.make_qkv(w, device=dev)
     p = Params.make(w.B, w.H, w.N, w.d, w.grid, bits=args.bits, heads_per_pass=args.heads_per_pass,
-                    kernel_variant=args.variant, flags=15 | (16 if args.int8_qk else 0))
+                    kernel_variant=args.variant, flags=15 | (16 if args.int8_qk else 0),
+                    p_format={"default": 0, "expcast": 1, "exp": 2, "exp_poly": 4, "exp_mix": 5}[args.p_format])
     group_k, group_every = 64, 4
     if args.perm == "group":
         gwork = torch.empty(vc.vc_group_workspace_bytes(p), dtype=torch.uint8, device=dev)
@@ -320,7 +324,7 @@ def main():
         "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": ("int8 QK / e4m3 PV" if args.int8_qk else "e4m3") if args.bits == 8 else "nvfp4", "data": "synthetic",
         "config": {"workload": w.name, "B": w.B, "H": w.H, "N": w.N, "d": w.d, "grid": list(w.grid),
-                   "bits": args.bits, "perm": args.perm, "data": args.data, "l2": "inputs larger than L2 (Q+K+V = %.0f MB)" % (3 * q.numel() * 2 / 1e6),
+                   "bits": args.bits, "p_format": args.p_format, "perm": args.perm, "data": args.data, "l2": "inputs larger than L2 (Q+K+V = %.0f MB)" % (3 * q.numel() * 2 / 1e6),
                    "step": "vc_prep + vc_attn_fwd" + (" (+ vc_group every 4th step)" if args.perm == "group" else "")},
         "clocks": clocks, "gpu_launches": launches, "e2e": e2e,
         "roofline": {"bound": "tensor", "kernel": "vc_attn_fwd", "achieved": achieved, "peak": peak, "unit": UNIT,

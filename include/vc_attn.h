@@ -56,7 +56,14 @@ enum {
   VC_P_DEFAULT = 0,         /* ExpCast-FP8 at 8 bits, NVFP4 at 4 bits                */
   VC_P_EXPCAST_E4M3 = 1,    /* Eq. 7: one FMA, the byte viewed as E4M3               */
   VC_P_EXP_E4M3 = 2,        /* exponentiate, then cast to E4M3 (Fig. 4a upper box)   */
-  VC_P_NVFP4 = 3            /* E2M1 under a per-16-key E4M3 microscale               */
+  VC_P_NVFP4 = 3,           /* E2M1 under a per-16-key E4M3 microscale               */
+  /* the same result as VC_P_EXP_E4M3 up to the polynomial's error (relative 3.7e-6, so a code
+   * differs from the exactly exponentiated one for about one score in 10^4): 2^u evaluated on
+   * the FMA pipe by a degree-4 polynomial instead of the special-function unit, for every
+   * score (POLY) or for one score in four (MIX).  They exist to measure where the exponential
+   * belongs on this GPU (Sec. 3.3); kernel_variant 1 computes them like VC_P_EXP_E4M3.        */
+  VC_P_EXP_POLY_E4M3 = 4,
+  VC_P_EXP_MIX_E4M3 = 5
 };
 
 /* stages of the chain that can be switched off (all on = the paper's method) */

@@ -13,6 +13,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _LIB_PATH = os.path.join(_HERE, "libvc.so")
 
 VC_P_DEFAULT, VC_P_EXPCAST_E4M3, VC_P_EXP_E4M3, VC_P_NVFP4 = 0, 1, 2, 3
+VC_P_EXP_POLY_E4M3, VC_P_EXP_MIX_E4M3 = 4, 5
 VC_FLAG_ROPE, VC_FLAG_HADAMARD, VC_FLAG_K_SMOOTH, VC_FLAG_V_SMOOTH, VC_FLAG_ALL = 1, 2, 4, 8, 15
 VC_FLAG_INT8_QK = 16
 

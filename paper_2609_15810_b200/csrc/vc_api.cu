@@ -28,8 +28,9 @@ vc_status resolve(const vc_params* p, Problem* out) {
   if (pr.bits != 8 && pr.bits != 4) return VC_ERR_INVALID_ARG;
   pr.p_format = p->p_format;
   if (pr.p_format == VC_P_DEFAULT) pr.p_format = pr.bits == 8 ? VC_P_EXPCAST_E4M3 : VC_P_NVFP4;
-  if (pr.p_format < VC_P_EXPCAST_E4M3 || pr.p_format > VC_P_NVFP4) return VC_ERR_INVALID_ARG;
+  if (pr.p_format < VC_P_EXPCAST_E4M3 || pr.p_format > VC_P_EXP_MIX_E4M3) return VC_ERR_INVALID_ARG;
   if (pr.bits == 8 && pr.p_format == VC_P_NVFP4) return VC_ERR_UNSUPPORTED;
+  if (pr.p_format > VC_P_NVFP4 && (p->flags & VC_FLAG_INT8_QK)) return VC_ERR_UNSUPPORTED;
   if (pr.bits == 4 && pr.p_format != VC_P_NVFP4) return VC_ERR_UNSUPPORTED;
   pr.flags = p->flags;
   if (pr.flags & ~(VC_FLAG_ALL | VC_FLAG_INT8_QK)) return VC_ERR_INVALID_ARG;

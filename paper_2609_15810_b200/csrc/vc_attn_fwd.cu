@@ -233,7 +233,25 @@ attn_fwd_serial_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
 //                 row maximum moved, hands (r_hi, r_lo) alpha_j to the mean MMA, writes the output
 //
 // Tensor memory: S (128 columns) | A_0 (d + 16) | A_1 (d + 16).
-template <int D, bool EXPCAST, bool INT8>
+// P formats of the two-query-tile kernel
+constexpr int kPfExpCast = 0, kPfExp = 1, kPfExpPoly = 2, kPfExpMix = 3;
+
+// 2^x for x <= 8 without the special-function unit: x = n + f with n the nearest integer
+// (1.5 * 2^23 trick) and |f| <= 1/2, 2^f by a degree-4 polynomial (relative error 3.7e-6, a
+// 1/17000 of an E4M3 step), 2^n by an add into the exponent field.  Inputs below -24 give the
+// value at -24, which rounds to code 0 like the exact result.
+__device__ __forceinline__ float exp2_poly(float x) {
+  x = fmaxf(x, -24.0f);
+  const float t = x + 12582912.0f;
+  const float f = x - (t - 12582912.0f);
+  float p = fmaf(0.009676037356257439f, f, 0.05592203512787819f);
+  p = fmaf(p, f, 0.2402210682630539f);
+  p = fmaf(p, f, 0.6931210160255432f);
+  p = fmaf(p, f, 1.0000001192092896f);
+  return __uint_as_float(__float_as_uint(p) + (__float_as_uint(t) << 23));
+}
+
+template <int D, int PF, bool INT8>
 __global__ void __launch_bounds__(640, 1)
 attn_fwd_2q_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                    const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_mu,
@@ -452,7 +470,7 @@ attn_fwd_2q_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
 
       const float fa = cs * 0.0625f, fb = (a.code_off - 8.0f * m_new) * 0.0078125f, nm = 8.0f - m_new;
       auto code4 = [&](const uint32_t (&sv)[32], int w) -> uint32_t {
-        if constexpr (EXPCAST) {
+        if constexpr (PF == kPfExpCast) {
           // Eq. 7 in two FMAs: t = sat((8 u + 120 + beta) / 128) clips to [0, 1], then
           // t * 128 + 1.5 * 2^23 rounds to the nearest even integer in the low mantissa bits.
           const uint32_t r0 = __float_as_uint(fmaf(fma_sat(__uint_as_float(sv[4 * w]), fa, fb), 128.0f, 12582912.0f));
@@ -461,9 +479,18 @@ attn_fwd_2q_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
           const uint32_t r3 = __float_as_uint(fmaf(fma_sat(__uint_as_float(sv[4 * w + 3]), fa, fb), 128.0f, 12582912.0f));
           return __byte_perm(__byte_perm(r0, r1, 0x0040), __byte_perm(r2, r3, 0x0040), 0x5410);
         } else {
-          // exponentiate, then cast (Fig. 4a upper box)
-          const float p0 = exp2f(fmaf(__uint_as_float(sv[4 * w]), cs, nm)), p1 = exp2f(fmaf(__uint_as_float(sv[4 * w + 1]), cs, nm));
-          const float p2 = exp2f(fmaf(__uint_as_float(sv[4 * w + 2]), cs, nm)), p3 = exp2f(fmaf(__uint_as_float(sv[4 * w + 3]), cs, nm));
+          // exponentiate, then cast (Fig. 4a upper box): on the special-function unit, on the
+          // FMA pipe by a polynomial, or three and one per word
+          const float x0 = fmaf(__uint_as_float(sv[4 * w]), cs, nm), x1 = fmaf(__uint_as_float(sv[4 * w + 1]), cs, nm);
+          const float x2 = fmaf(__uint_as_float(sv[4 * w + 2]), cs, nm), x3 = fmaf(__uint_as_float(sv[4 * w + 3]), cs, nm);
+          float p0, p1, p2, p3;
+          if constexpr (PF == kPfExp) {
+            p0 = ex2_approx(x0); p1 = ex2_approx(x1); p2 = ex2_approx(x2); p3 = ex2_approx(x3);
+          } else if constexpr (PF == kPfExpPoly) {
+            p0 = exp2_poly(x0); p1 = exp2_poly(x1); p2 = exp2_poly(x2); p3 = exp2_poly(x3);
+          } else {
+            p0 = ex2_approx(x0); p1 = ex2_approx(x1); p2 = ex2_approx(x2); p3 = exp2_poly(x3);
+          }
           const uint32_t lo = __nv_cvt_float2_to_fp8x2(make_float2(p0, p1), __NV_SATFINITE, __NV_E4M3);
           const uint32_t hi = __nv_cvt_float2_to_fp8x2(make_float2(p2, p3), __NV_SATFINITE, __NV_E4M3);
           return lo | (hi << 16);
@@ -816,10 +843,18 @@ cudaError_t run8(const Problem& pr, const QuantLayout& ql, const WorkLayout& wl,
     if ((e = cudaFuncSetAttribute(attn_fwd_2q_kernel<D, EC, I8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem2)) != cudaSuccess) return e; \
     attn_fwd_2q_kernel<D, EC, I8><<<grid, 640, smem2, s>>>(tq, tk, tv, tmt, a);                                           \
   }
-    if (pr.p_format == VC_P_EXPCAST_E4M3) {
-      if (int8) VC_LAUNCH_2Q(true, true) else VC_LAUNCH_2Q(true, false)
+    const int pf = pr.p_format == VC_P_EXPCAST_E4M3 ? kPfExpCast
+                   : pr.p_format == VC_P_EXP_E4M3   ? kPfExp
+                   : pr.p_format == VC_P_EXP_POLY_E4M3 ? kPfExpPoly : kPfExpMix;
+    if (int8) {
+      if (pf == kPfExpCast) VC_LAUNCH_2Q(kPfExpCast, true)
+      else if (pf == kPfExp) VC_LAUNCH_2Q(kPfExp, true)
+      else return cudaErrorNotSupported;
     } else {
-      if (int8) VC_LAUNCH_2Q(false, true) else VC_LAUNCH_2Q(false, false)
+      if (pf == kPfExpCast) VC_LAUNCH_2Q(kPfExpCast, false)
+      else if (pf == kPfExp) VC_LAUNCH_2Q(kPfExp, false)
+      else if (pf == kPfExpPoly) VC_LAUNCH_2Q(kPfExpPoly, false)
+      else VC_LAUNCH_2Q(kPfExpMix, false)
     }
 #undef VC_LAUNCH_2Q
     count_launches(2);

@@ -74,10 +74,12 @@ def test_prep_strided_inputs_and_head_groups():
     assert torch.equal(quant, quant0)
 
 
-@pytest.mark.parametrize("p_format", [vc.VC_P_EXPCAST_E4M3, vc.VC_P_EXP_E4M3])
+@pytest.mark.parametrize("p_format", [vc.VC_P_EXPCAST_E4M3, vc.VC_P_EXP_E4M3, vc.VC_P_EXP_POLY_E4M3, vc.VC_P_EXP_MIX_E4M3],
+                         ids=["expcast", "exp_sfu", "exp_poly", "exp_mix"])
 @pytest.mark.parametrize("case", SMALL, ids=[c[0] for c in SMALL])
 def test_attn_fwd_on_oracle_bundle(case, p_format):
-    """Stage 2: isolates the attention kernel from code flips in prep."""
+    """Stage 2: isolates the attention kernel from code flips in prep.  The polynomial forms of
+    exponentiate-then-cast are held to the same oracle result as the special-function one."""
     _, B, H, N, d, grid = case
     q, k, v = _inputs(B, H, N, d, grid, seed=21)
     perm = vc_inputs.random_perm(B, H, N, 6).cuda()
