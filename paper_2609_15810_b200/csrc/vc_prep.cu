@@ -216,10 +216,12 @@ template <> struct RopeSplit<64> { static constexpr int p1 = 12, p2 = 22; };    
 
 // Reads the thread's row out of the stage, releases the stage, then transforms the row.
 // `red` is [2][4] floats and `kmean_s` [D] floats of compute-warp scratch.
-template <int D, int TENSOR /*0 = Q, 1 = K*/, int STAGE>
-__device__ __forceinline__ void qk_row_item(const PrepArgs& a, const unsigned char* stage, unsigned char* out_tile, float* red,
-                                            float* kmean_s, const float2* tab, int bh, int blk, int iter, bool new_head,
-                                            int src_row) {
+// Q and K run through one copy of the row body (TENSOR is a run-time argument): the unrolled body
+// is tens of KB of code, and two copies of it thrash the instruction cache.
+template <int D, int STAGE>
+__device__ __forceinline__ void qk_row_item(const PrepArgs& a, const int TENSOR /*0 = Q, 1 = K*/, const unsigned char* stage,
+                                            unsigned char* out_tile, float* red, float* kmean_s, const float2* tab, int bh,
+                                            int blk, int iter, bool new_head, int src_row) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const bool do_rope = a.flags & VC_FLAG_ROPE;
   const bool do_had = a.flags & VC_FLAG_HADAMARD;
@@ -726,12 +728,9 @@ __global__ void __launch_bounds__(kRowThreads, 2) prep_qk_kernel(const PrepArgs 
     const Item w = decode_item(item, a.nb, nh, a.bh0);
     const unsigned char* stage = smem + (i & 1) * Geo<D>::stage_bytes;
     const int s0 = src_ring[(i % 3) * kBlock + tid];
-    if (w.z + z0 == 0) {
-      qk_row_item<D, 0, STAGE>(a, stage, out_tile, red, kmean_s, tab, w.bh, w.blk, i, false, s0);
-    } else {
-      qk_row_item<D, 1, STAGE>(a, stage, out_tile, red, kmean_s, tab, w.bh, w.blk, i, w.bh != last_bh, s0);
-      last_bh = w.bh;
-    }
+    const int tensor = w.z + z0;
+    qk_row_item<D, STAGE>(a, tensor, stage, out_tile, red, kmean_s, tab, w.bh, w.blk, i, tensor == 1 && w.bh != last_bh, s0);
+    if (tensor == 1) last_bh = w.bh;
     if constexpr (STAGE != kStageAmax) {
       __syncthreads();                        // the code tile is complete
       uint8_t* gdst = (w.z + z0 == 0 ? a.q_codes : a.k_codes) + ((size_t)w.bh * a.n_pad + (size_t)w.blk * kBlock) * kRowBytes;
