@@ -155,3 +155,37 @@ def nvfp4_quantize_groups(x, outer_scale=np.float32(1.0)):
     codes = np.where(sdec[..., None] > 0, codes, np.uint8(0)).astype(np.uint8)
     deq = e2m1_decode(codes) * sdec[..., None].astype(np.float64)
     return codes.reshape(x.shape), micro, deq.reshape(x.shape)
+
+
+# ----------------------------------------------------------------------------- E2M1 under UE8M0 (MXFP4)
+def ue8m0_decode(code):
+    """Unsigned 8-bit exponent code -> 2^(code - 127) as float64 (code 255 is not produced here)."""
+    return np.exp2(np.asarray(code).astype(np.float64) - 127.0)
+
+
+def mxfp4_quantize_groups(x):
+    """Quantize the LAST axis of x (fp32, length divisible by 32) in groups of 32: E2M1
+    elements under a power-of-two scale per group (the format of the FP8 x FP4 block-scaled
+    product, used by the hybrid 4-bit arrangement: ExpCast-FP8 P times 4-bit values).
+
+    The paper gives no rule for the exponent; taken here: the smallest power of two that maps
+    the group maximum into the E2M1 range without clipping.  y = max|x| / 6 as ONE IEEE fp32
+    division; e = exponent(y), plus one unless y is a power of two; scale = 2^e (stored as
+    e + 127, clamped to [0, 254]); element = E2M1(x / 2^e), exact scaling, one rounding.  A
+    group of zeros stores code 0 and zero elements.  Returns (codes uint8 0..15, scale codes
+    uint8, deq fp64 = dec(code) * 2^e).
+    """
+    x = np.asarray(x, dtype=np.float32)
+    g = x.reshape(x.shape[:-1] + (x.shape[-1] // 32, 32))
+    amax = np.max(np.abs(g), axis=-1).astype(np.float32)
+    y = (amax / np.float32(6.0)).astype(np.float32)
+    bits = y.view(np.uint32).astype(np.int64)
+    e = ((bits >> 23) & 0xFF) - 127 + ((bits & 0x7FFFFF) != 0).astype(np.int64)
+    code = np.clip(e + 127, 0, 254)
+    code = np.where(amax > 0, code, 0).astype(np.uint8)
+    scale = ue8m0_decode(code)
+    yv = (g.astype(np.float64) / scale[..., None]).astype(np.float32)       # exact: power of two
+    codes = e2m1_encode(yv)
+    codes = np.where(amax[..., None] > 0, codes, np.uint8(0)).astype(np.uint8)
+    deq = e2m1_decode(codes) * scale[..., None]
+    return codes.reshape(x.shape), code, deq.reshape(x.shape)

@@ -42,6 +42,9 @@ class PrepConfig:
     rope_dims: tuple = None          # channels per axis, sum == d
     rope_theta: float = 10000.0
     qk_format: str = "e4m3"          # 8-bit Q/K codes: "e4m3", or "int8" (the INT8 Q K^T of Fig. 3)
+    v_format: str = "nvfp4"          # 4-bit V codes: "nvfp4" (E4M3 factor per 16 tokens), or "mxfp4"
+                                     # (power-of-two factor per 32 tokens: the hybrid arrangement,
+                                     # ExpCast-FP8 P times 4-bit values)
 
     def __post_init__(self):
         if self.rope_dims is None:
@@ -238,9 +241,11 @@ def prep_v(v, perm, cfg):
                     "v_deq": C.e4m3_decode(codes)})                # in code units; x s_V in the epilogue
     elif cfg.bits == 4:
         # groups of 16 consecutive permuted tokens per channel: quantize the transpose
-        codes_t, micro_t, deq_t = C.nvfp4_quantize_groups(np.ascontiguousarray(r.T))
+        # (nvfp4), or of 32 under a power-of-two factor (mxfp4)
+        quant = C.mxfp4_quantize_groups if cfg.v_format == "mxfp4" else C.nvfp4_quantize_groups
+        codes_t, micro_t, deq_t = quant(np.ascontiguousarray(r.T))
         out.update({"v_codes": np.ascontiguousarray(codes_t.T),    # [n_pad, d]
-                    "v_micro": np.ascontiguousarray(micro_t.T),    # [n_pad/16, d]
+                    "v_micro": np.ascontiguousarray(micro_t.T),    # [n_pad/16, d] (mxfp4: [n_pad/32, d])
                     "v_means": C.bf16_round(mu),                   # unscaled  (App. B)
                     "v_scale": np.ones(d, dtype=np.float32),
                     "v_deq": np.ascontiguousarray(deq_t.T)})

@@ -110,6 +110,35 @@ def test_nvfp4_group_quantizer_brute_force():
     assert not z.any() and not mz.any() and not dz.any()
 
 
+def test_mxfp4_group_quantizer_brute_force():
+    """E2M1 under a power-of-two factor per 32: the factor is the smallest power of two that
+    leaves the group maximum inside the E2M1 range (checked by exhaustive search over the
+    exponent), elements are the nearest grid values, and a power-of-two input is reproduced."""
+    rng = np.random.default_rng(5)
+    x = (rng.standard_normal((48, 64)) * rng.uniform(1e-3, 50, (48, 1))).astype(np.float32)
+    x[0, :32] = 0.0
+    x[1, :32] = 4.0 * np.array([0, 0.5, 1, 1.5, 2, 3, 4, 6] * 4, np.float32) * rng.choice([-1.0, 1.0], 32)   # grid values x 2^2
+    x[2, :32] = np.float32(6.0000005) * 4                                         # just above: next power
+    codes, sc, deq = C.mxfp4_quantize_groups(x)
+    grid = np.array([0, 0.5, 1, 1.5, 2, 3, 4, 6])
+    for r in range(x.shape[0]):
+        for g in range(2):
+            seg = x[r, 32 * g:32 * g + 32].astype(np.float64)
+            amax = np.abs(seg).max()
+            if amax == 0:
+                assert sc[r, g] == 0 and not codes[r, 32 * g:32 * g + 32].any()
+                continue
+            e = int(sc[r, g]) - 127
+            es = [k for k in range(-40, 40) if amax <= 6.0 * 2.0 ** k]
+            assert e == min(es)                                   # no clipping, and no smaller factor does that
+            y = np.abs(seg) / 2.0 ** e
+            best = np.abs(y[:, None] - grid[None, :]).min(axis=1)
+            got = np.abs(np.abs(deq[r, 32 * g:32 * g + 32]) / 2.0 ** e - y)
+            assert np.array_equal(got, best)                      # exact scaling: the nearest value, no slack
+    assert np.array_equal(deq[1, :32], x[1, :32].astype(np.float64))
+    assert sc[2, 0] == 127 + 3 and C.ue8m0_decode(sc[2, 0]) == 8.0
+
+
 # ----------------------------------------------------------------------------- bf16
 def test_bf16_round_matches_library_cast():
     rng = np.random.default_rng(11)

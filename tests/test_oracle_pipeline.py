@@ -211,6 +211,27 @@ def test_quantized_pipeline_tracks_exact_attention(bits, cos_min, tol):
     assert np.abs(o - ref).max() < tol * np.abs(v).max()
 
 
+def test_hybrid_4bit_arrangement_tracks_exact_attention():
+    """ExpCast-FP8 P over 4-bit Q, K and values under power-of-two factors per 32 tokens: the
+    value codes decode to the residual within half a grid step of their group, and the output
+    is closer to exact attention than with the NVFP4 probability."""
+    w = vc_inputs.WORKLOADS["c1"]
+    q, k, v = [t[0, 0].float().numpy() for t in vc_inputs.make_qkv(w, heads=[0])]
+    rows = np.arange(0, w.N, 7)
+    cfg = P.PrepConfig(N=w.N, d=w.d, grid=w.grid, bits=4, v_format="mxfp4")
+    b = P.prep_head(q, k, v, None, cfg)
+    assert b["v_micro"].shape == (cfg.n_pad // 32, w.d)
+    step = np.repeat(np.exp2(b["v_micro"].astype(np.float64) - 127.0), 32, axis=0)   # factor per element
+    assert np.all(np.abs(b["v_deq"] - b["v_pre"]) <= step + 1e-12)                    # widest E2M1 gap is 2: half of it
+    ref = A.reference_head(q, k, v, cfg, rows=rows)
+    o = A.emulate_head(b, cfg, rows=rows, p_format=A.P_EXPCAST).astype(np.float64)
+    cos = (o * ref).sum() / np.linalg.norm(o) / np.linalg.norm(ref)
+    assert cos > 0.995 and np.abs(o - ref).max() < 8e-2 * np.abs(v).max()
+    b4 = P.prep_head(q, k, v, None, P.PrepConfig(N=w.N, d=w.d, grid=w.grid, bits=4))
+    o4 = A.emulate_head(b4, cfg, rows=rows).astype(np.float64)
+    assert np.sqrt(((o - ref) ** 2).mean()) < 1.05 * np.sqrt(((o4 - ref) ** 2).mean())
+
+
 def test_smoothing_helps_on_data_it_is_meant_for():
     """K smoothing on K with channel offsets, V smoothing on V with block shifts: each must
     lower the error against exact attention (the directions the paper claims)."""
