@@ -111,6 +111,15 @@ def job_throughput(flops_per_rank, ms_per_step_this_rank, world, device=None):
     return world * flops_per_rank / (ms * 1e-3) / 1e12, ms
 
 
+def _oracle_cfg(w, bits, hybrid):
+    """(PrepConfig, probability format) of the oracle for the arrangement the bench runs."""
+    from oracle import attention as OA
+    from oracle import prep as OP
+    if hybrid:
+        return OP.PrepConfig(N=w.N, d=w.d, grid=w.grid, bits=4, v_format="mxfp4"), OA.P_EXPCAST
+    return OP.PrepConfig(N=w.N, d=w.d, grid=w.grid, bits=bits), None
+
+
 def run_reference(args, w, bits):
     """The oracle as it stands, timed on the host cores on a bounded sample of the workload."""
     import numpy as np
@@ -118,12 +127,12 @@ def run_reference(args, w, bits):
     from oracle import prep as OP
     rows_per_step = args.ref_rows
     q, k, v = [t[0, 0].float().numpy() for t in vc_inputs.make_qkv(w, heads=[0])]
-    cfg = OP.PrepConfig(N=w.N, d=w.d, grid=w.grid, bits=bits)
+    cfg, pf = _oracle_cfg(w, bits, bits == 4 and args.p_format == "expcast")
     rows = np.linspace(0, w.N - 1, rows_per_step).astype(np.int64)
 
     def step():
         bundle = OP.prep_head(q, k, v, None, cfg)
-        OA.emulate_head(bundle, cfg, rows=rows)
+        OA.emulate_head(bundle, cfg, rows=rows, p_format=pf)
 
     for _ in range(args.warmup):
         step()
@@ -142,12 +151,12 @@ def run_reference(args, w, bits):
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
 
 
-def cpu_baseline(w, bits, budget_rows=4096, heads=2):
+def cpu_baseline(w, bits, hybrid=False, budget_rows=4096, heads=2):
     """The oracle as it stands on a bounded sample (about 10-30 s of CPU work)."""
     import numpy as np
     from oracle import attention as OA
     from oracle import prep as OP
-    cfg = OP.PrepConfig(N=w.N, d=w.d, grid=w.grid, bits=bits)
+    cfg, pf = _oracle_cfg(w, bits, hybrid)
     rows = np.linspace(0, w.N - 1, min(budget_rows, w.N)).astype(np.int64)
     tp = ta = 0.0
     for h in range(heads):
@@ -155,7 +164,7 @@ def cpu_baseline(w, bits, budget_rows=4096, heads=2):
         t0 = time.perf_counter()
         bundle = OP.prep_head(q, k, v, None, cfg)
         t1 = time.perf_counter()
-        OA.emulate_head(bundle, cfg, rows=rows)
+        OA.emulate_head(bundle, cfg, rows=rows, p_format=pf)
         t2 = time.perf_counter()
         tp += t1 - t0
         ta += t2 - t1
@@ -307,7 +316,10 @@ def main():
     # dominant kernel: the attention forward (dense contraction on the tensor cores).  Its peak is
     # the measured bf16 figure x the nominal FP8:bf16 ratio of 2 (x4 for FP4); the kernel runs inside
     # a long step, so the sustained figure applies.
-    ratio = 2.0 if args.bits == 8 else 4.0   # nominal dense FP8 : bf16 = 2, FP4 : bf16 = 4
+    # (the hybrid 4-bit arrangement runs the score product at the FP4 rate and the value product at
+    # the FP8 rate: the two halves of the FLOPs take 1/4 + 1/2 of a bf16 pass, a ratio of 8/3)
+    hybrid = args.bits == 4 and args.p_format == "expcast"
+    ratio = 2.0 if args.bits == 8 else (8.0 / 3.0 if hybrid else 4.0)   # nominal dense FP8 : bf16 = 2, FP4 : bf16 = 4
     peak = peaks["bf16_sustained"] * ratio
     achieved = w.flops / (attn_ms * 1e-3) / 1e12
     # DRAM traffic of one attention launch: measured once under ncu on a smaller case of the same
@@ -322,7 +334,7 @@ def main():
     out = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
-        "vs_baseline": None, "dtype": ("int8 QK / e4m3 PV" if args.int8_qk else "e4m3") if args.bits == 8 else "nvfp4", "data": "synthetic",
+        "vs_baseline": None, "dtype": ("int8 QK / e4m3 PV" if args.int8_qk else "e4m3") if args.bits == 8 else ("nvfp4 QK / e4m3 x e2m1 PV" if hybrid else "nvfp4"), "data": "synthetic",
         "config": {"workload": w.name, "B": w.B, "H": w.H, "N": w.N, "d": w.d, "grid": list(w.grid),
                    "bits": args.bits, "p_format": args.p_format, "perm": args.perm, "data": args.data, "l2": "inputs larger than L2 (Q+K+V = %.0f MB)" % (3 * q.numel() * 2 / 1e6),
                    "step": "vc_prep + vc_attn_fwd" + (" (+ vc_group every 4th step)" if args.perm == "group" else "")},
@@ -331,8 +343,9 @@ def main():
                      "frac": achieved / peak, "traffic": traffic,
                      "traffic_source": "ncu dram__bytes_read+write of this kernel on B2 H16 N16384 d128 "
                                        "(profiles/), scaled by head-tokens: %.0f B per (head, token)" % per_ht,
-                     "peak_source": f"{peaks['source']}: bf16 sustained {peaks['bf16_sustained']} TF/s x {ratio:g}" + (" (nominal FP8:bf16)" if args.bits == 8 else " (nominal FP4:bf16)"),
-                     ("frac_of_nominal_fp8_4500" if args.bits == 8 else "frac_of_nominal_fp4_9000"): achieved / (4500.0 if args.bits == 8 else 9000.0),
+                     "peak_source": f"{peaks['source']}: bf16 sustained {peaks['bf16_sustained']} TF/s x {ratio:g}" + (" (nominal FP8:bf16)" if args.bits == 8 else (" (half the FLOPs at FP4:bf16 = 4, half at FP8:bf16 = 2)" if hybrid else " (nominal FP4:bf16)")),
+                     ("frac_of_nominal_fp8_4500" if args.bits == 8 else ("frac_of_nominal_fp4_fp8_mix_6000" if hybrid else "frac_of_nominal_fp4_9000")):
+                         achieved / (4500.0 if args.bits == 8 else (6000.0 if hybrid else 9000.0)),
                      "ms": attn_ms},
         "group": group,
         "prep": {"ms": prep_ms, "algorithmic_gb": prep_bytes / 1e9, "gbs": prep_gbs,
@@ -354,7 +367,7 @@ def main():
         except Exception as exc:  # pragma: no cover
             out["bf16_sdpa"] = {"error": str(exc)[:200]}
     if not args.no_cpu_baseline:
-        out["cpu_baseline"] = cpu_baseline(w, args.bits)
+        out["cpu_baseline"] = cpu_baseline(w, args.bits, hybrid)
     print(json.dumps(out), flush=True)
     if world > 1:
         dist.destroy_process_group()

@@ -31,7 +31,7 @@ vc_status resolve(const vc_params* p, Problem* out) {
   if (pr.p_format < VC_P_EXPCAST_E4M3 || pr.p_format > VC_P_EXP_MIX_E4M3) return VC_ERR_INVALID_ARG;
   if (pr.bits == 8 && pr.p_format == VC_P_NVFP4) return VC_ERR_UNSUPPORTED;
   if (pr.p_format > VC_P_NVFP4 && (p->flags & VC_FLAG_INT8_QK)) return VC_ERR_UNSUPPORTED;
-  if (pr.bits == 4 && pr.p_format != VC_P_NVFP4) return VC_ERR_UNSUPPORTED;
+  if (pr.bits == 4 && pr.p_format != VC_P_NVFP4 && pr.p_format != VC_P_EXPCAST_E4M3) return VC_ERR_UNSUPPORTED;
   pr.flags = p->flags;
   if (pr.flags & ~(VC_FLAG_ALL | VC_FLAG_INT8_QK)) return VC_ERR_INVALID_ARG;
   pr.softmax_scale = p->softmax_scale != 0.f ? p->softmax_scale : 1.0f / sqrtf((float)pr.d);
@@ -61,6 +61,7 @@ vc_status resolve(const vc_params* p, Problem* out) {
   pr.kernel_variant = p->kernel_variant;
   if (pr.kernel_variant < 0 || pr.kernel_variant > 1) return VC_ERR_INVALID_ARG;
   if ((pr.flags & VC_FLAG_INT8_QK) && (pr.bits != 8 || pr.kernel_variant != 0)) return VC_ERR_INVALID_ARG;
+  if (hybrid4(pr) && pr.kernel_variant != 0) return VC_ERR_UNSUPPORTED;
   *out = pr;
   return VC_OK;
 }
@@ -79,7 +80,7 @@ QuantLayout quant_layout(const Problem& pr) {
   L.k_mean_bytes = BH * d * 4;
   L.q_micro_bytes = four ? BH * np_ * d / 16 : 0;
   L.k_micro_bytes = L.q_micro_bytes;
-  L.v_micro_bytes = L.q_micro_bytes;
+  L.v_micro_bytes = hybrid4(pr) ? BH * np_ * d / 32 : L.q_micro_bytes;
   size_t off = 0;
   auto place = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 1024); return o; };
   L.q_codes = place(L.q_codes_bytes);

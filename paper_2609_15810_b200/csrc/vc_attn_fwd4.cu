@@ -17,6 +17,12 @@
 // half a conversion:  code = E2M1(2^(s cs + log2 2688 - m' - log2 f_g)).  (Moving part of the
 // exponentials to a polynomial on the FMA pipe was measured and is slower: the stage is bound by
 // issue slots and hand-off latency before the special-function unit, which runs at 64 %.)
+//
+// HYB = true is the hybrid 4-bit arrangement: the score product stays NVFP4, but P is the
+// ExpCast-FP8 code of Eq. 7 (two FMAs per score, as in the 8-bit kernel) and the value product
+// runs as kind::mxf8f6f4: E4M3 P^ times E2M1 R^ under power-of-two factors per 32 tokens.  The
+// value tile arrives through a 4-bit tensor map that spreads it into the 16-byte containers
+// that instruction kind reads; P^ carries the constant factor 1.
 #include <cuda_bf16.h>
 #include <cuda_fp8.h>
 
@@ -33,14 +39,16 @@ using namespace attn;
 // Factor arrays -> MMA chunk order.  One CTA per (b, h, 128-row tile), thread r = operand row.
 //   sf_q  [BH*nb][D/64][512]          Q^ factors of query tile
 //   sf_kv [BH*nb][D/64 + 2][512]      K^ factors of key tile, then the R^ factors of the same
-//                                     tile (operand rows = channels, groups = 16 tokens)
+//                                     tile (operand rows = channels, groups = 16 tokens);
+//                                     HYB: [D/64 + 1] chunks, the last one holding the four
+//                                     power-of-two factors (32 tokens each) of every channel
 // Chunk byte 16 (r % 32) + 4 (r / 32) + k  <-  factor of row r, group 4 kb + k.
-template <int D>
+template <int D, bool HYB>
 __global__ void __launch_bounds__(128)
 nvfp4_sf_tiles_kernel(const uint8_t* __restrict__ q_micro, const uint8_t* __restrict__ k_micro,
                       const uint8_t* __restrict__ v_micro, uint8_t* __restrict__ sf_q, uint8_t* __restrict__ sf_kv,
                       int nb, int n_pad) {
-  constexpr int KB = D / 64;
+  constexpr int KB = D / 64, NVC = HYB ? 1 : 2;
   const int tile = blockIdx.x, bh = blockIdx.y, r = threadIdx.x;
   const size_t t_idx = (size_t)bh * nb + tile;
   const uint32_t pos = (r & 31) * 16 + (r >> 5) * 4;
@@ -50,7 +58,14 @@ nvfp4_sf_tiles_kernel(const uint8_t* __restrict__ q_micro, const uint8_t* __rest
 #pragma unroll
   for (int kb = 0; kb < KB; ++kb) {
     *reinterpret_cast<uint32_t*>(sf_q + t_idx * (KB * 512) + kb * 512 + pos) = qm[kb];
-    *reinterpret_cast<uint32_t*>(sf_kv + t_idx * ((KB + 2) * 512) + kb * 512 + pos) = km[kb];
+    *reinterpret_cast<uint32_t*>(sf_kv + t_idx * ((KB + NVC) * 512) + kb * 512 + pos) = km[kb];
+  }
+  if constexpr (HYB) {
+    uint32_t w = 0;
+    if (r < D) w = *reinterpret_cast<const uint32_t*>(v_micro + ((size_t)bh * D + r) * (n_pad / 32) + (size_t)tile * 4);
+    else if (r < D + 16) w = 0x7f7f7f7fu;   // the rows of ones: factor 2^0
+    *reinterpret_cast<uint32_t*>(sf_kv + t_idx * ((KB + NVC) * 512) + KB * 512 + pos) = w;
+    return;
   }
   uint32_t w0 = 0, w1 = 0;
   if (r < D) {
@@ -71,6 +86,7 @@ struct Attn4Args {
   uint32_t* status;
   int N, n_pad, nb;
   float sl;                        // softmax_scale * log2(e)
+  float code_off;                  // 120 + beta  (Eq. 7; hybrid arrangement only)
 };
 
 // Value of a non-negative E4M3 byte.
@@ -86,7 +102,7 @@ __device__ __forceinline__ float decode_ue4m3(uint32_t code) {
 //   warps 4-11    softmax warpgroups (tile 0, tile 1), one thread per query row
 //   warps 12-19   correction warpgroups, one thread per query row
 // Tensor memory: S (128 columns) | A_0 (d + 16) | A_1 (d + 16) | scale factors (56 columns).
-template <int D>
+template <int D, bool HYB>
 __global__ void __launch_bounds__(640, 1)
 attn4_fwd_2q_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                     const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_mu,
@@ -99,18 +115,21 @@ attn4_fwd_2q_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   constexpr uint32_t SFQ_COL = SF_COL, SFK_COL = SF_COL + 16, SFP_COL = SF_COL + 24, SFV_COL = SF_COL + 40;
   constexpr int kRegCtl = 48, kRegSoftmax = 160, kRegCorr = 56;
   static_assert(kRegCtl + 2 * kRegSoftmax + 2 * kRegCorr <= 5 * 96, "register budget exceeds the CTA's allocation");
-  constexpr uint32_t kQBytes = 128 * kRowB, kKBytes = 128 * kRowB, kVBytes = D * 64, kOnesBytes = 16 * 64;
+  constexpr int NVC = HYB ? 1 : 2;                  // value factor chunks per key tile
+  constexpr uint32_t kVRow = HYB ? 128 : 64;        // bytes of a value row in shared memory
+  constexpr uint32_t kQBytes = 128 * kRowB, kKBytes = 128 * kRowB, kVBytes = D * kVRow, kOnesBytes = 16 * kVRow;
+  constexpr uint32_t kVTx = D * 64;                 // bytes the value copy reports (the packed ones)
   constexpr uint32_t kMuBytes = D * 32, kMuPad = ((kMuBytes + 1023) / 1024) * 1024;
-  constexpr uint32_t kSfqBytes = KB * 512, kSfBytes = (KB + 2) * 512, kSfPad = ((kSfBytes + 1023) / 1024) * 1024;
+  constexpr uint32_t kSfqBytes = KB * 512, kSfBytes = (KB + NVC) * 512, kSfPad = ((kSfBytes + 1023) / 1024) * 1024;
   constexpr uint32_t kStageBytes = kKBytes + kVBytes + kOnesBytes + kMuPad + kSfPad;
-  constexpr uint32_t kPBytes = 128 * 64, kSfpBytes = 1024, kAmBytes = 128 * 32;
+  constexpr uint32_t kPBytes = 128 * kVRow, kSfpBytes = 1024, kAmBytes = 128 * 32;
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   unsigned char* sQ = smem;                                    // [2][128 x D/2]
-  unsigned char* sP = sQ + 2 * kQBytes;                        // [2][128 x 64] probability codes
+  unsigned char* sP = sQ + 2 * kQBytes;                        // [2][128 x 64] probability codes (HYB: 128 x 128)
   unsigned char* sAm = sP + 2 * kPBytes;                       // [2][128 x 8 fp32] row-sum pairs
   unsigned char* sSfq = sAm + 2 * kAmBytes;                    // [2][KB][512] Q^ factors
-  unsigned char* sSfp = sSfq + 2 * 1024;                       // [2][2][512]  P^ factors
+  unsigned char* sSfp = sSfq + 2 * 1024;                       // [2][2][512]  P^ factors (HYB: one chunk of ones)
   unsigned char* sSfOnes = sSfp + 2 * kSfpBytes;               // [512] factors of value rows 128..143
   unsigned char* sStage = sSfOnes + 1024;                      // [kStages2]{K, V | ones, Mu, factors}
   FaSmem* sh = reinterpret_cast<FaSmem*>(sStage + kStages2 * kStageBytes);
@@ -134,10 +153,14 @@ attn4_fwd_2q_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   for (int i = tid; i < 2 * (int)kAmBytes / 16; i += 640) reinterpret_cast<uint4*>(sAm)[i] = make_uint4(0, 0, 0, 0);
   // 16 rows of E2M1 1.0 (two per byte) behind every value tile; their factor chunk: 1.0 for
   // rows 0..15 of the second 128-row half, group bytes 0..3
+  // (HYB: the same bytes, of which the product reads the low 8 of every 16; factor code 127 = 2^0,
+  // and a chunk of that code for every row of P^)
   for (int i = tid; i < kStages2 * (int)kOnesBytes / 4; i += 640)
     reinterpret_cast<uint32_t*>(sStage + (i / (kOnesBytes / 4)) * kStageBytes + kKBytes + kVBytes)[i % (kOnesBytes / 4)] = 0x22222222u;
   for (int i = tid; i < 128; i += 640)
-    reinterpret_cast<uint32_t*>(sSfOnes)[i] = ((i & 3) == 0 && i < 64) ? 0x38383838u : 0u;
+    reinterpret_cast<uint32_t*>(sSfOnes)[i] = ((i & 3) == 0 && i < 64) ? (HYB ? 0x7f7f7f7fu : 0x38383838u) : 0u;
+  if constexpr (HYB)
+    for (int i = tid; i < 128; i += 640) reinterpret_cast<uint32_t*>(sSfp)[i] = 0x7f7f7f7fu;
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy stores -> tensor-core reads
   if (warp == 2) { tmem_alloc<kTmemCols>(&sh->tmem_base); tmem_relinquish(); }
   tc_fence_before();
@@ -163,9 +186,9 @@ attn4_fwd_2q_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         unsigned char* base = sStage + st * kStageBytes;
         if (!warp_wait2(&sh->kv_empty[st], (it & 1) ^ 1, sh, a.status, 11)) break;
         if (elect_one()) {
-          mbar_expect_tx(&sh->kv_full[st], kKBytes + kVBytes + kMuBytes + kSfBytes);
+          mbar_expect_tx(&sh->kv_full[st], kKBytes + kVTx + kMuBytes + kSfBytes);
           tma_load_3d(base, &tm_k, &sh->kv_full[st], 0, j * 128, bh);
-          tma_load_3d(base + kKBytes, &tm_v, &sh->kv_full[st], j * 64, 0, bh);
+          tma_load_3d(base + kKBytes, &tm_v, &sh->kv_full[st], HYB ? j * 128 : j * 64, 0, bh);   // elements resp. bytes
           tma_load_3d(base + kKBytes + kVBytes + kOnesBytes, &tm_mu, &sh->kv_full[st], 0, 0, bh * nb + j);
           bulk_load(base + kKBytes + kVBytes + kOnesBytes + kMuPad, a.sf_kv + ((size_t)bh * nb + j) * kSfBytes, kSfBytes,
                     &sh->kv_full[st]);
@@ -213,11 +236,14 @@ attn4_fwd_2q_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     } else if (warp == 3) {
       // ------------------------------------------------------------------ accumulator issuer
       const uint32_t idesc_pv = idesc_nvfp4(128, D + 16), idesc_mu = idesc_tf32(128, D);
-      const uint64_t dp[2] = {smem_desc_kmajor(smem_u32(sP), 64), smem_desc_kmajor(smem_u32(sP + kPBytes), 64)};
+      const uint64_t dp[2] = {smem_desc_kmajor(smem_u32(sP), kVRow), smem_desc_kmajor(smem_u32(sP + kPBytes), kVRow)};
       const uint64_t dam[2] = {smem_desc_kmajor(smem_u32(sAm), 32), smem_desc_kmajor(smem_u32(sAm + kAmBytes), 32)};
-      if (D == 128 && elect_one()) {                       // factors of the rows of ones (value rows 128..143)
-        tmem_cp_sf(tmem + SFV_COL + 4, smem_desc_sf_chunk(smem_u32(sSfOnes)));
-        tmem_cp_sf(tmem + SFV_COL + 12, smem_desc_sf_chunk(smem_u32(sSfOnes)));
+      if (elect_one()) {
+        if (D == 128) {                                    // factors of the rows of ones (value rows 128..143)
+          tmem_cp_sf(tmem + SFV_COL + 4, smem_desc_sf_chunk(smem_u32(sSfOnes)));
+          if (!HYB) tmem_cp_sf(tmem + SFV_COL + 12, smem_desc_sf_chunk(smem_u32(sSfOnes)));
+        }
+        if (HYB) tmem_cp_sf(tmem + SFP_COL, smem_desc_sf_chunk(smem_u32(sSfp)));   // P^: factor 1 everywhere
       }
       __syncwarp();
       bool ok = true;
@@ -226,7 +252,7 @@ attn4_fwd_2q_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         const int stp = (j + kStages2 - 1) % kStages2;    // stage of tile j-1
         if (!(ok = warp_wait2(&sh->kv_full[st], it & 1, sh, a.status, 25))) break;
         const unsigned char* base = sStage + st * kStageBytes;
-        const uint64_t dv = smem_desc_kmajor(smem_u32(base + kKBytes), 64);
+        const uint64_t dv = smem_desc_kmajor(smem_u32(base + kKBytes), kVRow);
         const uint64_t dm = smem_desc_kmajor(smem_u32(sStage + stp * kStageBytes + kKBytes + kVBytes + kOnesBytes), 32);
         const uint32_t sfv_smem = smem_u32(base + kKBytes + kVBytes + kOnesBytes + kMuPad + KB * 512);
 #pragma unroll
@@ -235,16 +261,24 @@ attn4_fwd_2q_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
           if (elect_one()) {
             tc_fence_after();
             const uint32_t o_col = tmem + O_COL + O_STRIDE * t;
-            if (t == 0) {
-              tmem_cp_sf(tmem + SFV_COL, smem_desc_sf_chunk(sfv_smem));
-              tmem_cp_sf(tmem + SFV_COL + 8, smem_desc_sf_chunk(sfv_smem + 512));
-            }
-            tmem_cp_sf(tmem + SFP_COL + t * 8, smem_desc_sf_chunk(smem_u32(sSfp + t * kSfpBytes)));
-            tmem_cp_sf(tmem + SFP_COL + t * 8 + 4, smem_desc_sf_chunk(smem_u32(sSfp + t * kSfpBytes + 512)));
+            if constexpr (HYB) {
+              if (t == 0) tmem_cp_sf(tmem + SFV_COL, smem_desc_sf_chunk(sfv_smem));
 #pragma unroll
-            for (int kb = 0; kb < 2; ++kb)
-              mma_nvfp4_ss(o_col, dp[t] + 2 * kb, dv + 2 * kb, idesc_pv, (j > 0) | (kb > 0), tmem + SFP_COL + t * 8 + kb * 4,
-                           tmem + SFV_COL + kb * 8);
+              for (int k = 0; k < 4; ++k)                  // 32 keys each; factor byte k of the value rows
+                mma_mxf8_ss(o_col, dp[t] + 2 * k, dv + 2 * k, idesc_mxf8_e4m3_e2m1(128, D + 16, k), (j > 0) | (k > 0),
+                            tmem + SFP_COL, tmem + SFV_COL);
+            } else {
+              if (t == 0) {
+                tmem_cp_sf(tmem + SFV_COL, smem_desc_sf_chunk(sfv_smem));
+                tmem_cp_sf(tmem + SFV_COL + 8, smem_desc_sf_chunk(sfv_smem + 512));
+              }
+              tmem_cp_sf(tmem + SFP_COL + t * 8, smem_desc_sf_chunk(smem_u32(sSfp + t * kSfpBytes)));
+              tmem_cp_sf(tmem + SFP_COL + t * 8 + 4, smem_desc_sf_chunk(smem_u32(sSfp + t * kSfpBytes + 512)));
+#pragma unroll
+              for (int kb = 0; kb < 2; ++kb)
+                mma_nvfp4_ss(o_col, dp[t] + 2 * kb, dv + 2 * kb, idesc_pv, (j > 0) | (kb > 0), tmem + SFP_COL + t * 8 + kb * 4,
+                             tmem + SFV_COL + kb * 8);
+            }
             if (j > 0) mma_tf32_ss(o_col, dam[t], dm, idesc_mu, 1);
             mma_commit(&sh->o_done[t]);
             if (j > 0) mma_commit(&sh->kv_empty[stp]);    // this tile is done with stage j-1
@@ -270,7 +304,8 @@ attn4_fwd_2q_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     const int t = (warp - 4) >> 2;                         // query tile of this warpgroup
     const int row = (warp & 3) * 32 + lane;
     // my row of the swizzled code tile: 64-byte rows, chunk c sits at chunk position c ^ ((row / 2) % 4)
-    unsigned char* p_row = sP + t * kPBytes + row * 64;
+    // (HYB: 128-byte rows, chunk c at position c ^ (row % 8))
+    unsigned char* p_row = sP + t * kPBytes + row * kVRow;
     const int p_xor = (row >> 1) & 3;
     uint32_t* sfp_row = reinterpret_cast<uint32_t*>(sSfp + t * kSfpBytes + (row & 31) * 16 + (row >> 5) * 4);
     const float cs = (a.q_g[bh] * a.k_g[bh]) * a.sl;       // code units -> log2 domain
@@ -318,6 +353,28 @@ attn4_fwd_2q_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       sh->alpha[t][row] = ex2_approx(m_run - m_new);      // alpha; 0 on the first tile
       mbar_arrive(&sh->a_full[t][j & 1]);
       m_run = m_new;
+      if constexpr (HYB) {
+        // ExpCast-FP8 (Eq. 7) in two FMAs: t = sat((8 u + 120 + beta) / 128) clips to [0, 1], then
+        // t * 128 + 1.5 * 2^23 rounds to the nearest even integer in the low mantissa bits.
+        if (j > 0 && !warp_wait2(&sh->o_done[t], (j - 1) & 1, sh, a.status, 31)) break;
+        const float fa = cs * 0.0625f, fb = (a.code_off - 8.0f * m_new) * 0.0078125f;
+        auto code4 = [&](const uint32_t (&sv)[32], int w) -> uint32_t {
+          const uint32_t r0 = __float_as_uint(fmaf(fma_sat(__uint_as_float(sv[4 * w]), fa, fb), 128.0f, 12582912.0f));
+          const uint32_t r1 = __float_as_uint(fmaf(fma_sat(__uint_as_float(sv[4 * w + 1]), fa, fb), 128.0f, 12582912.0f));
+          const uint32_t r2 = __float_as_uint(fmaf(fma_sat(__uint_as_float(sv[4 * w + 2]), fa, fb), 128.0f, 12582912.0f));
+          const uint32_t r3 = __float_as_uint(fmaf(fma_sat(__uint_as_float(sv[4 * w + 3]), fa, fb), 128.0f, 12582912.0f));
+          return __byte_perm(__byte_perm(r0, r1, 0x0040), __byte_perm(r2, r3, 0x0040), 0x5410);
+        };
+        auto store16 = [&](const uint32_t (&sv)[32], int half, int chunk) {   // keys 16 chunk .. +15
+          const uint4 v = make_uint4(code4(sv, 4 * half), code4(sv, 4 * half + 1), code4(sv, 4 * half + 2), code4(sv, 4 * half + 3));
+          *reinterpret_cast<uint4*>(p_row + ((chunk ^ (row & 7)) << 4)) = v;
+        };
+        store16(s0, 0, 0); store16(s0, 1, 1); store16(s1, 0, 2); store16(s1, 1, 3);
+        store16(s2, 0, 4); store16(s2, 1, 5); store16(s3, 0, 6); store16(s3, 1, 7);
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");          // my stores -> tensor-core reads
+        mbar_arrive(&sh->pc_full[t][j & 1]);
+        continue;
+      }
       // p = 2^(s cs - m') * 2688: the row maximum maps to 6 * 448, so the largest factor is 448.
       // Per 16-key group: factor = E4M3(max p / 6); element / factor = 2^(s cs + c0 - log2 factor),
       // a zero factor zeroes the group.  The eight factor chains run before the wait below: they
@@ -431,21 +488,23 @@ attn4_fwd_2q_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   if (warp == 2) tmem_dealloc<kTmemCols>(tmem);
 }
 
-template <int D>
+template <int D, bool HYB>
 cudaError_t run4(const Problem& pr, const QuantLayout& ql, const WorkLayout& wl, const uint8_t* quant,
                  void* o, uint8_t* work, cudaStream_t s) {
-  constexpr int KB = D / 64;
+  constexpr int KB = D / 64, NVC = HYB ? 1 : 2;
+  constexpr size_t kVRow = HYB ? 128 : 64;
   alignas(64) CUtensorMap tq, tk, tv, tmt;
   if (!make_map(&tq, quant + ql.q_codes, D / 2, pr.n_pad, pr.BH, D / 2, 128) ||
       !make_map(&tk, quant + ql.k_codes, D / 2, pr.n_pad, pr.BH, D / 2, 128) ||
-      !make_map(&tv, quant + ql.v_codes, (uint64_t)pr.n_pad / 2, D, pr.BH, 64, D) ||
+      !(HYB ? make_map_u4(&tv, quant + ql.v_codes, (uint64_t)pr.n_pad, D, pr.BH, D)
+            : make_map(&tv, quant + ql.v_codes, (uint64_t)pr.n_pad / 2, D, pr.BH, 64, D)) ||
       !make_map(&tmt, work + wl.mu_mma, 32, D, (uint64_t)pr.BH * pr.nb, 32, D))
     return cudaErrorUnknown;
   const size_t n = (size_t)pr.BH * pr.nb * D;
   means_tile_layout_kernel<D><<<(unsigned)((n + 255) / 256), 256, 0, s>>>((const __nv_bfloat16*)(quant + ql.v_means),
                                                                         (float*)(work + wl.mu_mma), n);
-  nvfp4_sf_tiles_kernel<D><<<dim3(pr.nb, pr.BH), 128, 0, s>>>(quant + ql.q_micro, quant + ql.k_micro, quant + ql.v_micro,
-                                                             work + wl.sf_q, work + wl.sf_kv, pr.nb, pr.n_pad);
+  nvfp4_sf_tiles_kernel<D, HYB><<<dim3(pr.nb, pr.BH), 128, 0, s>>>(quant + ql.q_micro, quant + ql.k_micro, quant + ql.v_micro,
+                                                                  work + wl.sf_q, work + wl.sf_kv, pr.nb, pr.n_pad);
   Attn4Args a{};
   a.q_g = (const float*)(quant + ql.q_scale);
   a.k_g = (const float*)(quant + ql.k_scale);
@@ -455,11 +514,13 @@ cudaError_t run4(const Problem& pr, const QuantLayout& ql, const WorkLayout& wl,
   a.status = (uint32_t*)(work + wl.status);
   a.N = pr.N; a.n_pad = pr.n_pad; a.nb = pr.nb;
   a.sl = pr.softmax_scale * 1.4426950408889634f;
-  constexpr size_t stage = 128 * (D / 2) + D * 64 + 1024 + ((D * 32 + 1023) / 1024) * 1024 + (((KB + 2) * 512 + 1023) / 1024) * 1024;
-  constexpr size_t smem = 1024 + 2 * 128 * (D / 2) + 2 * 128 * 64 + 2 * 128 * 32 + 2 * 1024 + 2 * 1024 + 1024 + kStages2 * stage + sizeof(FaSmem);
-  cudaError_t e = cudaFuncSetAttribute(attn4_fwd_2q_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  a.code_off = 120.0f + pr.beta;
+  constexpr size_t stage = 128 * (D / 2) + (D + 16) * kVRow + ((D * 32 + 1023) / 1024) * 1024 + (((KB + NVC) * 512 + 1023) / 1024) * 1024;
+  constexpr size_t smem = 1024 + 2 * 128 * (D / 2) + 2 * 128 * kVRow + 2 * 128 * 32 + 2 * 1024 + 2 * 1024 + 1024 + kStages2 * stage + sizeof(FaSmem);
+  static_assert(smem <= 227 * 1024, "shared memory of the 4-bit kernel exceeds the SM");
+  cudaError_t e = cudaFuncSetAttribute(attn4_fwd_2q_kernel<D, HYB>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
-  attn4_fwd_2q_kernel<D><<<dim3((pr.nb + 1) / 2, pr.BH), 640, smem, s>>>(tq, tk, tv, tmt, a);
+  attn4_fwd_2q_kernel<D, HYB><<<dim3((pr.nb + 1) / 2, pr.BH), 640, smem, s>>>(tq, tk, tv, tmt, a);
   count_launches(3);
   return cudaGetLastError();
 }
@@ -468,7 +529,9 @@ cudaError_t run4(const Problem& pr, const QuantLayout& ql, const WorkLayout& wl,
 
 cudaError_t launch_attn_fwd4(const Problem& pr, const QuantLayout& ql, const WorkLayout& wl,
                              const uint8_t* quant, void* o, uint8_t* work, cudaStream_t stream) {
-  return pr.d == 128 ? run4<128>(pr, ql, wl, quant, o, work, stream) : run4<64>(pr, ql, wl, quant, o, work, stream);
+  if (hybrid4(pr))
+    return pr.d == 128 ? run4<128, true>(pr, ql, wl, quant, o, work, stream) : run4<64, true>(pr, ql, wl, quant, o, work, stream);
+  return pr.d == 128 ? run4<128, false>(pr, ql, wl, quant, o, work, stream) : run4<64, false>(pr, ql, wl, quant, o, work, stream);
 }
 
 }  // namespace vc

@@ -96,5 +96,23 @@ inline bool make_map(CUtensorMap* m, const void* base, uint64_t dim0, uint64_t d
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+
+// 3-D tensor of packed 4-bit elements [dim2][dim1][dim0 elements]; a box of 128 elements x box1
+// rows lands in shared memory as 128-byte rows of 16-byte containers (16 elements in the low 8
+// bytes, 128-byte swizzle): the layout kind::mxf8f6f4 reads 4-bit operands in.  The copy reports
+// the packed bytes (64 per row) to its mbarrier.  `base` must be 32-byte aligned, dim0 a
+// multiple of 128.
+inline bool make_map_u4(CUtensorMap* m, const void* base, uint64_t dim0, uint64_t dim1, uint64_t dim2, uint32_t box1) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn || ((uintptr_t)base & 31) || (dim0 & 127)) return false;
+  const cuuint64_t dims[3] = {dim0, dim1, dim2};
+  const cuuint64_t strides[2] = {dim0 / 2, dim0 / 2 * dim1};
+  const cuuint32_t box[3] = {128, box1, 1};
+  const cuuint32_t estr[3] = {1, 1, 1};
+  return fn(m, CU_TENSOR_MAP_DATA_TYPE_16U4_ALIGN16B, 3, const_cast<void*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 }  // namespace attn
 }  // namespace vc

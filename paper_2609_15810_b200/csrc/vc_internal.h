@@ -23,6 +23,11 @@ struct Problem {
   int kernel_variant;
 };
 
+// The hybrid 4-bit arrangement: NVFP4 Q^ and K^, ExpCast-FP8 P, E2M1 values under power-of-two
+// factors per 32 tokens (the FP8 x FP4 block-scaled product).  Selected by bits = 4 with
+// p_format = VC_P_EXPCAST_E4M3.
+inline bool hybrid4(const Problem& pr) { return pr.bits == 4 && pr.p_format == VC_P_EXPCAST_E4M3; }
+
 // Byte offsets of the sections of the quantized bundle.
 struct QuantLayout {
   size_t q_codes, k_codes, v_codes, q_scale, k_scale, v_scale, v_means, k_mean;

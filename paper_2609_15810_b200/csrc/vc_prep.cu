@@ -393,7 +393,7 @@ __device__ __forceinline__ void qk_row_item(const PrepArgs& a, const int TENSOR 
 // ---------------------------------------------------------------------------------------
 // V.  A thread owns one channel pair and 128 / (256 / (D/2)) consecutive tokens of the gathered
 // block, so block means and the channel-major (token-contiguous) code rows need no transposition.
-enum { kVStats = 0, kVQuant8 = 1, kVQuant4 = 2 };
+enum { kVStats = 0, kVQuant8 = 1, kVQuant4 = 2, kVQuant4M = 3 };   // 4M: E2M1 under power-of-two factors per 32 tokens
 
 template <int D, int STAGE>
 __device__ __forceinline__ void v_item(const PrepArgs& a, const unsigned char* stage, float* red, int bh, int blk,
@@ -528,6 +528,57 @@ __device__ __forceinline__ void v_item(const PrepArgs& a, const unsigned char* s
       } else {
         *reinterpret_cast<uint2*>(d) = make_uint2(packed[0], packed[1]);
         *md = (uint8_t)micro;
+      }
+    }
+    if (tg == 0)
+      *reinterpret_cast<__nv_bfloat162*>(a.v_means + mu_at) = __floats2bfloat162_rn(mu0, mu1);
+  }
+
+  if constexpr (STAGE == kVQuant4M) {
+    // E2M1 under one power-of-two factor per channel per 32 consecutive permuted tokens (the
+    // operand format of the FP8 x FP4 block-scaled product).  Factor 2^e with e the smallest
+    // exponent that keeps the group maximum inside the E2M1 range: y = max / 6 (one division),
+    // e = exponent(y), plus one unless y is a power of two.  Scaling by 2^-e is exact.
+    float m0 = 0.f, m1 = 0.f;
+#pragma unroll
+    for (int i = 0; i < TPG; ++i) { m0 = fmaxf(m0, fabsf(r0[i])); m1 = fmaxf(m1, fabsf(r1[i])); }
+    if constexpr (TPG == 16) {               // a group spans two threads (token groups 2g, 2g + 1)
+      __syncthreads();                       // the previous item's reads of `red` are done
+      red[tg * D + 2 * cp] = m0;
+      red[tg * D + 2 * cp + 1] = m1;
+      __syncthreads();
+      m0 = fmaxf(m0, red[(tg ^ 1) * D + 2 * cp]);
+      m1 = fmaxf(m1, red[(tg ^ 1) * D + 2 * cp + 1]);
+    }
+#pragma unroll
+    for (int half = 0; half < 2; ++half) {
+      const float* r = half == 0 ? r0 : r1;
+      const float m = half == 0 ? m0 : m1;
+      const int c = 2 * cp + half;
+      const unsigned int yb = __float_as_uint(__fdiv_rn(m, 6.0f));
+      int code = (int)((yb >> 23) & 0xffu) + ((yb & 0x7fffffu) ? 1 : 0);     // e + 127
+      code = m > 0.f ? min(max(code, 0), 254) : 0;
+      const float rs = __uint_as_float((unsigned int)(254 - code) << 23);     // 2^-e
+      unsigned int packed[TPG / 8];
+#pragma unroll
+      for (int wi = 0; wi < TPG / 8; ++wi) {
+        unsigned int word = 0;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const int i = 8 * wi + 2 * j;
+          const unsigned int two = __nv_cvt_float2_to_fp4x2(make_float2(r[i] * rs, r[i + 1] * rs), __NV_E2M1, cudaRoundNearest);
+          word |= (two & 0xffu) << (8 * j);
+        }
+        packed[wi] = m > 0.f ? word : 0u;
+      }
+      uint8_t* d = a.v_codes + ((size_t)bh * D + c) * (a.n_pad / 2) + tok0 / 2;
+      uint8_t* md = a.v_micro + ((size_t)bh * D + c) * (a.n_pad / 32) + tok0 / 32;
+      if constexpr (TPG == 32) {
+        *reinterpret_cast<uint4*>(d) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
+        *md = (uint8_t)code;
+      } else {
+        *reinterpret_cast<uint2*>(d) = make_uint2(packed[0], packed[1]);
+        if ((tg & 1) == 0) *md = (uint8_t)code;
       }
     }
     if (tg == 0)
@@ -773,6 +824,8 @@ cudaError_t run(const Problem& pr, PrepArgs a, const WorkLayout& wl, uint8_t* wo
   if ((e = allow_smem(prep_kcolsum_kernel<D>, colsum_smem)) != cudaSuccess) return e;
   if ((e = allow_smem(prep_v_kernel<D, kVStats>, v_smem)) != cudaSuccess) return e;
   if ((e = allow_smem(prep_v_kernel<D, kVQuant>, v_smem)) != cudaSuccess) return e;
+  if (BITS == 4 && (e = allow_smem(prep_v_kernel<D, kVQuant4M>, v_smem)) != cudaSuccess) return e;
+  const bool v_pow2 = hybrid4(pr);           // 4-bit values under power-of-two factors per 32 tokens
   if ((e = allow_smem(prep_qk_kernel<D, kQuant>, row_smem)) != cudaSuccess) return e;
   if (BITS == 8 && (e = allow_smem(prep_qk_kernel<D, kStageQuant8I>, row_smem)) != cudaSuccess) return e;
   if (BITS == 4 && (e = allow_smem(prep_qk_kernel<D, kStageAmax>, row_smem)) != cudaSuccess) return e;
@@ -806,7 +859,10 @@ cudaError_t run(const Problem& pr, PrepArgs a, const WorkLayout& wl, uint8_t* wo
       prep_qk_kernel<D, kStageQuant8I><<<persistent_grid(2 * per), kRowThreads, row_smem, s>>>(a, 2 * per, nh, 0);
     else
       prep_qk_kernel<D, kQuant><<<persistent_grid(2 * per), kRowThreads, row_smem, s>>>(a, 2 * per, nh, 0);
-    prep_v_kernel<D, kVQuant><<<persistent_grid(per), kThreads, v_smem, s>>>(a, per, nh);
+    if (BITS == 4 && v_pow2)
+      prep_v_kernel<D, kVQuant4M><<<persistent_grid(per), kThreads, v_smem, s>>>(a, per, nh);
+    else
+      prep_v_kernel<D, kVQuant><<<persistent_grid(per), kThreads, v_smem, s>>>(a, per, nh);
     count_launches(2);
   }
   return cudaGetLastError();

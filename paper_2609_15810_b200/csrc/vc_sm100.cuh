@@ -289,6 +289,21 @@ __device__ __forceinline__ void mma_nvfp4_ss(uint32_t d_tmem, uint64_t a_desc, u
       ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(sfa_tmem), "r"(sfb_tmem)
       : "memory");
 }
+// Instruction descriptor for kind::mxf8f6f4 with A = E4M3 and B = E2M1 (4-bit elements in 16-byte
+// containers: 16 elements in the low 8 bytes), UE8M0 scale factors per 32 elements, FP32
+// accumulation, both operands K-major, K = 32 per instruction.  A scale factor is one byte of a
+// 32-bit tensor-memory word; `sf_b` (0..3) picks the byte for B, A uses byte 0.
+__device__ __forceinline__ constexpr uint32_t idesc_mxf8_e4m3_e2m1(int M, int N, int sf_b) {
+  return ((uint32_t)sf_b << 4) | (0u << 7) | (5u << 10) | ((uint32_t)(N >> 3) << 17) | (1u << 23) | ((uint32_t)(M >> 4) << 24);
+}
+__device__ __forceinline__ void mma_mxf8_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                            uint32_t accumulate, uint32_t sfa_tmem, uint32_t sfb_tmem) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::mxf8f6f4.block_scale.block32 [%0], %1, %2, %3, [%5], [%6], p;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(sfa_tmem), "r"(sfb_tmem)
+      : "memory");
+}
 // Eight floats -> eight E2M1 codes (round to nearest even, saturating), element 0 in the low nibble.
 __device__ __forceinline__ uint32_t cvt_e2m1x8(float v0, float v1, float v2, float v3, float v4, float v5, float v6, float v7) {
   uint32_t out;

@@ -10,8 +10,15 @@ from oracle import compare as CMP
 from oracle import prep as OP
 
 
+def is_hybrid(p):
+    """The hybrid 4-bit arrangement: bits = 4 with the ExpCast-FP8 probability format."""
+    return p.bits == 4 and p.p_format == vc.VC_P_EXPCAST_E4M3
+
+
 def oracle_cfg(p, **kw):
     dims = (p.rope_dim_t, p.rope_dim_h, p.rope_dim_w)
+    if is_hybrid(p):
+        kw.setdefault("v_format", "mxfp4")
     return OP.PrepConfig(N=p.N, d=p.d, grid=(p.grid_t, p.grid_h, p.grid_w), bits=p.bits,
                          rope=bool(p.flags & vc.VC_FLAG_ROPE), hadamard=bool(p.flags & vc.VC_FLAG_HADAMARD),
                          k_smooth=bool(p.flags & vc.VC_FLAG_K_SMOOTH), v_smooth=bool(p.flags & vc.VC_FLAG_V_SMOOTH),
@@ -50,7 +57,7 @@ def gpu_sections(p, quant):
         out["v_codes"] = CMP.unpack_nibbles(s("v_codes").numpy().reshape(BH, d, n_pad // 2)).transpose(0, 2, 1)
         out["q_micro"] = s("q_micro").numpy().reshape(BH, n_pad, d // 16)
         out["k_micro"] = s("k_micro").numpy().reshape(BH, n_pad, d // 16)
-        out["v_micro"] = s("v_micro").numpy().reshape(BH, d, n_pad // 16).transpose(0, 2, 1)
+        out["v_micro"] = s("v_micro").numpy().reshape(BH, d, n_pad // (32 if is_hybrid(p) else 16)).transpose(0, 2, 1)
         out["q_scale"] = s("q_scale", torch.float32).numpy().reshape(BH)
         out["k_scale"] = s("k_scale", torch.float32).numpy().reshape(BH)
     out["v_scale"] = s("v_scale", torch.float32).numpy().reshape(BH, d)
@@ -89,7 +96,9 @@ def check_prep_head(p, got, bh, ref, what=""):
     else:
         assert rel(got["q_scale"][bh], ref["q_g"]) < 1e-5 and rel(got["k_scale"][bh], ref["k_g"]) < 1e-5, what
         for t in ("q", "k", "v"):
-            stats[t + "_micro"] = CMP.assert_codes_close(got[t + "_micro"][bh], ref[t + "_micro"], 7, what=what + t + "_micro")
+            # (the power-of-two factors of the hybrid arrangement are 8-bit magnitudes)
+            stats[t + "_micro"] = CMP.assert_codes_close(got[t + "_micro"][bh], ref[t + "_micro"],
+                                                         8 if t == "v" and is_hybrid(p) else 7, what=what + t + "_micro")
     for t in ("q", "k", "v"):
         if p.bits == 8 and t != "v" and (p.flags & vc.VC_FLAG_INT8_QK):
             diff = np.abs(got[t + "_codes"][bh].astype(np.int32) - ref[t + "_codes"].astype(np.int32))
@@ -99,7 +108,8 @@ def check_prep_head(p, got, bh, ref, what=""):
             stats[t] = CMP.assert_codes_close(got[t + "_codes"][bh], ref[t + "_codes"], mag, what=what + " " + t + "_codes")
         else:
             # elements under a differing microscale are compared after decoding
-            same = np.repeat(got[t + "_micro"][bh] == ref[t + "_micro"], 16, axis=1 if t != "v" else 0)
+            same = np.repeat(got[t + "_micro"][bh] == ref[t + "_micro"], 32 if t == "v" and is_hybrid(p) else 16,
+                             axis=1 if t != "v" else 0)
             g, r = got[t + "_codes"][bh], ref[t + "_codes"]
             frac, dist = CMP.code_mismatch(g[same], r[same], 3)
             assert dist <= 1 and frac <= 1e-3, f"{what} {t}_codes: frac {frac:.2e} dist {dist}"

@@ -152,6 +152,31 @@ def test_vc_attn_4bit_end_to_end(case, perm_kind, variant):
             Hh.check_output(o[b, h].float().cpu().numpy(), ref, vmax)
 
 
+@pytest.mark.parametrize("perm_kind", ["identity", "random"])
+@pytest.mark.parametrize("case", SMALL, ids=[c[0] for c in SMALL])
+def test_hybrid_4bit_arrangement(case, perm_kind):
+    """bits = 4 with the ExpCast-FP8 probability: NVFP4 Q^ and K^, E2M1 values under power-of-two
+    factors per 32 tokens, the value product as an FP8 x FP4 block-scaled MMA.  vc_prep's value
+    codes and factors against the oracle, then vc_attn end to end against its emulation."""
+    _, B, H, N, d, grid = case
+    q, k, v = _inputs(B, H, N, d, grid, seed=51)
+    perm = None if perm_kind == "identity" else vc_inputs.random_perm(B, H, N, 10).cuda()
+    p = Params.make(B, H, N, d, grid, bits=4, p_format=vc.VC_P_EXPCAST_E4M3)
+    quant, work = Hh.run_prep(p, q, k, v, perm)
+    got = Hh.gpu_sections(p, quant)
+    o = torch.empty(B, H, N, d, dtype=torch.bfloat16, device="cuda")
+    vc.vc_attn(p, q, k, v, perm, o, quant, work)
+    vc.vc_poll_status(work)
+    vmax = float(v.float().abs().max())
+    for b in range(B):
+        for h in range(H):
+            bundle, cfg = Hh.oracle_prep(p, q, k, v, perm, b, h)
+            assert cfg.v_format == "mxfp4"
+            Hh.check_prep_head(p, got, b * H + h, bundle, what=f"hybrid head {b},{h}")
+            ref = OA.emulate_head(bundle, cfg, p_format=OA.P_EXPCAST)
+            Hh.check_output(o[b, h].float().cpu().numpy(), ref, vmax)
+
+
 def test_bad_arguments_are_rejected_on_the_host():
     p = Params.make(1, 1, 128, 128, (2, 8, 8))
     quant, work = alloc_buffers(p)
