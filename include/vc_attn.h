@@ -54,7 +54,13 @@ typedef enum {
 /* probability formats of the softmax stage (Sec. 3.3, App. A "Scope of ExpCast-FP8") */
 enum {
   VC_P_DEFAULT = 0,         /* ExpCast-FP8 at 8 bits, NVFP4 at 4 bits                */
-  VC_P_EXPCAST_E4M3 = 1,    /* Eq. 7: one FMA, the byte viewed as E4M3               */
+  /* Eq. 7: one FMA, the byte viewed as E4M3.  With bits = 4 this selects the HYBRID 4-bit
+   * arrangement: Q^ and K^ stay NVFP4, P is the ExpCast-FP8 code, and the value residual is
+   * stored as E2M1 under one power-of-two factor (an exponent byte, value 2^(byte - 127)) per
+   * channel and 32 consecutive permuted tokens, so that the value product runs as an
+   * FP8 x FP4 block-scaled MMA.  The factor is the smallest power of two that keeps the
+   * group's maximum inside the E2M1 range (no clipping); a group of zeros stores byte 0.   */
+  VC_P_EXPCAST_E4M3 = 1,
   VC_P_EXP_E4M3 = 2,        /* exponentiate, then cast to E4M3 (Fig. 4a upper box)   */
   VC_P_NVFP4 = 3,           /* E2M1 under a per-16-key E4M3 microscale               */
   /* the same result as VC_P_EXP_E4M3 up to the polynomial's error (relative 3.7e-6, so a code
@@ -112,6 +118,8 @@ typedef struct {
  *   v_means [BH][nb][d] bf16    block means / v_scale (4 bits: unscaled), App. B
  *   k_mean  [BH][d]  fp32       post-RoPE channel mean of K
  *   q_micro [BH][N_pad][d/16], k_micro [BH][N_pad][d/16], v_micro [BH][d][N_pad/16]  (4 bits)
+ * Hybrid 4-bit arrangement (bits = 4, p_format = VC_P_EXPCAST_E4M3): as at 4 bits, except
+ *   v_micro [BH][d][N_pad/32]   exponent bytes of the power-of-two factors, 32 tokens each
  */
 typedef struct {
   void *q_codes, *k_codes, *v_codes;

@@ -20,7 +20,9 @@ CASES = [("c2", 8, "kmeans"), ("c3", 8, "kmeans"), ("c3", 4, "random"), ("c4", 4
          ("c5_d64_n4096", 8, "random"), ("c5_d64_n4096", 4, "random"), ("c5_d128_n16384", 8, "kmeans"),
          ("c3", 8, "group"),          # the permutation from vc_group, as bench.py runs it
          ("c2", 8, "kmeans-int8"),    # the INT8 Q K^T arrangement
-         ("c4_2heads", 8, "random")]  # the longest sequence (929 key tiles, an odd count) at 8 bits
+         ("c4_2heads", 8, "random"),  # the longest sequence (929 key tiles, an odd count) at 8 bits
+         ("c3", 4, "group-hybrid"),   # the hybrid 4-bit arrangement (ExpCast-FP8 P over 4-bit Q, K, V)
+         ("c5_d64_n4096", 4, "random-hybrid")]
 
 vc_inputs.WORKLOADS.setdefault("c4_2heads", vc_inputs.Workload("c4_2heads", 1, 2, 118800, 128, (33, 45, 80), (8,), 1044, "field", True))
 
@@ -30,8 +32,10 @@ def test_fullsize_sampled_parity(name, bits, perm_kind):
     w = vc_inputs.WORKLOADS[name]
     q, k, v = vc_inputs.make_qkv(w, device="cuda")
     flags = vc.VC_FLAG_ALL | (vc.VC_FLAG_INT8_QK if perm_kind.endswith("int8") else 0)
-    p = Params.make(w.B, w.H, w.N, w.d, w.grid, bits=bits, flags=flags)
-    if perm_kind == "group":
+    hybrid = perm_kind.endswith("hybrid")
+    p = Params.make(w.B, w.H, w.N, w.d, w.grid, bits=bits, flags=flags,
+                    p_format=vc.VC_P_EXPCAST_E4M3 if hybrid else vc.VC_P_DEFAULT)
+    if perm_kind.startswith("group"):
         gwork = torch.empty(vc.vc_group_workspace_bytes(p), dtype=torch.uint8, device="cuda")
         cent = torch.zeros(w.B, w.H, 64, w.d, dtype=torch.float32, device="cuda")
         perm = torch.empty(w.B, w.H, w.N, dtype=torch.int32, device="cuda")
@@ -52,7 +56,7 @@ def test_fullsize_sampled_parity(name, bits, perm_kind):
     for (b, h) in [(0, 0), (w.B - 1, w.H - 1)]:
         ref, cfg = Hh.oracle_prep(p, q, k, v, perm, b, h)
         stats = Hh.check_prep_head(p, got, b * w.H + h, ref, what=f"{name} b{b} h{h}")
-        o_ref = OA.emulate_head(ref, cfg, rows=rows)
+        o_ref = OA.emulate_head(ref, cfg, rows=rows, p_format=OA.P_EXPCAST if hybrid else None)
         vmax = float(v[b, h].float().abs().max())
         m = Hh.check_output(o[b, h].float().cpu().numpy()[rows], o_ref, vmax)
         print(name, bits, (b, h), stats, m)
