@@ -31,6 +31,12 @@ def test_sizes_and_argument_validation_without_a_gpu():
     assert vc.vc_workspace_bytes(p) > 0
     p4 = Params.make(1, 40, 32760, 128, (21, 30, 52), bits=4)
     assert vc.vc_quant_bytes(p4) < 0.6 * qb
+    # the hybrid 4-bit arrangement: value factors per 32 tokens instead of 16, pipelined kernel only
+    ph = Params.make(1, 40, 32760, 128, (21, 30, 52), bits=4, p_format=vc.VC_P_EXPCAST_E4M3)
+    assert 0 < vc.vc_quant_bytes(p4) - vc.vc_quant_bytes(ph) <= 40 * n_pad * 128 // 32 + 2048
+    assert vc.vc_quant_bytes(Params.make(1, 2, 1024, 128, (4, 16, 16), bits=4, p_format=vc.VC_P_EXPCAST_E4M3, kernel_variant=1)) == 0
+    assert vc.vc_quant_bytes(Params.make(1, 2, 1024, 128, (4, 16, 16), bits=4, p_format=vc.VC_P_EXP_E4M3)) == 0
+    assert vc.vc_quant_bytes(Params.make(1, 2, 1024, 128, (4, 16, 16), bits=8, p_format=vc.VC_P_EXP_POLY_E4M3)) > 0
     for bad in (dict(d=100), dict(N=-1), dict(bits=3), dict(grid_t=20), dict(p_format=9)):
         pb = Params.make(1, 2, 1024, 128, (4, 16, 16))
         for k, v in bad.items():
