@@ -149,3 +149,26 @@ def test_8bit_kernel_variants_agree(shape, p_format):
     ref = OA.emulate_head(bundle, cfg, p_format=pf)
     for variant in (0, 1):
         Hh.check_output(outs[variant][0, 0].float().cpu().numpy(), ref, vmax)
+
+
+def test_sequence_parallel_wrapper_on_one_rank_is_vc_attn():
+    """The head-sharded wrapper with a single rank (no exchange) returns exactly what vc_attn does,
+    with and without the permutation from vc_group."""
+    from paper_2609_15810_b200 import sequence_parallel as SP
+    B, H, N, d, grid = 1, 2, 640, 128, (5, 8, 16)
+    w = vc_inputs.Workload("t", B, H, N, d, grid, (8,), 77, "gauss")
+    q, k, v = [t.cuda() for t in vc_inputs.make_qkv(w)]
+    for group_k in (0, 8):
+        got = SP.vc_attn_sequence_parallel(q, k, v, grid, bits=8, group_k=group_k, group_iters=2)
+        p = Params.make(B, H, N, d, grid, bits=8)
+        perm = None
+        if group_k:
+            gwork = torch.empty(vc.vc_group_workspace_bytes(p), dtype=torch.uint8, device="cuda")
+            cent = torch.zeros(B, H, group_k, d, dtype=torch.float32, device="cuda")
+            perm = torch.empty(B, H, N, dtype=torch.int32, device="cuda")
+            vc.vc_group(p, v, group_k, 2, False, cent, perm, gwork)
+        quant, work = alloc_buffers(p)
+        o = torch.empty(B, H, N, d, dtype=torch.bfloat16, device="cuda")
+        vc.vc_attn(p, q, k, v, perm, o, quant, work)
+        vc.vc_poll_status(work)
+        assert torch.equal(got, o)
