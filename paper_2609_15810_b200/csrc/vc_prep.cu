@@ -91,7 +91,10 @@ __global__ void rope_table_kernel(float2* tab, RopeDesc rd, double theta) {
 // (One bulk-async copy per gathered row was tried instead of cp.async: 128 small copies per
 // block kept the copy engine, not HBM, busy.)
 constexpr int kThreads = 256;      // threads of the column-sum and V passes
-constexpr int kRowThreads = 128;   // threads of the row-per-thread Q/K pass
+constexpr int kRowThreads = 128;   // rows of a Q/K item (threads of the pass = rows x threads per row)
+#ifndef VC_PREP_TPR
+#define VC_PREP_TPR 2
+#endif
 
 template <int D> struct Geo {
   static constexpr int pitch = 2 * D + 16;          // row pitch of the thread-per-row layout
@@ -218,31 +221,49 @@ template <> struct RopeSplit<64> { static constexpr int p1 = 12, p2 = 22; };    
 // `red` is [2][4] floats and `kmean_s` [D] floats of compute-warp scratch.
 // Q and K run through one copy of the row body (TENSOR is a run-time argument): the unrolled body
 // is tens of KB of code, and two copies of it thrash the instruction cache.
-template <int D, int STAGE>
+//
+// TPR = threads per row.  With TPR = 1 a thread holds all D channels of its row.  With TPR = 2 the
+// lanes 0..15 of a warp hold channels [0, D/2) of 16 rows and the lanes 16..31 channels [D/2, D)
+// of the same rows: half the registers per thread, so twice the warps per SM; the last Hadamard
+// level crosses the two halves with one shuffle per value.  RoPE pairs and NVFP4 groups stay
+// thread-local either way.
+template <int TPR> __device__ __forceinline__ int qk_row_of(int tid) {
+  return TPR == 1 ? tid : 16 * (tid >> 5) + (tid & 15);
+}
+template <int TPR> __device__ __forceinline__ int qk_part_of(int tid) { return TPR == 1 ? 0 : (tid >> 4) & 1; }
+
+template <int D> __device__ __forceinline__ constexpr int rope_axis_of(int p) {
+  return p < RopeSplit<D>::p1 ? 0 : (p < RopeSplit<D>::p2 ? 1 : 2);
+}
+
+template <int D, int STAGE, int TPR>
 __device__ __forceinline__ void qk_row_item(const PrepArgs& a, const int TENSOR /*0 = Q, 1 = K*/, const unsigned char* stage,
                                             unsigned char* out_tile, float* red, float* kmean_s, const float2* tab, int bh,
                                             int blk, int iter, bool new_head, int src_row) {
+  constexpr int C = D / TPR;                       // channels per thread
+  constexpr int NT = kRowThreads * TPR;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int row = qk_row_of<TPR>(tid), part = qk_part_of<TPR>(tid);
   const bool do_rope = a.flags & VC_FLAG_ROPE;
   const bool do_had = a.flags & VC_FLAG_HADAMARD;
   const bool center = TENSOR == 1 && (a.flags & VC_FLAG_K_SMOOTH);
   const bool valid = src_row >= 0;               // src_row: the input row behind this thread's row
   const int src = valid ? src_row : 0;           // (RoPE acts at the source position)
-  uint4 raw[D / 8];
+  uint4 raw[C / 8];
 #pragma unroll
-  for (int i = 0; i < D / 8; ++i) {
+  for (int i = 0; i < C / 8; ++i) {
     raw[i] = make_uint4(0, 0, 0, 0);
-    if (valid) raw[i] = *reinterpret_cast<const uint4*>(stage + tid * Geo<D>::pitch + 16 * i);
+    if (valid) raw[i] = *reinterpret_cast<const uint4*>(stage + row * Geo<D>::pitch + part * (2 * C) + 16 * i);
   }
   if (center && new_head) {
     __syncthreads();                               // everyone is done with the previous head's mean
-    for (int c = tid; c < D; c += kRowThreads) kmean_s[c] = a.k_mean[(size_t)bh * D + c];
+    for (int c = tid; c < D; c += NT) kmean_s[c] = a.k_mean[(size_t)bh * D + c];
     __syncthreads();
   }
 
-  float x[D];
+  float x[C];
 #pragma unroll
-  for (int i = 0; i < D / 8; ++i) {
+  for (int i = 0; i < C / 8; ++i) {
     const unsigned int w[4] = {raw[i].x, raw[i].y, raw[i].z, raw[i].w};
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
@@ -254,47 +275,63 @@ __device__ __forceinline__ void qk_row_item(const PrepArgs& a, const int TENSOR 
     int tt, ty, tx;
     grid_pos(a.rd, src, tt, ty, tx);
     // entry of pair p of axis ax: off[ax] + pos[ax] * pairs[ax] + (p - pair_start[ax])
-    const int e0 = a.rd.off[0] + tt * a.rd.pairs[0] - a.rd.pair_start[0];
-    const int e1 = a.rd.off[1] + ty * a.rd.pairs[1] - a.rd.pair_start[1];
-    const int e2 = a.rd.off[2] + tx * a.rd.pairs[2] - a.rd.pair_start[2];
-    if (a.rope_default) {                       // compile-time pair boundaries: one load per pair
+    const int e[3] = {a.rd.off[0] + tt * a.rd.pairs[0] - a.rd.pair_start[0],
+                      a.rd.off[1] + ty * a.rd.pairs[1] - a.rd.pair_start[1],
+                      a.rd.off[2] + tx * a.rd.pairs[2] - a.rd.pair_start[2]};
+    const int p0 = part * (C / 2);               // first pair of this thread
+    if (a.rope_default) {
+      // compile-time pair boundaries: the axis of local pair i is known for either part, so the
+      // table base of each (axis in part 0, axis in part 1) combination is selected once per row
+      int base[3][3];
 #pragma unroll
-      for (int p = 0; p < D / 2; ++p) {
-        const int e = p < RopeSplit<D>::p1 ? e0 : (p < RopeSplit<D>::p2 ? e1 : e2);
-        const float2 cs = tab[e + p];
-        const float x0 = x[2 * p], x1 = x[2 * p + 1];
-        x[2 * p] = x0 * cs.x - x1 * cs.y;
-        x[2 * p + 1] = x0 * cs.y + x1 * cs.x;
+      for (int a0 = 0; a0 < 3; ++a0)
+#pragma unroll
+        for (int a1 = 0; a1 < 3; ++a1) base[a0][a1] = (part ? e[a1] : e[a0]) + p0;
+#pragma unroll
+      for (int i = 0; i < C / 2; ++i) {
+        const float2 cs = tab[base[rope_axis_of<D>(i)][rope_axis_of<D>(TPR == 1 ? i : C / 2 + i)] + i];
+        const float x0 = x[2 * i], x1 = x[2 * i + 1];
+        x[2 * i] = x0 * cs.x - x1 * cs.y;
+        x[2 * i + 1] = x0 * cs.y + x1 * cs.x;
       }
     } else {
 #pragma unroll
-      for (int p = 0; p < D / 2; ++p) {
-        const int e = p < a.rd.pair_start[1] ? e0 : (p < a.rd.pair_start[2] ? e1 : e2);
-        const float2 cs = tab[e + p];
-        const float x0 = x[2 * p], x1 = x[2 * p + 1];
-        x[2 * p] = x0 * cs.x - x1 * cs.y;
-        x[2 * p + 1] = x0 * cs.y + x1 * cs.x;
+      for (int i = 0; i < C / 2; ++i) {
+        const int p = p0 + i;
+        const int eb = p < a.rd.pair_start[1] ? e[0] : (p < a.rd.pair_start[2] ? e[1] : e[2]);
+        const float2 cs = tab[eb + p];
+        const float x0 = x[2 * i], x1 = x[2 * i + 1];
+        x[2 * i] = x0 * cs.x - x1 * cs.y;
+        x[2 * i + 1] = x0 * cs.y + x1 * cs.x;
       }
     }
   }
   if (center && valid) {
+    const float4* km = reinterpret_cast<const float4*>(kmean_s + part * C);
 #pragma unroll
-    for (int c4 = 0; c4 < D / 4; ++c4) {
-      const float4 m = reinterpret_cast<const float4*>(kmean_s)[c4];
+    for (int c4 = 0; c4 < C / 4; ++c4) {
+      const float4 m = km[c4];
       x[4 * c4] -= m.x; x[4 * c4 + 1] -= m.y; x[4 * c4 + 2] -= m.z; x[4 * c4 + 3] -= m.w;
     }
   }
   if (do_had) {
 #pragma unroll
-    for (int sft = 1; sft < D; sft <<= 1) {
+    for (int sft = 1; sft < C; sft <<= 1) {
 #pragma unroll
-      for (int c = 0; c < D; ++c) {
+      for (int c = 0; c < C; ++c) {
         if (!(c & sft)) {
           const float u = x[c], v = x[c | sft];
           x[c] = u + v;
           x[c | sft] = u - v;
         }
       }
+    }
+    if constexpr (TPR == 2) {
+      // the level that pairs channel c with c + D/2: the lower half takes mine + theirs, the upper
+      // half theirs - mine (one fused multiply-add with +-1, exact)
+      const float sgn = part ? -1.0f : 1.0f;
+#pragma unroll
+      for (int c = 0; c < C; ++c) x[c] = fmaf(x[c], sgn, __shfl_xor_sync(0xffffffffu, x[c], 16));
     }
   }
   const float rs = do_had ? (D == 128 ? 0.08838834764831845f : 0.125f) : 1.0f;   // 1/sqrt(D)
@@ -303,21 +340,22 @@ __device__ __forceinline__ void qk_row_item(const PrepArgs& a, const int TENSOR 
   if constexpr (STAGE != kStageQuant4) {
     float m0 = 0.f, m1 = 0.f;
 #pragma unroll
-    for (int c = 0; c < D; c += 4) {
+    for (int c = 0; c < C; c += 4) {
       m0 = max3(m0, fabsf(x[c]), fabsf(x[c + 1]));
       m1 = max3(m1, fabsf(x[c + 2]), fabsf(x[c + 3]));
     }
     amax = warp_max(fmaxf(m0, m1) * rs);        // max and the (positive) scale commute exactly
-    float* rbuf = red + 4 * (iter & 1);         // alternate buffers: one barrier per item suffices
+    float* rbuf = red + 8 * (iter & 1);         // alternate buffers: one barrier per item suffices
     if (lane == 0) rbuf[warp] = amax;
     __syncthreads();
     amax = fmaxf(fmaxf(rbuf[0], rbuf[1]), fmaxf(rbuf[2], rbuf[3]));
+    if constexpr (TPR == 2) amax = fmaxf(amax, fmaxf(fmaxf(rbuf[4], rbuf[5]), fmaxf(rbuf[6], rbuf[7])));
   }
   if constexpr (STAGE == kStageAmax) {
     if (tid == 0) atomicMax(&a.qk_amax[TENSOR * a.BH + bh], __float_as_uint(amax));
     return;
   }
-  const size_t row_g = (size_t)bh * a.n_pad + (size_t)blk * kBlock + tid;
+  const size_t row_g = (size_t)bh * a.n_pad + (size_t)blk * kBlock + row;
 
   if constexpr (STAGE == kStageQuant8 || STAGE == kStageQuant8I) {
     // E4M3 codes (top value 448), or INT8 codes (top value 127; the INT8 Q K^T of Fig. 3)
@@ -327,10 +365,10 @@ __device__ __forceinline__ void qk_row_item(const PrepArgs& a, const int TENSOR 
     if (tid == 0) (TENSOR == 0 ? a.q_scale : a.k_scale)[(size_t)bh * a.nb + blk] = amax > 0.f ? amax / top : 1.0f;
     // codes go to the swizzled output tile; the CTA copies it out with coalesced stores
     constexpr int CPR = D / 16;
-    uint4* dst = reinterpret_cast<uint4*>(out_tile + tid * D);
-    const int sw = (tid / (8 / CPR)) & (CPR - 1);
+    uint4* dst = reinterpret_cast<uint4*>(out_tile + row * D);
+    const int sw = (row / (8 / CPR)) & (CPR - 1);
 #pragma unroll
-    for (int i = 0; i < D / 16; ++i) {
+    for (int i = 0; i < C / 16; ++i) {
       unsigned int w[4];
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
@@ -347,7 +385,7 @@ __device__ __forceinline__ void qk_row_item(const PrepArgs& a, const int TENSOR 
           w[j] = lo | (hi << 16);
         }
       }
-      dst[i ^ sw] = make_uint4(w[0], w[1], w[2], w[3]);
+      dst[(part * (C / 16) + i) ^ sw] = make_uint4(w[0], w[1], w[2], w[3]);
     }
   }
 
@@ -355,11 +393,12 @@ __device__ __forceinline__ void qk_row_item(const PrepArgs& a, const int TENSOR 
     // NVFP4: outer scale g per (b, h), microscale per token per 16 channels
     const float g = (TENSOR == 0 ? a.q_scale : a.k_scale)[bh];
     const float inv6 = 1.0f / (6.0f * g);
-    unsigned int codes[D / 8], micro[D / 64];
+    constexpr int MB = C / 16;                   // microscale bytes of this thread
+    unsigned int codes[C / 8], micro[(MB + 3) / 4];
 #pragma unroll
-    for (int i = 0; i < D / 64; ++i) micro[i] = 0;
+    for (int i = 0; i < (MB + 3) / 4; ++i) micro[i] = 0;
 #pragma unroll
-    for (int gq = 0; gq < D / 16; ++gq) {
+    for (int gq = 0; gq < C / 16; ++gq) {
       float m = 0.f;
 #pragma unroll
       for (int c = 0; c < 16; ++c) { x[16 * gq + c] *= rs; m = fmaxf(m, fabsf(x[16 * gq + c])); }
@@ -380,13 +419,18 @@ __device__ __forceinline__ void qk_row_item(const PrepArgs& a, const int TENSOR 
       }
     }
     constexpr int CPR = D / 32;
-    uint4* dst = reinterpret_cast<uint4*>(out_tile + tid * (D / 2));
-    const int sw = (tid / (8 / CPR)) & (CPR - 1);
+    uint4* dst = reinterpret_cast<uint4*>(out_tile + row * (D / 2));
+    const int sw = (row / (8 / CPR)) & (CPR - 1);
 #pragma unroll
-    for (int i = 0; i < D / 32; ++i) dst[i ^ sw] = make_uint4(codes[4 * i], codes[4 * i + 1], codes[4 * i + 2], codes[4 * i + 3]);
-    unsigned int* mdst = reinterpret_cast<unsigned int*>((TENSOR == 0 ? a.q_micro : a.k_micro) + row_g * (D / 16));
+    for (int i = 0; i < C / 32; ++i) dst[(part * (C / 32) + i) ^ sw] = make_uint4(codes[4 * i], codes[4 * i + 1], codes[4 * i + 2], codes[4 * i + 3]);
+    uint8_t* mrow = (TENSOR == 0 ? a.q_micro : a.k_micro) + row_g * (D / 16) + part * MB;
+    if constexpr (MB % 4 == 0) {
 #pragma unroll
-    for (int i = 0; i < D / 64; ++i) mdst[i] = micro[i];
+      for (int i = 0; i < MB / 4; ++i) reinterpret_cast<unsigned int*>(mrow)[i] = micro[i];
+    } else {
+      static_assert(MB == 2, "microscale bytes per thread");
+      *reinterpret_cast<unsigned short*>(mrow) = (unsigned short)micro[0];
+    }
   }
 }
 
@@ -729,19 +773,21 @@ __global__ void prep_finalize_kernel(const PrepArgs a, int which) {
 // rows taken from a small ring of permutation slices in shared memory), a thread then reads its
 // row from the padded tile; codes leave through a swizzled tile in the same way.
 // Shared memory: [2 stages x 128 x pitch][out tile 128 x D][src ring 3 x 128][scratch][RoPE table].
-template <int D, int STAGE>
-__global__ void __launch_bounds__(kRowThreads, 2) prep_qk_kernel(const PrepArgs a, int n_items, int nh, int z0) {
+template <int D, int STAGE, int TPR>
+__global__ void __launch_bounds__(kRowThreads * TPR, 2) prep_qk_kernel(const PrepArgs a, int n_items, int nh, int z0) {
+  constexpr int NT = kRowThreads * TPR;
   constexpr int kRowBytes = STAGE == kStageQuant4 ? D / 2 : D;      // code bytes per row
   constexpr int CPR = kRowBytes / 16;                                // 16-byte chunks per code row
   extern __shared__ __align__(128) unsigned char smem[];
   unsigned char* out_tile = smem + 2 * Geo<D>::stage_bytes;
   int* src_ring = reinterpret_cast<int*>(out_tile + kBlock * D);     // [3][128]
-  float* red = reinterpret_cast<float*>(src_ring + 3 * kBlock);      // [2][4]
+  float* red = reinterpret_cast<float*>(src_ring + 3 * kBlock);      // [2][8]
   float* kmean_s = red + 16;                                         // [D]
   const float2* tab = stage_rope_table(a, reinterpret_cast<unsigned char*>(kmean_s + D));
   const int tid = threadIdx.x;
-  auto fetch = [&](int item) -> int {        // input row behind my row of the item, -1 if none
-    if (item >= n_items) return -1;
+  const int my_row = qk_row_of<TPR>(tid);
+  auto fetch = [&](int item) -> int {        // input row behind row `tid` of the item, -1 if none
+    if (item >= n_items || tid >= kBlock) return -1;
     const Item w = decode_item(item, a.nb, nh, a.bh0);
     const int t = w.blk * kBlock + tid;
     if (t >= a.N) return -1;
@@ -756,16 +802,18 @@ __global__ void __launch_bounds__(kRowThreads, 2) prep_qk_kernel(const PrepArgs 
       const __nv_bfloat16* base = ((w.z + z0) == 0 ? a.q : a.k) + b * a.stride_b + h * a.stride_h + 8 * (tid % (D / 8));
       unsigned char* dst = smem + st * Geo<D>::stage_bytes + 16 * (tid % (D / 8));
 #pragma unroll
-      for (int c = 0; c < D / 8; ++c) {
-        const int row = (c * kRowThreads + tid) / (D / 8);
+      for (int c = 0; c < kBlock * (D / 8) / NT; ++c) {
+        const int row = (c * NT + tid) / (D / 8);
         const int sr = src[row];
         if (sr >= 0) cp_async16(dst + row * Geo<D>::pitch, base + (int64_t)sr * a.stride_n);
       }
     }
     cp_async_commit();
   };
-  src_ring[tid] = fetch(blockIdx.x);
-  src_ring[kBlock + tid] = fetch(blockIdx.x + gridDim.x);
+  if (tid < kBlock) {
+    src_ring[tid] = fetch(blockIdx.x);
+    src_ring[kBlock + tid] = fetch(blockIdx.x + gridDim.x);
+  }
   int nxt = fetch(blockIdx.x + 2 * gridDim.x);
   __syncthreads();
   issue(blockIdx.x, 0, src_ring);
@@ -773,21 +821,21 @@ __global__ void __launch_bounds__(kRowThreads, 2) prep_qk_kernel(const PrepArgs 
   for (int item = blockIdx.x; item < n_items; item += gridDim.x, ++i) {
     cp_async_wait<0>();                       // my chunks of item i have landed ...
     __syncthreads();                          // ... and everyone's; item i-1 is finished everywhere
-    src_ring[((i + 2) % 3) * kBlock + tid] = nxt;
+    if (tid < kBlock) src_ring[((i + 2) % 3) * kBlock + tid] = nxt;
     nxt = fetch(item + 3 * gridDim.x);
     issue(item + gridDim.x, (i + 1) & 1, src_ring + ((i + 1) % 3) * kBlock);
     const Item w = decode_item(item, a.nb, nh, a.bh0);
     const unsigned char* stage = smem + (i & 1) * Geo<D>::stage_bytes;
-    const int s0 = src_ring[(i % 3) * kBlock + tid];
+    const int s0 = src_ring[(i % 3) * kBlock + my_row];
     const int tensor = w.z + z0;
-    qk_row_item<D, STAGE>(a, tensor, stage, out_tile, red, kmean_s, tab, w.bh, w.blk, i, tensor == 1 && w.bh != last_bh, s0);
+    qk_row_item<D, STAGE, TPR>(a, tensor, stage, out_tile, red, kmean_s, tab, w.bh, w.blk, i, tensor == 1 && w.bh != last_bh, s0);
     if (tensor == 1) last_bh = w.bh;
     if constexpr (STAGE != kStageAmax) {
       __syncthreads();                        // the code tile is complete
       uint8_t* gdst = (w.z + z0 == 0 ? a.q_codes : a.k_codes) + ((size_t)w.bh * a.n_pad + (size_t)w.blk * kBlock) * kRowBytes;
 #pragma unroll
-      for (int c = 0; c < CPR; ++c) {
-        const int idx = c * kRowThreads + tid, row = idx / CPR, chunk = idx % CPR;
+      for (int c = 0; c < CPR * kBlock / NT; ++c) {
+        const int idx = c * NT + tid, row = idx / CPR, chunk = idx % CPR;
         const int sw = (row / (8 / CPR)) & (CPR - 1);
         const uint4 v = *reinterpret_cast<const uint4*>(out_tile + row * kRowBytes + ((chunk ^ sw) << 4));
         *reinterpret_cast<uint4*>(gdst + (size_t)idx * 16) = v;
@@ -819,6 +867,7 @@ cudaError_t run(const Problem& pr, PrepArgs a, const WorkLayout& wl, uint8_t* wo
   const size_t row_smem = 2 * (size_t)Geo<D>::stage_bytes + (size_t)kBlock * D + 3 * kBlock * 4 + 64 + D * 4 + rope_bytes;
   const size_t v_smem = 3 * (size_t)kBlock * 2 * D + 8 * D * 4;
   constexpr int kQuant = BITS == 8 ? kStageQuant8 : kStageQuant4;
+  constexpr int kTpr = VC_PREP_TPR;            // threads per Q/K row
   constexpr int kVQuant = BITS == 8 ? kVQuant8 : kVQuant4;
   cudaError_t e;
   if ((e = allow_smem(prep_kcolsum_kernel<D>, colsum_smem)) != cudaSuccess) return e;
@@ -826,9 +875,9 @@ cudaError_t run(const Problem& pr, PrepArgs a, const WorkLayout& wl, uint8_t* wo
   if ((e = allow_smem(prep_v_kernel<D, kVQuant>, v_smem)) != cudaSuccess) return e;
   if (BITS == 4 && (e = allow_smem(prep_v_kernel<D, kVQuant4M>, v_smem)) != cudaSuccess) return e;
   const bool v_pow2 = hybrid4(pr);           // 4-bit values under power-of-two factors per 32 tokens
-  if ((e = allow_smem(prep_qk_kernel<D, kQuant>, row_smem)) != cudaSuccess) return e;
-  if (BITS == 8 && (e = allow_smem(prep_qk_kernel<D, kStageQuant8I>, row_smem)) != cudaSuccess) return e;
-  if (BITS == 4 && (e = allow_smem(prep_qk_kernel<D, kStageAmax>, row_smem)) != cudaSuccess) return e;
+  if ((e = allow_smem(prep_qk_kernel<D, kQuant, kTpr>, row_smem)) != cudaSuccess) return e;
+  if (BITS == 8 && (e = allow_smem(prep_qk_kernel<D, kStageQuant8I, kTpr>, row_smem)) != cudaSuccess) return e;
+  if (BITS == 4 && (e = allow_smem(prep_qk_kernel<D, kStageAmax, kTpr>, row_smem)) != cudaSuccess) return e;
   if ((e = cudaMemsetAsync(work + wl.status, 0, 4, s)) != cudaSuccess) return e;
   if ((e = cudaMemsetAsync(work + wl.amax, 0, wl.amax_bytes, s)) != cudaSuccess) return e;
   if (a.flags & VC_FLAG_ROPE) {
@@ -847,18 +896,18 @@ cudaError_t run(const Problem& pr, PrepArgs a, const WorkLayout& wl, uint8_t* wo
       count_launches(1);
     }
     prep_v_kernel<D, kVStats><<<persistent_grid(per), kThreads, v_smem, s>>>(a, per, nh);
-    if (BITS == 4) { prep_qk_kernel<D, kStageAmax><<<persistent_grid(per), kRowThreads, row_smem, s>>>(a, per, nh, 0); count_launches(1); }
+    if (BITS == 4) { prep_qk_kernel<D, kStageAmax, kTpr><<<persistent_grid(per), kRowThreads * kTpr, row_smem, s>>>(a, per, nh, 0); count_launches(1); }
     prep_finalize_kernel<D, BITS><<<nh, D, 0, s>>>(a, 0);
     count_launches(2);
     if (BITS == 4) {
-      prep_qk_kernel<D, kStageAmax><<<persistent_grid(per), kRowThreads, row_smem, s>>>(a, per, nh, 1);
+      prep_qk_kernel<D, kStageAmax, kTpr><<<persistent_grid(per), kRowThreads * kTpr, row_smem, s>>>(a, per, nh, 1);
       prep_finalize_kernel<D, BITS><<<nh, 32, 0, s>>>(a, 1);
       count_launches(2);
     }
     if (BITS == 8 && (a.flags & VC_FLAG_INT8_QK))
-      prep_qk_kernel<D, kStageQuant8I><<<persistent_grid(2 * per), kRowThreads, row_smem, s>>>(a, 2 * per, nh, 0);
+      prep_qk_kernel<D, kStageQuant8I, kTpr><<<persistent_grid(2 * per), kRowThreads * kTpr, row_smem, s>>>(a, 2 * per, nh, 0);
     else
-      prep_qk_kernel<D, kQuant><<<persistent_grid(2 * per), kRowThreads, row_smem, s>>>(a, 2 * per, nh, 0);
+      prep_qk_kernel<D, kQuant, kTpr><<<persistent_grid(2 * per), kRowThreads * kTpr, row_smem, s>>>(a, 2 * per, nh, 0);
     if (BITS == 4 && v_pow2)
       prep_v_kernel<D, kVQuant4M><<<persistent_grid(per), kThreads, v_smem, s>>>(a, per, nh);
     else
