@@ -194,6 +194,7 @@ def main():
     ap.add_argument("--ref-rows", type=int, default=1024)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-others", action="store_true", help="skip the short measurement of the 4-bit arrangements")
     ap.add_argument("--no-sdpa", action="store_true")
     ap.add_argument("--data", default="workload", choices=["workload", "gauss"],
                     help="gauss: same shapes, inputs drawn with three randn calls (for profiler runs, where the\n"
@@ -307,6 +308,35 @@ def main():
                "h2d_bytes_per_step": 3 * nbytes + (perm.numel() * 4 if perm is not None else 0),
                "d2h_bytes_per_step": nbytes, "steps": n_e2e}
 
+    # the 4-bit arrangements on the same inputs and permutation, for the record (the metric names
+    # both widths); the headline numbers above stay those of the arrangement asked for
+    others = None
+    if (world == 1 and not args.no_others and args.bits == 8 and args.p_format == "default" and not args.int8_qk
+            and args.variant == 0):
+        others = []
+        for name, kw in (("4-bit: NVFP4 Q, K, V and P", dict(bits=4)),
+                         ("4-bit hybrid: NVFP4 QK^T, ExpCast-FP8 P, FP8 x FP4 PV", dict(bits=4, p_format=1))):
+            p2 = Params.make(w.B, w.H, w.N, w.d, w.grid, **kw)
+            quant2, work2 = alloc_buffers(p2, device=dev)
+            for _ in range(3):
+                vc.vc_attn(p2, q, k, v, perm, o, quant2, work2)
+            n2 = max(3, min(args.steps, 10))
+            ev2 = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(n2)]
+            torch.cuda.synchronize()
+            for s in range(n2):
+                ev2[s][0].record(stream)
+                vc.vc_prep(p2, q, k, v, perm, quant2, work2)
+                ev2[s][1].record(stream)
+                vc.vc_attn_fwd(p2, quant2, o, work2)
+                ev2[s][2].record(stream)
+            torch.cuda.synchronize()
+            vc.vc_poll_status(work2)
+            pm = statistics.mean(e[0].elapsed_time(e[1]) for e in ev2)
+            am = statistics.mean(e[1].elapsed_time(e[2]) for e in ev2)
+            others.append({"arrangement": name, "steps": n2, "prep_ms": pm, "attn_ms": am,
+                           "attn_tflops": w.flops / (am * 1e-3) / 1e12, "step_tflops": w.flops / ((pm + am) * 1e-3) / 1e12})
+            del quant2, work2
+
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
@@ -338,7 +368,7 @@ def main():
         "config": {"workload": w.name, "B": w.B, "H": w.H, "N": w.N, "d": w.d, "grid": list(w.grid),
                    "bits": args.bits, "p_format": args.p_format, "perm": args.perm, "data": args.data, "l2": "inputs larger than L2 (Q+K+V = %.0f MB)" % (3 * q.numel() * 2 / 1e6),
                    "step": "vc_prep + vc_attn_fwd" + (" (+ vc_group every 4th step)" if args.perm == "group" else "")},
-        "clocks": clocks, "gpu_launches": launches, "e2e": e2e,
+        "clocks": clocks, "gpu_launches": launches, "e2e": e2e, "other_arrangements": others,
         "roofline": {"bound": "tensor", "kernel": "vc_attn_fwd", "achieved": achieved, "peak": peak, "unit": UNIT,
                      "frac": achieved / peak, "traffic": traffic,
                      "traffic_source": "ncu dram__bytes_read+write of this kernel on B2 H16 N16384 d128 "
