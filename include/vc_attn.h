@@ -59,7 +59,8 @@ enum {
    * stored as E2M1 under one power-of-two factor (an exponent byte, value 2^(byte - 127)) per
    * channel and 32 consecutive permuted tokens, so that the value product runs as an
    * FP8 x FP4 block-scaled MMA.  The factor is the smallest power of two that keeps the
-   * group's maximum inside the E2M1 range (no clipping); a group of zeros stores byte 0.   */
+   * group's maximum inside the E2M1 range (no clipping); a group of zeros stores byte 0.
+   * vc_attn_fwd then wants the bundle 32-byte aligned; kernel_variant must be 0.            */
   VC_P_EXPCAST_E4M3 = 1,
   VC_P_EXP_E4M3 = 2,        /* exponentiate, then cast to E4M3 (Fig. 4a upper box)   */
   VC_P_NVFP4 = 3,           /* E2M1 under a per-16-key E4M3 microscale               */

@@ -164,6 +164,8 @@ vc_status vc_attn_fwd(const vc_params* p, const void* quant, void* o, void* work
   if (st != VC_OK) return st;
   if (!quant || !o || !workspace) return VC_ERR_INVALID_ARG;
   if (misaligned(quant) || misaligned(o) || misaligned(workspace)) return VC_ERR_INVALID_ARG;
+  // the 4-bit tensor map of the hybrid arrangement's value codes wants a 32-byte aligned base
+  if (hybrid4(pr) && ((uintptr_t)quant & 31)) return VC_ERR_INVALID_ARG;
   QuantLayout ql = quant_layout(pr);
   WorkLayout wl = work_layout(pr);
   cudaError_t e = launch_attn_fwd(pr, ql, wl, (const uint8_t*)quant, o, (uint8_t*)workspace,

@@ -172,3 +172,25 @@ def test_sequence_parallel_wrapper_on_one_rank_is_vc_attn():
         vc.vc_attn(p, q, k, v, perm, o, quant, work)
         vc.vc_poll_status(work)
         assert torch.equal(got, o)
+
+
+@pytest.mark.parametrize("flags", [0, vc.VC_FLAG_ROPE | vc.VC_FLAG_HADAMARD, vc.VC_FLAG_K_SMOOTH | vc.VC_FLAG_V_SMOOTH])
+def test_hybrid_4bit_stage_switches_and_parameters(flags):
+    """The hybrid 4-bit arrangement with stages switched off, a non-default softmax scale and
+    ExpCast offset, and a bundle that is only 16-byte aligned (rejected)."""
+    B, H, N, d, grid = 1, 2, 333, 128, (3, 3, 37)
+    w = vc_inputs.Workload("t", B, H, N, d, grid, (4,), 91, "gauss")
+    q, k, v = [t.cuda() for t in vc_inputs.make_qkv(w)]
+    p = Params.make(B, H, N, d, grid, bits=4, p_format=vc.VC_P_EXPCAST_E4M3, flags=flags, softmax_scale=0.11, beta=-0.2)
+    quant, work = alloc_buffers(p)
+    o = torch.empty(B, H, N, d, dtype=torch.bfloat16, device="cuda")
+    vc.vc_attn(p, q, k, v, None, o, quant, work)
+    vc.vc_poll_status(work)
+    vmax = float(v.float().abs().max())
+    for h in range(H):
+        bundle, cfg = Hh.oracle_prep(p, q, k, v, None, 0, h)
+        ref = OA.emulate_head(bundle, cfg, p_format=OA.P_EXPCAST, softmax_scale=0.11, beta=-0.2)
+        Hh.check_output(o[0, h].float().cpu().numpy(), ref, vmax)
+    shifted = torch.empty(quant.numel() + 16, dtype=torch.uint8, device="cuda")[16:]
+    with pytest.raises(vc.VcError):
+        vc.vc_attn_fwd(p, shifted, o, work)
