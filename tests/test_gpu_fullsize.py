@@ -22,7 +22,8 @@ CASES = [("c2", 8, "kmeans"), ("c3", 8, "kmeans"), ("c3", 4, "random"), ("c4", 4
          ("c2", 8, "kmeans-int8"),    # the INT8 Q K^T arrangement
          ("c4_2heads", 8, "random"),  # the longest sequence (929 key tiles, an odd count) at 8 bits
          ("c3", 4, "group-hybrid"),   # the hybrid 4-bit arrangement (ExpCast-FP8 P over 4-bit Q, K, V)
-         ("c5_d64_n4096", 4, "random-hybrid")]
+         ("c5_d64_n4096", 4, "random-hybrid"),
+         ("c4_2heads", 4, "random-hybrid")]   # 929 key tiles through the FP8 x FP4 value product
 
 vc_inputs.WORKLOADS.setdefault("c4_2heads", vc_inputs.Workload("c4_2heads", 1, 2, 118800, 128, (33, 45, 80), (8,), 1044, "field", True))
 
