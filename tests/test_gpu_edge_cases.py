@@ -100,7 +100,7 @@ def test_strided_inputs_through_vc_attn():
 
 
 @pytest.mark.parametrize("shape", [(2, 6, 300, 64, (3, 10, 10)), (1, 3, 257, 128, (1, 1, 257))], ids=["12_heads_6_groups", "3_heads"])
-@pytest.mark.parametrize("bits", [8, 4])
+@pytest.mark.parametrize("bits", [8, 4, "4-hybrid"])
 def test_host_entry_point_equals_the_device_path(shape, bits):
     """vc_attn_host (pinned host buffers in and out, pipelined over groups of heads) gives exactly
     the output of vc_attn on the same inputs, with and without a permutation."""
@@ -108,7 +108,8 @@ def test_host_entry_point_equals_the_device_path(shape, bits):
     w = vc_inputs.Workload("t", B, H, N, d, grid, (8,), 77, "gauss")
     q, k, v = [t.cuda() for t in vc_inputs.make_qkv(w)]
     for perm in (None, vc_inputs.random_perm(B, H, N, 3).cuda()):
-        p = Params.make(B, H, N, d, grid, bits=bits)
+        p = (Params.make(B, H, N, d, grid, bits=4, p_format=vc.VC_P_EXPCAST_E4M3) if bits == "4-hybrid"
+             else Params.make(B, H, N, d, grid, bits=bits))
         quant, work = alloc_buffers(p)
         o_ref = torch.empty(B, H, N, d, dtype=torch.bfloat16, device="cuda")
         vc.vc_attn(p, q, k, v, perm, o_ref, quant, work)
