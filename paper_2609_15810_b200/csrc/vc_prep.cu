@@ -460,7 +460,11 @@ __device__ __forceinline__ void v_item(const PrepArgs& a, const unsigned char* s
   const size_t mu_at = ((size_t)bh * a.nb + blk) * D + 2 * cp;
   float mu0 = 0.f, mu1 = 0.f;
 
-  if constexpr (STAGE == kVStats) {
+  // At 4 bits the values have no tensor-level scale, so nothing of a block's codes depends on
+  // other blocks: the block mean is formed here, in the quantizing pass, and the statistics
+  // launch is not needed.
+  constexpr bool kFusedMean = STAGE == kVQuant4 || STAGE == kVQuant4M;
+  if constexpr (STAGE == kVStats || kFusedMean) {
     __syncthreads();                         // the previous item's reads of `red` are done
     if (smooth) {
       float s0 = 0.f, s1 = 0.f;
@@ -476,6 +480,8 @@ __device__ __forceinline__ void v_item(const PrepArgs& a, const unsigned char* s
       mu1 = s1 / (float)n_valid;
       __syncthreads();
     }
+  }
+  if constexpr (STAGE == kVStats) {
     if (tg == 0) { a.v_mu[mu_at] = mu0; a.v_mu[mu_at + 1] = mu1; }
     float m0 = 0.f, m1 = 0.f;
 #pragma unroll
@@ -497,8 +503,10 @@ __device__ __forceinline__ void v_item(const PrepArgs& a, const unsigned char* s
     return;
   }
 
-  mu0 = mu_in.x;
-  mu1 = mu_in.y;
+  if constexpr (!kFusedMean) {
+    mu0 = mu_in.x;
+    mu1 = mu_in.y;
+  }
   float r0[TPG], r1[TPG];
 #pragma unroll
   for (int i = 0; i < TPG; ++i) {
@@ -712,7 +720,7 @@ __global__ void __launch_bounds__(kThreads, 2) prep_v_kernel(const PrepArgs a, i
   // per-item scalars of the quantizing stage, fetched one item ahead
   const int cp = tid % (D / 2);
   auto fetch_mu = [&](int item, const Item& w) -> float2 {
-    if (STAGE == kVStats || item >= n_items) return make_float2(0.f, 0.f);
+    if (STAGE == kVStats || STAGE == kVQuant4 || STAGE == kVQuant4M || item >= n_items) return make_float2(0.f, 0.f);
     return *reinterpret_cast<const float2*>(a.v_mu + ((size_t)w.bh * a.nb + w.blk) * D + 2 * cp);
   };
   int src[NL];
@@ -895,10 +903,10 @@ cudaError_t run(const Problem& pr, PrepArgs a, const WorkLayout& wl, uint8_t* wo
       prep_kcolsum_kernel<D><<<persistent_grid(per), kThreads, colsum_smem, s>>>(a, per, nh);
       count_launches(1);
     }
-    prep_v_kernel<D, kVStats><<<persistent_grid(per), kThreads, v_smem, s>>>(a, per, nh);
+    if (BITS == 8) prep_v_kernel<D, kVStats><<<persistent_grid(per), kThreads, v_smem, s>>>(a, per, nh);
     if (BITS == 4) { prep_qk_kernel<D, kStageAmax, kTpr><<<persistent_grid(per), kRowThreads * kTpr, row_smem, s>>>(a, per, nh, 0); count_launches(1); }
     prep_finalize_kernel<D, BITS><<<nh, D, 0, s>>>(a, 0);
-    count_launches(2);
+    count_launches(BITS == 8 ? 2 : 1);
     if (BITS == 4) {
       prep_qk_kernel<D, kStageAmax, kTpr><<<persistent_grid(per), kRowThreads * kTpr, row_smem, s>>>(a, per, nh, 1);
       prep_finalize_kernel<D, BITS><<<nh, 32, 0, s>>>(a, 1);
