@@ -202,11 +202,26 @@ vc_status vc_attn_host(const vc_params* p, const void* q_host, const void* k_hos
   // group, which is safe because the groups' kernels run in order on `stream`.
   cudaStream_t s = (cudaStream_t)stream;
   // heads per group: about a tenth of the heads, in multiples that keep a group's slice of
-  // perm 16-byte aligned (N * 4 bytes per head)
+  // perm 16-byte aligned (N * 4 bytes per head).  The input copy is the longest of the three
+  // pipelined activities, so what the call costs beyond it is the first group's copy (nothing
+  // can run before it) and the last group's compute and output copy: the groups at both ends are
+  // small (1, 2, ... and ..., 2, 1 multiples), the ones in between large enough to run efficiently.
   const int mult = pr.N % 4 == 0 ? 1 : (pr.N % 2 == 0 ? 2 : 4);
   int hg = pr.BH >= 10 ? (pr.BH + 9) / 10 : 1;
   hg = (hg + mult - 1) / mult * mult;
-  const int groups = (pr.BH + hg - 1) / hg;
+  std::vector<int> sizes;
+  if (pr.BH >= 12 * mult && hg > 2 * mult) {
+    const int last = mult + pr.BH % mult;              // the last group absorbs a remainder
+    int middle = pr.BH - last - 2 * mult - 3 * mult;   // after the leading 1, 2 and before the trailing 2, 1
+    sizes.push_back(mult);
+    sizes.push_back(2 * mult);
+    for (; middle > 0; middle -= hg) sizes.push_back(middle < hg ? middle : hg);
+    sizes.push_back(2 * mult);
+    sizes.push_back(last);
+  } else {
+    for (int h = 0; h < pr.BH; h += hg) sizes.push_back(pr.BH - h < hg ? pr.BH - h : hg);
+  }
+  const int groups = (int)sizes.size();
   const size_t head_elems = (size_t)pr.N * pr.d;
   cudaStream_t s_in = nullptr, s_out = nullptr;
   std::vector<cudaEvent_t> ev(2 * groups + 2, nullptr);
@@ -221,8 +236,9 @@ vc_status vc_attn_host(const vc_params* p, const void* q_host, const void* k_hos
     vc_params sub = *p;
     sub.B = 1;
     sub.stride_b = sub.stride_h = sub.stride_n = 0;
-    for (int g = 0; ok && g < groups; ++g) {
-      const int h0 = g * hg, nh = pr.BH - h0 < hg ? pr.BH - h0 : hg;
+    int h0 = 0;
+    for (int g = 0; ok && g < groups; h0 += sizes[g], ++g) {
+      const int nh = sizes[g];
       const size_t off = (size_t)h0 * head_elems * 2, bytes = (size_t)nh * head_elems * 2;
       ok = cudaMemcpyAsync((char*)q_dev + off, (const char*)q_host + off, bytes, cudaMemcpyHostToDevice, s_in) == cudaSuccess &&
            cudaMemcpyAsync((char*)k_dev + off, (const char*)k_host + off, bytes, cudaMemcpyHostToDevice, s_in) == cudaSuccess &&

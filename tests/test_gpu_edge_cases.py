@@ -99,7 +99,9 @@ def test_strided_inputs_through_vc_attn():
     assert torch.equal(outs[0], outs[1])
 
 
-@pytest.mark.parametrize("shape", [(2, 6, 300, 64, (3, 10, 10)), (1, 3, 257, 128, (1, 1, 257))], ids=["12_heads_6_groups", "3_heads"])
+@pytest.mark.parametrize("shape", [(2, 6, 300, 64, (3, 10, 10)), (1, 3, 257, 128, (1, 1, 257)), (2, 16, 200, 64, (2, 10, 10)),
+                                   (1, 48, 257, 128, (1, 1, 257))],
+                         ids=["12_heads_6_groups", "3_heads", "32_heads_graduated_groups", "48_heads_odd_length"])
 @pytest.mark.parametrize("bits", [8, 4, "4-hybrid"])
 def test_host_entry_point_equals_the_device_path(shape, bits):
     """vc_attn_host (pinned host buffers in and out, pipelined over groups of heads) gives exactly
