@@ -280,7 +280,9 @@ def main():
     vc.vc_poll_status(work)
     ms_total = t_start.elapsed_time(t_end)
     prep_ms = statistics.mean(e[0].elapsed_time(e[1]) for e in ev)
-    attn_ms = statistics.mean(e[1].elapsed_time(e[2]) for e in ev)
+    attn_all = [e[1].elapsed_time(e[2]) for e in ev]
+    prep_all = [e[0].elapsed_time(e[1]) for e in ev]
+    attn_ms = statistics.mean(attn_all)
     group = None
     if args.perm == "group":
         calls = [e[3].elapsed_time(e[0]) for i, e in enumerate(ev) if i % group_every == 0]
@@ -376,9 +378,9 @@ def main():
                      "peak_source": f"{peaks['source']}: bf16 sustained {peaks['bf16_sustained']} TF/s x {ratio:g}" + (" (nominal FP8:bf16)" if args.bits == 8 else (" (half the FLOPs at FP4:bf16 = 4, half at FP8:bf16 = 2)" if hybrid else " (nominal FP4:bf16)")),
                      ("frac_of_nominal_fp8_4500" if args.bits == 8 else ("frac_of_nominal_fp4_fp8_mix_6000" if hybrid else "frac_of_nominal_fp4_9000")):
                          achieved / (4500.0 if args.bits == 8 else (6000.0 if hybrid else 9000.0)),
-                     "ms": attn_ms},
+                     "ms": attn_ms, "ms_median": statistics.median(attn_all), "ms_min": min(attn_all)},
         "group": group,
-        "prep": {"ms": prep_ms, "algorithmic_gb": prep_bytes / 1e9, "gbs": prep_gbs,
+        "prep": {"ms": prep_ms, "ms_median": statistics.median(prep_all), "ms_min": min(prep_all), "algorithmic_gb": prep_bytes / 1e9, "gbs": prep_gbs,
                  "frac_of_measured_hbm": prep_gbs / peaks["hbm_gbs"], "frac_of_8tbs": prep_gbs / 8000.0},
     }
     if not args.no_sdpa:
