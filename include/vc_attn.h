@@ -145,7 +145,10 @@ vc_status vc_prep(const vc_params *p, const void *q, const void *k, const void *
                   const int32_t *perm, void *quant, void *workspace, void *stream);
 
 /* Quantized attention forward (Eq. 1, Eq. 6, Eq. 7) from a bundle in vc_prep's layout.
- * o: [B][H][N][d] bf16.  workspace as above. */
+ * o: [B][H][N][d] bf16.  workspace as above.  `p` must describe the bundle: the same shape,
+ * bits, p_format (it selects the value format at 4 bits) and flags as the vc_prep call that
+ * wrote it; a mismatch is not detected and gives meaningless output (never an out-of-bounds
+ * access: every section is sized for its largest variant). */
 vc_status vc_attn_fwd(const vc_params *p, const void *quant, void *o, void *workspace,
                       void *stream);
 
