@@ -147,8 +147,7 @@ vc_status vc_prep(const vc_params *p, const void *q, const void *k, const void *
 /* Quantized attention forward (Eq. 1, Eq. 6, Eq. 7) from a bundle in vc_prep's layout.
  * o: [B][H][N][d] bf16.  workspace as above.  `p` must describe the bundle: the same shape,
  * bits, p_format (it selects the value format at 4 bits) and flags as the vc_prep call that
- * wrote it; a mismatch is not detected and gives meaningless output (never an out-of-bounds
- * access: every section is sized for its largest variant). */
+ * wrote it, and `quant` must hold vc_quant_bytes(p) bytes; a mismatch is not detected. */
 vc_status vc_attn_fwd(const vc_params *p, const void *quant, void *o, void *workspace,
                       void *stream);
 
