@@ -437,13 +437,15 @@ attn4_fwd_2q_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         if (__any_sync(0xffffffffu, alpha != 1.0f)) {        // a row maximum moved: A <- alpha A (l included)
           uint32_t r[16];
 #pragma unroll 1
-          for (int c = 0; c < (D + 16) / 16; ++c) {
+          for (int c = 0; c < D / 16; ++c) {
             tmem_ld16(o_base + 16 * c, r);
             tmem_wait_ld();
 #pragma unroll
             for (int i = 0; i < 16; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * alpha);
             tmem_st16(o_base + 16 * c, r);
           }
+          // of the 16 row-sum columns only column d is ever read, and its value is at hand
+          tmem_st1(o_base + L_COL, __float_as_uint(l_now * alpha));
           tmem_wait_st();
           tc_fence_before();
         }
