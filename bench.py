@@ -169,7 +169,17 @@ def cpu_baseline(w, bits, hybrid=False, budget_rows=4096, heads=2):
         tp += t1 - t0
         ta += t2 - t1
     flops = 4.0 * heads * len(rows) * w.N * w.d
-    return {"value": flops / (tp + ta) / 1e12, "unit": UNIT, "cores": os.cpu_count(), "kind": "oracle",
+    # what the synthetic inputs look like to the softmax (not timed): spread of the exact scores
+    # and the effective number of keys 1 / sum p^2 per row, on 64 rows of the last sampled head
+    rs = np.linspace(0, w.N - 1, 64).astype(np.int64)
+    cos, sin = OP.rope_tables(cfg)
+    qr, kr = OP.rope_apply(q, cos, sin).astype(np.float64), OP.rope_apply(k, cos, sin).astype(np.float64)
+    sc = (qr[rs] @ kr.T) / np.sqrt(w.d)
+    pr_ = np.exp(sc - sc.max(axis=1, keepdims=True))
+    pr_ /= pr_.sum(axis=1, keepdims=True)
+    stats = {"score_std": float(sc.std(axis=1).mean()), "effective_keys": float((1.0 / (pr_ ** 2).sum(axis=1)).mean()),
+             "rows": int(len(rs))}
+    return {"value": flops / (tp + ta) / 1e12, "unit": UNIT, "cores": os.cpu_count(), "kind": "oracle", "input_statistics": stats,
             "sample": f"{heads} of {w.B * w.H} heads: preprocessing in full ({tp:.1f} s) + {len(rows)} of {w.N} query rows x "
                       f"all keys per head ({ta:.1f} s); NumPy, threads as its BLAS picks"}
 
