@@ -184,6 +184,39 @@ def cpu_baseline(w, bits, hybrid=False, budget_rows=4096, heads=2):
                       f"all keys per head ({ta:.1f} s); NumPy, threads as its BLAS picks"}
 
 
+def parity_report(w, p, q, k, v, perm, o, quant, work, bits, hybrid, int8_qk, n_rows=256):
+    """The GPU output of one head on sampled query rows against the oracle's emulation of the same
+    arrangement (the parity target) and against exact fp64 attention (accuracy), same buffers,
+    same permutation.  Not timed."""
+    import numpy as np
+    import paper_2609_15810_b200 as vc
+    from oracle import attention as OA
+    from oracle import compare as CMP
+    from oracle import prep as OP
+    vc.vc_attn(p, q, k, v, perm, o, quant, work)          # the arrangement asked for, once more
+    vc.vc_poll_status(work)
+    h = w.H - 1
+    f = lambda t: t[0, h].float().cpu().numpy()
+    qh, kh, vh = f(q), f(k), f(v)
+    pm = None if perm is None else perm[0, h].cpu().numpy().astype(np.int64)
+    cfg, pf = _oracle_cfg(w, bits, hybrid)
+    if int8_qk:
+        cfg.qk_format = "int8"
+    nb = (w.N + 127) // 128
+    tiles = sorted({nb // 2, nb - 1})                      # a full tile and the ragged last one
+    rows = np.concatenate([np.arange(128 * t, min(128 * (t + 1), w.N)) for t in tiles])[:n_rows]
+    bundle = OP.prep_head(qh, kh, vh, pm, cfg)
+    emu = OA.emulate_head(bundle, cfg, rows=rows, p_format=pf).astype(np.float64)
+    exact = OA.reference_head(qh, kh, vh, cfg, rows=rows)
+    got = o[0, h].float().cpu().numpy()[rows].astype(np.float64)
+    vmax = float(np.abs(vh).max())
+    pick = lambda m: {"max_err_over_vmax": m["max_err_over_vmax"], "cos": m["cos"], "psnr_db": float(m["psnr_db"])}
+    return {"head": [0, h], "rows": int(len(rows)), "tolerance": "|delta| <= 2e-2 max|V| and cos >= 0.999 against the emulation",
+            "gpu_vs_emulation": pick(CMP.output_metrics(got, emu, vmax)),
+            "gpu_vs_exact_fp64": pick(CMP.output_metrics(got, exact, vmax)),
+            "emulation_vs_exact_fp64": pick(CMP.output_metrics(emu, exact, vmax))}
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -410,6 +443,8 @@ def main():
             out["bf16_sdpa"] = {"error": str(exc)[:200]}
     if not args.no_cpu_baseline:
         out["cpu_baseline"] = cpu_baseline(w, args.bits, hybrid)
+        if args.data == "workload":
+            out["parity"] = parity_report(w, p, q, k, v, perm, o, quant, work, args.bits, hybrid, args.int8_qk)
     print(json.dumps(out), flush=True)
     if world > 1:
         dist.destroy_process_group()
