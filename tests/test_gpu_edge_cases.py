@@ -16,7 +16,16 @@ import helpers as Hh
 pytestmark = pytest.mark.gpu
 
 
+def _params(B, H, N, d, grid, bits, **kw):
+    """bits = "4-hybrid" selects the hybrid 4-bit arrangement (ExpCast-FP8 P over 4-bit Q, K, V)."""
+    if bits == "4-hybrid":
+        return Params.make(B, H, N, d, grid, bits=4, p_format=vc.VC_P_EXPCAST_E4M3, **kw)
+    return Params.make(B, H, N, d, grid, bits=bits, **kw)
+
+
 def _run(p, q, k, v, perm, softmax_scale=None, beta=None, p_format=None):
+    if p_format is None and Hh.is_hybrid(p):
+        p_format = OA.P_EXPCAST
     quant, work = alloc_buffers(p)
     o = torch.empty(p.B, p.H, p.N, p.d, dtype=torch.bfloat16, device="cuda")
     vc.vc_attn(p, q, k, v, perm, o, quant, work)
@@ -44,12 +53,12 @@ def _run(p, q, k, v, perm, softmax_scale=None, beta=None, p_format=None):
     return worst
 
 
-@pytest.mark.parametrize("bits", [8, 4])
+@pytest.mark.parametrize("bits", [8, 4, "4-hybrid"])
 @pytest.mark.parametrize("N,grid", [(1, (1, 1, 1)), (2, (1, 1, 2)), (17, (1, 1, 17)), (127, (1, 1, 127))])
 def test_shortest_sequences(N, grid, bits):
     w = vc_inputs.Workload("t", 1, 2, N, 128, grid, (8,), 41, "gauss")
     q, k, v = [t.cuda() for t in vc_inputs.make_qkv(w)]
-    _run(Params.make(1, 2, N, 128, grid, bits=bits), q, k, v, None)
+    _run(_params(1, 2, N, 128, grid, bits), q, k, v, None)
 
 
 @pytest.mark.parametrize("flags", [0, vc.VC_FLAG_ROPE, vc.VC_FLAG_HADAMARD | vc.VC_FLAG_K_SMOOTH, vc.VC_FLAG_V_SMOOTH,
@@ -70,14 +79,14 @@ def test_softmax_scale_beta_and_exp_then_cast():
          softmax_scale=0.2, p_format=OA.P_EXP_E4M3)
 
 
-@pytest.mark.parametrize("bits", [8, 4])
+@pytest.mark.parametrize("bits", [8, 4, "4-hybrid"])
 def test_degenerate_scales(bits):
     w = vc_inputs.Workload("t", 1, 1, 384, 128, (6, 8, 8), (8,), 44, "gauss")
     q, k, v = [t.cuda() for t in vc_inputs.make_qkv(w)]
-    p = Params.make(1, 1, 384, 128, (6, 8, 8), bits=bits)
+    p = _params(1, 1, 384, 128, (6, 8, 8), bits)
     _run(p, q, k, torch.zeros_like(v), None)                                   # all-zero V: every scale degenerate
     _run(p, q, k, torch.full_like(v, 1.5), None)                               # constant V: zero residual, mean only
-    pk = Params.make(1, 1, 384, 128, (6, 8, 8), bits=bits, flags=vc.VC_FLAG_ALL & ~vc.VC_FLAG_ROPE)
+    pk = _params(1, 1, 384, 128, (6, 8, 8), bits, flags=vc.VC_FLAG_ALL & ~vc.VC_FLAG_ROPE)
     _run(pk, q, torch.full_like(k, 0.75), v, None)                             # constant K: centered keys vanish
     _run(p, torch.zeros_like(q), k, v, None)                                   # zero Q: uniform attention
 

@@ -23,8 +23,10 @@ CASES = [("c2", 8, "kmeans"), ("c3", 8, "kmeans"), ("c3", 4, "random"), ("c4", 4
          ("c4_2heads", 8, "random"),  # the longest sequence (929 key tiles, an odd count) at 8 bits
          ("c3", 4, "group-hybrid"),   # the hybrid 4-bit arrangement (ExpCast-FP8 P over 4-bit Q, K, V)
          ("c5_d64_n4096", 4, "random-hybrid"),
-         ("c4_2heads", 4, "random-hybrid")]   # 929 key tiles through the FP8 x FP4 value product
+         ("c4_2heads", 4, "random-hybrid"),   # 929 key tiles through the FP8 x FP4 value product
+         ("n262144", 8, "random")]            # 2048 key tiles: the longest sequence tested
 
+vc_inputs.WORKLOADS.setdefault("n262144", vc_inputs.Workload("n262144", 1, 1, 262144, 128, (64, 64, 64), (8,), 1077, "field", False))
 vc_inputs.WORKLOADS.setdefault("c4_2heads", vc_inputs.Workload("c4_2heads", 1, 2, 118800, 128, (33, 45, 80), (8,), 1044, "field", True))
 
 
