@@ -206,3 +206,27 @@ def test_hybrid_4bit_stage_switches_and_parameters(flags):
     shifted = torch.empty(quant.numel() + 16, dtype=torch.uint8, device="cuda")[16:]
     with pytest.raises(vc.VcError):
         vc.vc_attn_fwd(p, shifted, o, work)
+
+
+@pytest.mark.parametrize("bits", [8, 4, "4-hybrid"])
+def test_repeated_calls_are_bitwise_identical(bits):
+    """No floating-point atomics and no order that depends on timing: the bundle and the output of
+    two calls on the same inputs are the same bytes (the grouping call included)."""
+    B, H, N, d, grid = 1, 3, 1500, 128, (5, 15, 20)
+    w = vc_inputs.Workload("t", B, H, N, d, grid, (8,), 63, "field")
+    q, k, v = [t.cuda() for t in vc_inputs.make_qkv(w)]
+    p = _params(B, H, N, d, grid, bits)
+    outs = []
+    for _ in range(2):
+        gwork = torch.empty(vc.vc_group_workspace_bytes(p), dtype=torch.uint8, device="cuda")
+        cent = torch.zeros(B, H, 16, d, dtype=torch.float32, device="cuda")
+        perm = torch.empty(B, H, N, dtype=torch.int32, device="cuda")
+        vc.vc_group(p, v, 16, 3, False, cent, perm, gwork)
+        quant, work = alloc_buffers(p)
+        quant.zero_()
+        o = torch.empty(B, H, N, d, dtype=torch.bfloat16, device="cuda")
+        vc.vc_attn(p, q, k, v, perm, o, quant, work)
+        vc.vc_poll_status(work)
+        outs.append((perm.clone(), cent.clone(), quant.clone(), o.clone()))
+    for a, b in zip(*outs):
+        assert torch.equal(a, b)
