@@ -88,7 +88,7 @@ enum {
 };
 
 typedef struct {
-  int32_t B, H, N, d;               /* d in {64, 128}; N >= 1                           */
+  int32_t B, H, N, d;               /* d in {64, 128}; 1 <= N <= 2^22; B * H <= 65535   */
   int32_t grid_t, grid_h, grid_w;   /* grid_t * grid_h * grid_w == N                    */
   int32_t bits;                     /* 8 or 4                                           */
   int32_t p_format;                 /* VC_P_*                                           */

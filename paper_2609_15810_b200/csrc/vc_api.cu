@@ -17,7 +17,8 @@ vc_status resolve(const vc_params* p, Problem* out) {
   Problem pr{};
   pr.B = p->B; pr.H = p->H; pr.N = p->N; pr.d = p->d;
   if (pr.B < 1 || pr.H < 1 || pr.N < 1) return VC_ERR_INVALID_ARG;
-  if ((int64_t)pr.B * pr.H > (1 << 20) || pr.N > (1 << 22)) return VC_ERR_INVALID_ARG;
+  // B * H is the second grid dimension of several launches (limit 65535)
+  if ((int64_t)pr.B * pr.H > 65535 || pr.N > (1 << 22)) return VC_ERR_INVALID_ARG;
   if (pr.d != 64 && pr.d != 128) return VC_ERR_INVALID_ARG;
   pr.BH = pr.B * pr.H;
   pr.grid_t = p->grid_t; pr.grid_h = p->grid_h; pr.grid_w = p->grid_w;

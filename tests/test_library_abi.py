@@ -37,7 +37,7 @@ def test_sizes_and_argument_validation_without_a_gpu():
     assert vc.vc_quant_bytes(Params.make(1, 2, 1024, 128, (4, 16, 16), bits=4, p_format=vc.VC_P_EXPCAST_E4M3, kernel_variant=1)) == 0
     assert vc.vc_quant_bytes(Params.make(1, 2, 1024, 128, (4, 16, 16), bits=4, p_format=vc.VC_P_EXP_E4M3)) == 0
     assert vc.vc_quant_bytes(Params.make(1, 2, 1024, 128, (4, 16, 16), bits=8, p_format=vc.VC_P_EXP_POLY_E4M3)) > 0
-    for bad in (dict(d=100), dict(N=-1), dict(bits=3), dict(grid_t=20), dict(p_format=9)):
+    for bad in (dict(d=100), dict(N=-1), dict(bits=3), dict(grid_t=20), dict(p_format=9), dict(B=40000)):
         pb = Params.make(1, 2, 1024, 128, (4, 16, 16))
         for k, v in bad.items():
             setattr(pb, k, v)
