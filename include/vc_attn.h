@@ -42,7 +42,8 @@ extern "C" {
 
 typedef enum {
   VC_OK = 0,
-  VC_ERR_INVALID_ARG = 1,   /* null pointer, bad size, misaligned pointer            */
+  VC_ERR_INVALID_ARG = 1,   /* null pointer, bad size, misaligned pointer; from
+                               vc_poll_status: `perm` was not a permutation          */
   VC_ERR_UNSUPPORTED = 2,   /* a combination this build does not implement           */
   VC_ERR_WORKSPACE = 3,     /* reserved                                              */
   VC_ERR_CUDA = 4,          /* a CUDA runtime/driver call failed                     */
@@ -84,7 +85,13 @@ enum {
    * per 128 rows) and Q^ K^T as an integer product -- the arrangement the paper runs on B200
    * (Fig. 3); default is FP8 E4M3 for both products (the paper's B300 arrangement, Sec. 4.5).
    * bits = 8 and the pipelined kernel only. */
-  VC_FLAG_INT8_QK = 16
+  VC_FLAG_INT8_QK = 16,
+  /* check switch, not part of VC_FLAG_ALL: vc_prep also runs a validator over `perm` (Eq. 3
+   * needs a permutation of [0, N) per head).  An entry outside [0, N) or one that occurs twice
+   * is recorded in the status word and vc_poll_status returns VC_ERR_INVALID_ARG.  With or
+   * without this flag the gather itself clamps every entry into [0, N), so a bad `perm` gives a
+   * wrong bundle, never an out-of-bounds read. */
+  VC_FLAG_CHECK_PERM = 32
 };
 
 typedef struct {
@@ -104,6 +111,12 @@ typedef struct {
   int32_t kernel_variant;           /* attention kernel: 0 = pipelined, two query tiles per
                                        CTA (default); 1 = simple serial kernel, kept for
                                        A/B measurement and cross-checks                  */
+  int32_t block_q, block_k, block_v; /* rows per Q and per K scale block, tokens per value
+                                       block B_v of Eq. 4 (Sec. 3.2 "Block demeaning").  0 =>
+                                       128.  The kernels are laid out for 128 (one block = one
+                                       MMA tile, so a scale folds into the softmax constant and
+                                       a block mean into one rank-one update per tile); any
+                                       other value returns VC_ERR_UNSUPPORTED              */
 } vc_params;
 
 /* Device pointers into the quantized bundle written by vc_prep (N_pad = 128*ceil(N/128),
@@ -139,8 +152,13 @@ size_t vc_workspace_bytes(const vc_params *p);
 
 /* Preprocessing pass (Sec. 3.4, App. B).  perm: int32 [B][H][N], row t of the permuted
  * K/V is row perm[t] of the input (Eq. 3), or NULL for the identity; it must be a
- * permutation of [0, N) per (b, h) (not checked).  Writes `quant`; uses `workspace`
- * (contents on entry irrelevant; the first 4 bytes become the status word). */
+ * permutation of [0, N) per (b, h).  Entries are clamped into [0, N) before they are used
+ * as row indices; VC_FLAG_CHECK_PERM adds a validator that reports a bad entry through the
+ * status word.  Writes `quant`; uses `workspace` (contents on entry irrelevant; the first 4
+ * bytes become the status word).  At 8 bits the pass is ONE persistent launch: statistics
+ * items (K column sums, V block means and residual maxima) of a head run ahead of its
+ * quantizing items, which wait on a per-head counter in the workspace with a bounded spin
+ * (VC_ERR_TIMEOUT through the status word if it gives up); heads_per_pass is ignored there. */
 vc_status vc_prep(const vc_params *p, const void *q, const void *k, const void *v,
                   const int32_t *perm, void *quant, void *workspace, void *stream);
 
@@ -180,10 +198,14 @@ vc_status vc_attn_host(const vc_params *p, const void *q_host, const void *k_hos
  *   warm_start 0: centroids start at rows 0, N/k, 2 N/k, ... of V; 1: at the values in `centroids`
  *   centroids  [B][H][k][d] fp32, in (warm start) and out (after the last update)
  *   perm       out, int32 [B][H][N]
- *   workspace  vc_group_workspace_bytes(p) bytes; on return its first B*H*N int32 are the labels
+ *   workspace  vc_group_workspace_bytes(p) bytes; its first 4 bytes are the status word
+ *              (vc_poll_status(workspace, stream) reports a device-side wait that gave up as
+ *              VC_ERR_TIMEOUT; `perm` is then not valid), and on return the B*H*N int32 at byte
+ *              offset VC_GROUP_LABELS_OFFSET are the labels
  * The paper leaves k, the initialisation and the iteration count open; distances are squared
  * Euclidean on the fp32 rows, ties go to the lower cluster index, an empty cluster keeps its
  * centroid.  Deterministic (no floating-point atomics).  Returns VC_ERR_UNSUPPORTED for k > 64. */
+#define VC_GROUP_LABELS_OFFSET 1024
 size_t vc_group_workspace_bytes(const vc_params *p);
 vc_status vc_group(const vc_params *p, const void *v, int32_t k, int32_t iters, int32_t warm_start,
                    float *centroids, int32_t *perm, void *workspace, void *stream);
@@ -233,8 +255,18 @@ vc_status vc_prep_noalloc(const vc_params *p, const void *q, const void *k, cons
 vc_status vc_quant_view(const vc_params *p, const void *quant, vc_quant_ptrs *out);
 
 /* Synchronizes `stream` and returns VC_ERR_TIMEOUT if a kernel recorded a timed-out wait,
- * VC_ERR_CUDA on a CUDA error, VC_OK otherwise.  Clears the status word. */
+ * VC_ERR_INVALID_ARG if the validator of VC_FLAG_CHECK_PERM found `perm` not to be a
+ * permutation, VC_ERR_CUDA on a CUDA error, VC_OK otherwise.  Clears the status word.
+ * `workspace` is the workspace of vc_prep / vc_attn_fwd / vc_attn or that of vc_group. */
 vc_status vc_poll_status(void *workspace, void *stream);
+
+/* Test hook: the number of polls after which a device-side wait gives up (every mbarrier wait
+ * of the attention kernels, the per-head waits of the preprocessing pass, the waits of the
+ * grouping kernel).  0 restores the default (about one second).  A tiny value makes waits run
+ * out on a correct run, which is how the time-out path is exercised without hanging anything:
+ * the kernels then record VC_ERR_TIMEOUT, drain their own copies in flight, free their tensor
+ * memory and return; outputs of such a call are invalid.  Process-wide; not for production. */
+void vc_test_set_wait_limit(uint32_t polls);
 
 /* Number of kernels this library has launched in this process (diagnostics). */
 uint64_t vc_launch_count(void);

@@ -16,6 +16,9 @@ VC_P_DEFAULT, VC_P_EXPCAST_E4M3, VC_P_EXP_E4M3, VC_P_NVFP4 = 0, 1, 2, 3
 VC_P_EXP_POLY_E4M3, VC_P_EXP_MIX_E4M3 = 4, 5
 VC_FLAG_ROPE, VC_FLAG_HADAMARD, VC_FLAG_K_SMOOTH, VC_FLAG_V_SMOOTH, VC_FLAG_ALL = 1, 2, 4, 8, 15
 VC_FLAG_INT8_QK = 16
+VC_FLAG_CHECK_PERM = 32
+VC_GROUP_LABELS_OFFSET = 1024
+VC_OK, VC_ERR_INVALID_ARG, VC_ERR_UNSUPPORTED, VC_ERR_WORKSPACE, VC_ERR_CUDA, VC_ERR_TIMEOUT, VC_ERR_SCRATCH_LIMIT = range(7)
 
 
 class VcError(RuntimeError):
@@ -33,7 +36,8 @@ class Params(ctypes.Structure):
                 ("rope_dim_t", ctypes.c_int32), ("rope_dim_h", ctypes.c_int32), ("rope_dim_w", ctypes.c_int32),
                 ("rope_theta", ctypes.c_float),
                 ("stride_b", ctypes.c_int64), ("stride_h", ctypes.c_int64), ("stride_n", ctypes.c_int64),
-                ("heads_per_pass", ctypes.c_int32), ("kernel_variant", ctypes.c_int32)]
+                ("heads_per_pass", ctypes.c_int32), ("kernel_variant", ctypes.c_int32),
+                ("block_q", ctypes.c_int32), ("block_k", ctypes.c_int32), ("block_v", ctypes.c_int32)]
 
     @classmethod
     def make(cls, B, H, N, d, grid, bits=8, p_format=VC_P_DEFAULT, flags=VC_FLAG_ALL, **kw):
@@ -89,6 +93,8 @@ def load_library():
     lib.vc_quant_view.argtypes = [P, vp, ctypes.POINTER(QuantView)]
     lib.vc_poll_status.restype = ctypes.c_int
     lib.vc_poll_status.argtypes = [vp, vp]
+    lib.vc_test_set_wait_limit.restype = None
+    lib.vc_test_set_wait_limit.argtypes = [ctypes.c_uint32]
     lib.vc_launch_count.restype = ctypes.c_uint64
     lib.vc_launch_count.argtypes = []
     lib.vc_status_string.restype = ctypes.c_char_p
@@ -181,6 +187,11 @@ def vc_quant_view(p, quant):
 
 def vc_poll_status(workspace):
     _check(load_library().vc_poll_status(_ptr(workspace), _stream()), "vc_poll_status")
+
+
+def vc_test_set_wait_limit(polls):
+    """Test hook: polls after which a device-side wait gives up (0 = the default)."""
+    load_library().vc_test_set_wait_limit(int(polls))
 
 
 def vc_launch_count():

@@ -10,6 +10,9 @@ namespace vc {
 static std::atomic<uint64_t> g_launches{0};
 void count_launches(int n) { g_launches.fetch_add((uint64_t)n, std::memory_order_relaxed); }
 
+static std::atomic<uint32_t> g_wait_limit{0};
+uint32_t wait_limit_override() { return g_wait_limit.load(std::memory_order_relaxed); }
+
 static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 vc_status resolve(const vc_params* p, Problem* out) {
@@ -34,7 +37,11 @@ vc_status resolve(const vc_params* p, Problem* out) {
   if (pr.p_format > VC_P_NVFP4 && (p->flags & VC_FLAG_INT8_QK)) return VC_ERR_UNSUPPORTED;
   if (pr.bits == 4 && pr.p_format != VC_P_NVFP4 && pr.p_format != VC_P_EXPCAST_E4M3) return VC_ERR_UNSUPPORTED;
   pr.flags = p->flags;
-  if (pr.flags & ~(VC_FLAG_ALL | VC_FLAG_INT8_QK)) return VC_ERR_INVALID_ARG;
+  if (pr.flags & ~(VC_FLAG_ALL | VC_FLAG_INT8_QK | VC_FLAG_CHECK_PERM)) return VC_ERR_INVALID_ARG;
+  // scale blocks and the value block of Eq. 4: the kernels implement 128 only
+  if (p->block_q < 0 || p->block_k < 0 || p->block_v < 0) return VC_ERR_INVALID_ARG;
+  if ((p->block_q && p->block_q != kBlock) || (p->block_k && p->block_k != kBlock) || (p->block_v && p->block_v != kBlock))
+    return VC_ERR_UNSUPPORTED;
   pr.softmax_scale = p->softmax_scale != 0.f ? p->softmax_scale : 1.0f / sqrtf((float)pr.d);
   if (!(pr.softmax_scale > 0.f)) return VC_ERR_INVALID_ARG;
   pr.beta = p->beta != 0.f ? p->beta : -0.35f;
@@ -114,6 +121,10 @@ WorkLayout work_layout(const Problem& pr) {
   W.v_mu = place(BH * nb * d * 4);
   W.amax_bytes = BH * d * 4 + 2 * BH * 4;
   W.amax = place(W.amax_bytes);
+  W.sync_bytes = (2 * BH + 4) * 4;
+  W.sync = place(W.sync_bytes);
+  W.perm_bits_bytes = (pr.flags & VC_FLAG_CHECK_PERM) ? BH * (((size_t)pr.N + 31) / 32) * 4 : 0;
+  W.perm_bits = place(W.perm_bits_bytes);
   W.mu_mma = place(BH * nb * d * 32);
   W.sf_q = place(pr.bits == 4 ? BH * nb * (d / 64) * 512 : 0);
   W.sf_kv = place(pr.bits == 4 ? BH * nb * (d / 64 + 2) * 512 : 0);
@@ -158,8 +169,7 @@ vc_status vc_prep(const vc_params* p, const void* q, const void* k, const void* 
   return e == cudaSuccess ? VC_OK : VC_ERR_CUDA;
 }
 
-vc_status vc_attn_fwd(const vc_params* p, const void* quant, void* o, void* workspace,
-                      void* stream) {
+static vc_status attn_fwd_impl(const vc_params* p, const void* quant, void* o, void* workspace, void* stream, bool clear_status) {
   Problem pr;
   vc_status st = resolve(p, &pr);
   if (st != VC_OK) return st;
@@ -170,16 +180,20 @@ vc_status vc_attn_fwd(const vc_params* p, const void* quant, void* o, void* work
   QuantLayout ql = quant_layout(pr);
   WorkLayout wl = work_layout(pr);
   cudaError_t e = launch_attn_fwd(pr, ql, wl, (const uint8_t*)quant, o, (uint8_t*)workspace,
-                                  (cudaStream_t)stream);
+                                  (cudaStream_t)stream, clear_status);
   if (e == cudaErrorNotSupported) return VC_ERR_UNSUPPORTED;
   return e == cudaSuccess ? VC_OK : VC_ERR_CUDA;
+}
+
+vc_status vc_attn_fwd(const vc_params* p, const void* quant, void* o, void* workspace, void* stream) {
+  return attn_fwd_impl(p, quant, o, workspace, stream, true);
 }
 
 vc_status vc_attn(const vc_params* p, const void* q, const void* k, const void* v,
                   const int32_t* perm, void* o, void* quant, void* workspace, void* stream) {
   vc_status st = vc_prep(p, q, k, v, perm, quant, workspace, stream);
   if (st != VC_OK) return st;
-  return vc_attn_fwd(p, quant, o, workspace, stream);
+  return attn_fwd_impl(p, quant, o, workspace, stream, false);   // keeps what the pass recorded in the status word
 }
 
 vc_status vc_attn_host(const vc_params* p, const void* q_host, const void* k_host,
@@ -304,7 +318,7 @@ vc_status vc_poll_status(void* workspace, void* stream) {
   if (word != 0) {
     cudaMemsetAsync(workspace, 0, 4, s);
     cudaStreamSynchronize(s);
-    return VC_ERR_TIMEOUT;
+    return (word & kStatusTimeout) ? VC_ERR_TIMEOUT : VC_ERR_INVALID_ARG;
   }
   return VC_OK;
 }
@@ -315,6 +329,8 @@ int32_t vc_group_schedule(int32_t step, int32_t n_steps, int32_t reuse) {
   if (step >= window) return VC_GROUP_FROZEN;
   return step % reuse == 0 ? VC_GROUP_RECOMPUTE : VC_GROUP_REUSE;
 }
+
+void vc_test_set_wait_limit(uint32_t polls) { g_wait_limit.store(polls, std::memory_order_relaxed); }
 
 uint64_t vc_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 

@@ -285,7 +285,10 @@ attn_fwd_2q_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
       mbar_init(&sh->fin_full[i], 128); mbar_init(&sh->o_final[i], 1);
       for (int b = 0; b < 2; ++b) { mbar_init(&sh->a_full[i][b], 128); mbar_init(&sh->pc_full[i][b], 256); }
     }
+    mbar_init(&sh->drain[0], 1); mbar_init(&sh->drain[1], 1);
     sh->abort = 0;
+    sh->wait_limit = a.wait_limit;
+    sh->wait_hint_ns = a.wait_hint_ns;
     mbar_fence_init();
     tma_prefetch_desc(&tm_q); tma_prefetch_desc(&tm_k); tma_prefetch_desc(&tm_v); tma_prefetch_desc(&tm_mu);
   }
@@ -311,7 +314,8 @@ attn_fwd_2q_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         tma_load_3d(sQ, &tm_q, &sh->q_full, 0, (2 * qpair) * 128, bh);
         tma_load_3d(sQ + kQBytes, &tm_q, &sh->q_full, 0, (2 * qpair + 1) * 128, bh);   // past the end: zero fill
       }
-      for (int j = 0; j < nb; ++j) {
+      int j = 0;
+      for (; j < nb; ++j) {
         const int st = j % kStages2, it = j / kStages2;
         unsigned char* base = sStage + st * kStageBytes;
         if (!warp_wait2(&sh->kv_empty[st], (it & 1) ^ 1, sh, a.status, 11)) break;
@@ -323,6 +327,7 @@ attn_fwd_2q_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         }
         __syncwarp();
       }
+      drain_loads(sh, j);                                 // (returns at once on a normal run)
     } else if (warp == 1) {
       // ------------------------------------------------------------------ score issuer
       // Issues S_t = Q^_t K^_jT for both query tiles into the ONE score buffer, in the fixed order
@@ -356,6 +361,7 @@ attn_fwd_2q_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
           __syncwarp();
         }
       }
+      drain_mmas(sh, 0);
     } else if (warp == 3) {
       // ------------------------------------------------------------------ accumulator issuer
       // A_t += P^_t(j) [R^_j | 1] once the codes are written, A_t is rescaled by alpha_j and the
@@ -396,6 +402,7 @@ attn_fwd_2q_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         }
         __syncwarp();
       }
+      drain_mmas(sh, 1);
     }
   } else if (warp < 12) {
     // -------------------------------------------------------------------- softmax warpgroups
@@ -823,6 +830,8 @@ cudaError_t run8(const Problem& pr, const QuantLayout& ql, const WorkLayout& wl,
   a.N = pr.N; a.n_pad = pr.n_pad; a.nb = pr.nb; a.p_format = pr.p_format;
   a.sl = pr.softmax_scale * 1.4426950408889634f;
   a.code_off = 120.0f + pr.beta;
+  a.wait_limit = attn_wait_limit();
+  a.wait_hint_ns = attn_wait_hint_ns();
   cudaError_t e;
   if (pr.kernel_variant == 1) {     // serial reference kernel
     const size_t smem = 1024 + 2 * 128 * D + D * 128 + D * 4 + 64;
@@ -900,9 +909,11 @@ cudaError_t run4(const Problem& pr, const QuantLayout& ql, const WorkLayout& wl,
 }  // namespace
 
 cudaError_t launch_attn_fwd(const Problem& pr, const QuantLayout& ql, const WorkLayout& wl,
-                            const uint8_t* quant, void* o, uint8_t* work, cudaStream_t stream) {
-  cudaError_t e = cudaMemsetAsync(work + wl.status, 0, 4, stream);
-  if (e != cudaSuccess) return e;
+                            const uint8_t* quant, void* o, uint8_t* work, cudaStream_t stream, bool clear_status) {
+  if (clear_status) {
+    cudaError_t e = cudaMemsetAsync(work + wl.status, 0, 4, stream);
+    if (e != cudaSuccess) return e;
+  }
   if (pr.bits == 4 && pr.kernel_variant == 0) return launch_attn_fwd4(pr, ql, wl, quant, o, work, stream);
   if (pr.bits == 4) return pr.d == 128 ? run4<128>(pr, ql, wl, quant, o, work, stream) : run4<64>(pr, ql, wl, quant, o, work, stream);
   return pr.d == 128 ? run8<128>(pr, ql, wl, quant, o, work, stream) : run8<64>(pr, ql, wl, quant, o, work, stream);

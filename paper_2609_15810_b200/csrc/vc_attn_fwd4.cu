@@ -87,6 +87,8 @@ struct Attn4Args {
   int N, n_pad, nb;
   float sl;                        // softmax_scale * log2(e)
   float code_off;                  // 120 + beta  (Eq. 7; hybrid arrangement only)
+  uint32_t wait_limit;             // polls after which a wait gives up
+  uint32_t wait_hint_ns;
 };
 
 // Value of a non-negative E4M3 byte.
@@ -146,7 +148,10 @@ attn4_fwd_2q_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       mbar_init(&sh->fin_full[i], 128); mbar_init(&sh->o_final[i], 1);
       for (int b = 0; b < 2; ++b) { mbar_init(&sh->a_full[i][b], 128); mbar_init(&sh->pc_full[i][b], 256); }
     }
+    mbar_init(&sh->drain[0], 1); mbar_init(&sh->drain[1], 1);
     sh->abort = 0;
+    sh->wait_limit = a.wait_limit;
+    sh->wait_hint_ns = a.wait_hint_ns;
     mbar_fence_init();
     tma_prefetch_desc(&tm_q); tma_prefetch_desc(&tm_k); tma_prefetch_desc(&tm_v); tma_prefetch_desc(&tm_mu);
   }
@@ -181,7 +186,8 @@ attn4_fwd_2q_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
           bulk_load(sSfq + t * 1024, a.sf_q + ((size_t)bh * nb + min(qb, nb - 1)) * kSfqBytes, kSfqBytes, &sh->q_full);
         }
       }
-      for (int j = 0; j < nb; ++j) {
+      int j = 0;
+      for (; j < nb; ++j) {
         const int st = j % kStages2, it = j / kStages2;
         unsigned char* base = sStage + st * kStageBytes;
         if (!warp_wait2(&sh->kv_empty[st], (it & 1) ^ 1, sh, a.status, 11)) break;
@@ -195,6 +201,7 @@ attn4_fwd_2q_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         }
         __syncwarp();
       }
+      drain_loads(sh, j);                                 // (returns at once on a normal run)
     } else if (warp == 1) {
       // ------------------------------------------------------------------ score issuer
       const uint32_t idesc_qk = idesc_nvfp4(128, 128);
@@ -233,6 +240,7 @@ attn4_fwd_2q_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
           __syncwarp();
         }
       }
+      drain_mmas(sh, 0);
     } else if (warp == 3) {
       // ------------------------------------------------------------------ accumulator issuer
       const uint32_t idesc_pv = idesc_nvfp4(128, D + 16), idesc_mu = idesc_tf32(128, D);
@@ -297,6 +305,7 @@ attn4_fwd_2q_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         }
         __syncwarp();
       }
+      drain_mmas(sh, 1);
     }
   } else if (warp < 12) {
     // -------------------------------------------------------------------- softmax warpgroups
@@ -517,6 +526,8 @@ cudaError_t run4(const Problem& pr, const QuantLayout& ql, const WorkLayout& wl,
   a.N = pr.N; a.n_pad = pr.n_pad; a.nb = pr.nb;
   a.sl = pr.softmax_scale * 1.4426950408889634f;
   a.code_off = 120.0f + pr.beta;
+  a.wait_limit = attn_wait_limit();
+  a.wait_hint_ns = attn_wait_hint_ns();
   constexpr size_t stage = 128 * (D / 2) + (D + 16) * kVRow + ((D * 32 + 1023) / 1024) * 1024 + (((KB + NVC) * 512 + 1023) / 1024) * 1024;
   constexpr size_t smem = 1024 + 2 * 128 * (D / 2) + 2 * 128 * kVRow + 2 * 128 * 32 + 2 * 1024 + 2 * 1024 + 1024 + kStages2 * stage + sizeof(FaSmem);
   static_assert(smem <= 227 * 1024, "shared memory of the 4-bit kernel exceeds the SM");

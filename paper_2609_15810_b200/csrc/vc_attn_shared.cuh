@@ -6,6 +6,7 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include "vc_internal.h"
 #include "vc_sm100.cuh"
 
 namespace vc {
@@ -13,7 +14,7 @@ namespace attn {
 
 using namespace sm100;
 
-constexpr uint32_t kErrTimeout = 0x100;
+constexpr uint32_t kErrTimeout = kStatusTimeout;
 
 // Arguments of the 8-bit attention kernels.
 struct AttnArgs {
@@ -24,10 +25,20 @@ struct AttnArgs {
   int N, n_pad, nb, p_format;
   float sl;        // softmax_scale * log2(e)
   float code_off;  // 120 + beta  (Eq. 7)
+  uint32_t wait_limit;   // polls after which a wait gives up
+  uint32_t wait_hint_ns;
 };
 
 constexpr int kStages2 = 4;
-constexpr uint32_t kWaitLimit2 = 1u << 18;   // x up to 4 us per try: about one second
+constexpr uint32_t kWaitLimit2 = 1u << 18;   // default polls of a wait, x up to 4 us per try: about one second
+constexpr uint32_t kDrainLimit = 1u << 22;   // polls of the exit waits for a CTA's own copies and MMAs
+
+inline uint32_t attn_wait_limit() {
+  const uint32_t lim = wait_limit_override();
+  return lim ? lim : kWaitLimit2;
+}
+// with the test override a poll does not sleep, so that a tiny limit really is a short wait
+inline uint32_t attn_wait_hint_ns() { return wait_limit_override() ? 32u : 4000u; }
 
 struct FaSmem {
   uint64_t q_full, kv_full[kStages2], kv_empty[kStages2];
@@ -35,15 +46,19 @@ struct FaSmem {
   // alpha and codes+correction hand-offs can run one key tile ahead of their consumer, so they
   // alternate between two barriers (a parity wait aliases after two phases)
   uint64_t a_full[2][2], pc_full[2][2];
+  uint64_t drain[2];      // exit: "every MMA this issuer warp issued has completed"
   float alpha[2][128];
   uint32_t tmem_base;
+  uint32_t wait_limit;    // polls of a wait ...
+  uint32_t wait_hint_ns;  // ... each of which may sleep this long in hardware
   volatile int abort;
 };
 
 __device__ __forceinline__ bool wait2(uint64_t* bar, uint32_t parity, FaSmem* sh, uint32_t* status, uint32_t code) {
   if (mbar_try_wait(bar, parity)) return true;
-  for (uint32_t i = 0; i < kWaitLimit2; ++i) {
-    if (mbar_try_wait_hint(bar, parity, 4000u)) return true;
+  const uint32_t limit = sh->wait_limit;
+  for (uint32_t i = 0; i < limit; ++i) {
+    if (mbar_try_wait_hint(bar, parity, sh->wait_hint_ns)) return true;
     if ((i & 63u) == 63u && sh->abort) return false;
   }
   sh->abort = 1;
@@ -52,6 +67,25 @@ __device__ __forceinline__ bool wait2(uint64_t* bar, uint32_t parity, FaSmem* sh
 }
 __device__ __forceinline__ bool warp_wait2(uint64_t* bar, uint32_t parity, FaSmem* sh, uint32_t* status, uint32_t code) {
   return __all_sync(0xffffffffu, wait2(bar, parity, sh, status, code));
+}
+
+// Exit protocol of the pipelined kernels.  A CTA may leave early (a wait gave up and set `abort`),
+// and even then nothing it started may outlive it: shared memory and tensor memory go back to
+// the SM when the CTA exits, so a bulk copy still landing or an MMA still reading would touch
+// memory that belongs to somebody else by then.
+//   producer warp   waits (bounded, generous) for every copy it issued and nobody consumed
+//   issuer warps    commit to their own barrier and wait for it: all their MMAs have completed
+// tcgen05.ld / tcgen05.st of the other warps are complete at their wait::ld / wait::st.  Only
+// then does the CTA reach the barrier in front of the tensor-memory release.
+__device__ __forceinline__ void drain_loads(FaSmem* sh, int issued) {
+  mbar_wait(&sh->q_full, 0, kDrainLimit);
+  for (int jj = issued > kStages2 ? issued - kStages2 : 0; jj < issued; ++jj)
+    mbar_wait(&sh->kv_full[jj % kStages2], (jj / kStages2) & 1, kDrainLimit);
+}
+__device__ __forceinline__ void drain_mmas(FaSmem* sh, int which) {
+  if (elect_one()) mma_commit(&sh->drain[which]);
+  __syncwarp();
+  mbar_wait(&sh->drain[which], 0, kDrainLimit);
 }
 
 // Block means as the B operand of the per-tile mean-restoration MMA: per (b, h, key tile) a

@@ -44,6 +44,8 @@ struct GroupArgs {
   int32_t* counts;       // [BH][chunks][kGroupK]
   int32_t* offsets;      // [BH][chunks][kGroupK]
   int32_t* perm;         // [BH][N]
+  uint32_t* status;      // status word (first word of the workspace)
+  uint32_t wait_limit;   // polls after which a wait gives up
 };
 
 template <int D>
@@ -68,22 +70,29 @@ __global__ void group_init_kernel(const GroupArgs a) {
 //   warps 0-3   one thread per token: scores from tensor memory, argmin, label, one-hot entry
 // Tensor memory: two score buffers of 64 columns | cluster sums (d columns, rows = clusters).
 constexpr int kGStages = 4;
-constexpr uint32_t kGroupWaitLimit = 1u << 22;
+constexpr uint32_t kGroupWaitLimit = 1u << 22;   // default number of polls of a wait
 
 struct GroupSmem {
   uint64_t v_full[kGStages], v_free[kGStages], s_full[2], s_free[2], oh_full, oh_free;
+  uint64_t drain;        // exit: "every MMA of the control warp has completed"
   float cnorm[kGroupK];
   int count_acc[kGroupK];
   uint32_t tmem_base;
   int abort;
+  uint32_t wait_limit;
+  uint32_t* status;
 };
 
+// Bounded wait.  When it gives up, the labels of this chunk are garbage (but in range) and the
+// status word says so: vc_poll_status on the workspace returns VC_ERR_TIMEOUT.
 __device__ __forceinline__ bool gwait(uint64_t* bar, uint32_t parity, GroupSmem* sh) {
-  for (uint32_t i = 0; i < kGroupWaitLimit; ++i) {
+  if (mbar_try_wait(bar, parity)) return true;
+  for (uint32_t i = 0; i < sh->wait_limit; ++i) {
     if (mbar_try_wait(bar, parity)) return true;
     if ((i & 255u) == 255u && *reinterpret_cast<volatile int*>(&sh->abort)) return false;
   }
-  *reinterpret_cast<volatile int*>(&sh->abort) = 1;     // labels of this chunk are then garbage but in range
+  *reinterpret_cast<volatile int*>(&sh->abort) = 1;
+  atomicExch(sh->status, kStatusTimeout | 0x60u);
   return false;
 }
 
@@ -132,7 +141,10 @@ __global__ void __launch_bounds__(160, 1) group_assign_kernel(const __grid_const
     for (int i = 0; i < kGStages; ++i) { mbar_init(&sh->v_full[i], 1); mbar_init(&sh->v_free[i], 1); }
     for (int i = 0; i < 2; ++i) { mbar_init(&sh->s_full[i], 1); mbar_init(&sh->s_free[i], 4); }
     mbar_init(&sh->oh_full, 128); mbar_init(&sh->oh_free, 1);
+    mbar_init(&sh->drain, 1);
     sh->abort = 0;
+    sh->wait_limit = a.wait_limit;
+    sh->status = a.status;
     mbar_fence_init();
     tma_prefetch_desc(&tm_v);
   }
@@ -190,8 +202,10 @@ __global__ void __launch_bounds__(160, 1) group_assign_kernel(const __grid_const
     // ------------------------------------------------------------------ loads and MMA issue
     const uint32_t idesc_s = idesc_bf16(128, kGroupK);
     const uint32_t idesc_sum = idesc_bf16(128, D) | (1u << 16);        // B operand MN-major
+    int loaded = 0;                                    // value tiles whose copies have been issued
     auto load = [&](int i) {
       const int st = i % kGStages;
+      loaded = i + 1;
       if (elect_one()) {
         mbar_expect_tx(&sh->v_full[st], kVStage);
         for (int kh = 0; kh < KH; ++kh)
@@ -244,6 +258,13 @@ __global__ void __launch_bounds__(160, 1) group_assign_kernel(const __grid_const
       }
       __syncwarp();
     }
+    // Nothing this CTA started may outlive it (shared and tensor memory are released at exit, also
+    // after a wait gave up): wait for the copies nobody consumed and for the MMAs issued so far.
+    for (int jj = loaded > kGStages ? loaded - kGStages : 0; jj < loaded; ++jj)
+      mbar_wait(&sh->v_full[jj % kGStages], (jj / kGStages) & 1, 1u << 22);
+    if (elect_one()) mma_commit(&sh->drain);
+    __syncwarp();
+    mbar_wait(&sh->drain, 0, 1u << 22);
   } else {
     // ------------------------------------------------------------------ labels and one-hot entries
     const uint32_t lane_base = tmem + ((uint32_t)(warp * 32) << 16);
@@ -410,7 +431,7 @@ cudaError_t run_group(const Problem& pr, GroupArgs a, int iters, int warm, cudaS
 }
 
 struct GroupLayout {
-  size_t labels, psum, counts, offsets, total;
+  size_t status, labels, psum, counts, offsets, total;
   int chunks;
 };
 GroupLayout group_layout(const Problem& pr) {
@@ -418,6 +439,7 @@ GroupLayout group_layout(const Problem& pr) {
   g.chunks = (pr.N + kChunk - 1) / kChunk;
   size_t off = 0;
   auto place = [&](size_t bytes) { size_t o = off; off = (off + bytes + 1023) / 1024 * 1024; return o; };
+  g.status = place(VC_GROUP_LABELS_OFFSET);          // the status word, then the labels
   g.labels = place((size_t)pr.BH * pr.N * 4);
   g.psum = place((size_t)pr.BH * g.chunks * kGroupK * pr.d * 4);
   g.counts = place((size_t)pr.BH * g.chunks * kGroupK * 4);
@@ -458,6 +480,10 @@ extern "C" vc_status vc_group(const vc_params* p, const void* v, int32_t k, int3
   a.counts = (int32_t*)(work + gl.counts);
   a.offsets = (int32_t*)(work + gl.offsets);
   a.perm = perm;
+  a.status = (uint32_t*)(work + gl.status);
+  const uint32_t lim = wait_limit_override();
+  a.wait_limit = lim ? lim : kGroupWaitLimit;
+  if (cudaMemsetAsync(a.status, 0, 4, (cudaStream_t)stream) != cudaSuccess) return VC_ERR_CUDA;
   const cudaError_t e = pr.d == 128 ? run_group<128>(pr, a, iters, warm_start, (cudaStream_t)stream)
                                     : run_group<64>(pr, a, iters, warm_start, (cudaStream_t)stream);
   return e == cudaSuccess ? VC_OK : VC_ERR_CUDA;

@@ -13,57 +13,10 @@
 // can be processed in groups so that the second read of K and V may hit L2.  All passes are
 // persistent kernels that prefetch the next row blocks with cp.async while they transform
 // the current one.
-#include <cuda_bf16.h>
-#include <cuda_fp4.h>
-#include <cuda_fp8.h>
-
-#include "vc_internal.h"
-#include "vc_sm100.cuh"
+#include "vc_prep_common.cuh"
 
 namespace vc {
 namespace {
-
-using namespace sm100;
-
-struct RopeDesc {
-  int pair_start[3];   // first channel pair of each axis
-  int pairs[3];        // channel pairs per axis
-  int off[3];          // entry offset of each axis table
-  int len[3];          // positions per axis
-  int entries;
-  int grid_h, grid_w;
-  unsigned long long mul_w, mul_h;   // ceil(2^40 / divisor)
-};
-
-struct PrepArgs {
-  const __nv_bfloat16 *q, *k, *v;
-  const int32_t* perm;
-  int64_t stride_b, stride_h, stride_n;
-  int H, N, n_pad, nb, bh0, flags, rope_in_smem, rope_default;
-  uint8_t *q_codes, *k_codes, *v_codes, *q_micro, *k_micro, *v_micro;
-  float *q_scale, *k_scale, *v_scale, *k_mean;
-  __nv_bfloat16* v_means;
-  const float2* rope;
-  float *k_part, *v_mu;
-  unsigned int *v_amax, *qk_amax;   // qk_amax: [2][BH]
-  int BH;
-  RopeDesc rd;
-};
-
-__device__ __forceinline__ unsigned int div40(unsigned int x, unsigned long long mul) {
-  return (unsigned int)(((unsigned long long)x * mul) >> 40);
-}
-
-__device__ __forceinline__ float warp_max(float v) {
-#pragma unroll
-  for (int s = 16; s > 0; s >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, s));
-  return v;
-}
-
-__device__ __forceinline__ float e4m3_to_float(unsigned int code) {
-  __half_raw h = __nv_cvt_fp8_to_halfraw((__nv_fp8_storage_t)code, __NV_E4M3);
-  return __half2float(__half(h));
-}
 
 // ---------------------------------------------------------------------------------------
 // RoPE tables: per axis a, entry [pos][i] = (cos, sin)(pos * theta^(-2 i / d_a)), evaluated
@@ -101,12 +54,6 @@ template <int D> struct Geo {
   static constexpr int stage_bytes = kBlock * pitch;
 };
 
-__device__ __forceinline__ void cp_async16(void* dst, const void* src) {
-  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_u32(dst)), "l"(src) : "memory");
-}
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
-
 struct Item {
   int z, bh, blk;
 };
@@ -118,14 +65,6 @@ __device__ __forceinline__ Item decode_item(int item, int nb, int nh, int bh0) {
   it.bh = bh0 + r % nh;
   it.z = r / nh;
   return it;
-}
-
-// Token position -> (t, y, x) of the grid.
-__device__ __forceinline__ void grid_pos(const RopeDesc& rd, int src, int& tt, int& ty, int& tx) {
-  const unsigned int q1 = div40((unsigned)src, rd.mul_w);
-  tx = src - q1 * rd.grid_w;
-  tt = div40(q1, rd.mul_h);
-  ty = q1 - tt * rd.grid_h;
 }
 
 // ---------------------------------------------------------------------------------------
@@ -704,7 +643,7 @@ __global__ void __launch_bounds__(kThreads, 2) prep_v_kernel(const PrepArgs a, i
 #pragma unroll
     for (int c = 0; c < NL; ++c) {
       const int t = w.blk * kBlock + (tid + c * kThreads) / LPR;
-      if (t < a.N) src[c] = a.perm ? __ldg(prow + t) : t;
+      if (t < a.N) src[c] = a.perm ? min(max(__ldg(prow + t), 0), a.N - 1) : t;   // clamped: never a bad address
     }
   };
   auto issue = [&](int item, const Item& w, int st, const int (&src)[NL]) {
@@ -801,7 +740,7 @@ __global__ void __launch_bounds__(kRowThreads * TPR, 2) prep_qk_kernel(const Pre
     if (t >= a.N) return -1;
     // the head amax is a maximum over all rows: that stage reads the rows in place
     const bool gather = (w.z + z0) == 1 && a.perm != nullptr && STAGE != kStageAmax;
-    return gather ? __ldg(&a.perm[(size_t)w.bh * a.N + t]) : t;
+    return gather ? min(max(__ldg(&a.perm[(size_t)w.bh * a.N + t]), 0), a.N - 1) : t;   // clamped: never a bad address
   };
   auto issue = [&](int item, int st, const int* src) {
     if (item < n_items) {
@@ -886,13 +825,6 @@ cudaError_t run(const Problem& pr, PrepArgs a, const WorkLayout& wl, uint8_t* wo
   if ((e = allow_smem(prep_qk_kernel<D, kQuant, kTpr>, row_smem)) != cudaSuccess) return e;
   if (BITS == 8 && (e = allow_smem(prep_qk_kernel<D, kStageQuant8I, kTpr>, row_smem)) != cudaSuccess) return e;
   if (BITS == 4 && (e = allow_smem(prep_qk_kernel<D, kStageAmax, kTpr>, row_smem)) != cudaSuccess) return e;
-  if ((e = cudaMemsetAsync(work + wl.status, 0, 4, s)) != cudaSuccess) return e;
-  if ((e = cudaMemsetAsync(work + wl.amax, 0, wl.amax_bytes, s)) != cudaSuccess) return e;
-  if (a.flags & VC_FLAG_ROPE) {
-    rope_table_kernel<<<(a.rd.entries + 255) / 256, 256, 0, s>>>(
-        reinterpret_cast<float2*>(work + wl.rope), a.rd, (double)pr.rope_theta);
-    count_launches(1);
-  }
   int group = pr.heads_per_pass > 0 ? pr.heads_per_pass : pr.BH;
   if (group > 32768) group = 32768;
   for (int bh0 = 0; bh0 < pr.BH; bh0 += group) {
@@ -962,8 +894,18 @@ cudaError_t launch_prep(const Problem& pr, const QuantLayout& ql, const WorkLayo
     const int sdef = 2 * (pr.d / 6);
     a.rope_default = pr.rope_dim[0] == pr.d - 2 * sdef && pr.rope_dim[1] == sdef && pr.rope_dim[2] == sdef;
   }
-  if (pr.d == 128) return pr.bits == 8 ? run<128, 8>(pr, a, wl, work, stream) : run<128, 4>(pr, a, wl, work, stream);
-  return pr.bits == 8 ? run<64, 8>(pr, a, wl, work, stream) : run<64, 4>(pr, a, wl, work, stream);
+  cudaError_t e;
+  if ((e = cudaMemsetAsync(work + wl.status, 0, 4, stream)) != cudaSuccess) return e;
+  if ((e = cudaMemsetAsync(work + wl.amax, 0, wl.amax_bytes, stream)) != cudaSuccess) return e;
+  if (a.flags & VC_FLAG_ROPE) {
+    rope_table_kernel<<<(a.rd.entries + 255) / 256, 256, 0, stream>>>(
+        reinterpret_cast<float2*>(work + wl.rope), a.rd, (double)pr.rope_theta);
+    count_launches(1);
+  }
+  if ((e = launch_perm_check(pr, perm, wl, work, stream)) != cudaSuccess) return e;
+  // 8 bits: one fused persistent launch; 4 bits: the pass-per-launch kernels of this file
+  if (pr.bits == 8) return launch_prep8(pr, a, wl, work, stream);
+  return pr.d == 128 ? run<128, 4>(pr, a, wl, work, stream) : run<64, 4>(pr, a, wl, work, stream);
 }
 
 }  // namespace vc

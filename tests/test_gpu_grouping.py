@@ -34,7 +34,9 @@ def _run(p, v, k, iters, warm=False, centroids=None):
     perm = torch.empty(p.B, p.H, p.N, dtype=torch.int32, device="cuda")
     vc.vc_group(p, v, k, iters, warm, centroids, perm, work)
     torch.cuda.synchronize()
-    labels = work[: p.B * p.H * p.N * 4].view(torch.int32).view(p.B, p.H, p.N).clone()
+    off = vc.VC_GROUP_LABELS_OFFSET
+    labels = work[off: off + p.B * p.H * p.N * 4].view(torch.int32).view(p.B, p.H, p.N).clone()
+    vc.vc_poll_status(work)
     return perm, centroids, labels
 
 

@@ -37,13 +37,27 @@ def test_sizes_and_argument_validation_without_a_gpu():
     assert vc.vc_quant_bytes(Params.make(1, 2, 1024, 128, (4, 16, 16), bits=4, p_format=vc.VC_P_EXPCAST_E4M3, kernel_variant=1)) == 0
     assert vc.vc_quant_bytes(Params.make(1, 2, 1024, 128, (4, 16, 16), bits=4, p_format=vc.VC_P_EXP_E4M3)) == 0
     assert vc.vc_quant_bytes(Params.make(1, 2, 1024, 128, (4, 16, 16), bits=8, p_format=vc.VC_P_EXP_POLY_E4M3)) > 0
+    qb0 = vc.vc_quant_bytes(Params.make(1, 2, 1024, 128, (4, 16, 16)))
     for bad in (dict(d=100), dict(N=-1), dict(bits=3), dict(grid_t=20), dict(p_format=9), dict(B=40000)):
         pb = Params.make(1, 2, 1024, 128, (4, 16, 16))
         for k, v in bad.items():
             setattr(pb, k, v)
         assert vc.vc_quant_bytes(pb) == 0 and vc.vc_workspace_bytes(pb) == 0
     assert vc.vc_status_string(0) == "ok" and "timed out" in vc.vc_status_string(5)
-    assert ctypes.sizeof(Params) == 96
+    assert ctypes.sizeof(Params) == 112
+    # block sizes are arguments (Eq. 4's B_v, the scale blocks): 0 means 128, nothing else is implemented
+    assert vc.vc_quant_bytes(Params.make(1, 2, 1024, 128, (4, 16, 16), block_q=128, block_k=128, block_v=128)) == qb0
+    for name in ("block_q", "block_k", "block_v"):
+        assert vc.vc_quant_bytes(Params.make(1, 2, 1024, 128, (4, 16, 16), **{name: 64})) == 0
+    import ctypes as C
+    lib = vc.load_library()
+    pb = Params.make(1, 2, 1024, 128, (4, 16, 16), block_v=64)
+    assert lib.vc_prep(C.byref(pb), 16, 16, 16, None, 16, 16, None) == vc.VC_ERR_UNSUPPORTED      # refused before any launch
+    pb = Params.make(1, 2, 1024, 128, (4, 16, 16), block_v=-1)
+    assert lib.vc_prep(C.byref(pb), 16, 16, 16, None, 16, 16, None) == vc.VC_ERR_INVALID_ARG
+    # the validator's bitmap is part of the workspace only when it is asked for
+    pc = Params.make(1, 2, 1024, 128, (4, 16, 16), flags=vc.VC_FLAG_ALL | vc.VC_FLAG_CHECK_PERM)
+    assert vc.vc_workspace_bytes(pc) > vc.vc_workspace_bytes(Params.make(1, 2, 1024, 128, (4, 16, 16)))
     assert vc.vc_launch_count() == 0
 
 
