@@ -23,6 +23,7 @@ sys.path.insert(0, ROOT)
 import torch  # noqa: E402
 
 import vc_inputs  # noqa: E402
+import vc_kmeans_harness  # noqa: E402
 
 METRIC = "quantized attn fwd TFLOPS (hot path: prep + attention forward)"
 UNIT = "TFLOP/s"
@@ -281,7 +282,7 @@ def main():
         perm = torch.empty(w.B, w.H, w.N, dtype=torch.int32, device=dev)
         vc.vc_group(p, v, group_k, 4, False, centroids, perm, gwork)      # cold start: 4 Lloyd iterations
     elif args.perm == "kmeans":
-        perm = vc_inputs.kmeans_perm_all(v)
+        perm = vc_kmeans_harness.kmeans_perm_all(v)
     elif args.perm == "random":
         perm = vc_inputs.random_perm(w.B, w.H, w.N, w.seed, device=dev)
     else:

@@ -155,10 +155,7 @@ size_t vc_workspace_bytes(const vc_params *p);
  * permutation of [0, N) per (b, h).  Entries are clamped into [0, N) before they are used
  * as row indices; VC_FLAG_CHECK_PERM adds a validator that reports a bad entry through the
  * status word.  Writes `quant`; uses `workspace` (contents on entry irrelevant; the first 4
- * bytes become the status word).  At 8 bits the pass is ONE persistent launch: statistics
- * items (K column sums, V block means and residual maxima) of a head run ahead of its
- * quantizing items, which wait on a per-head counter in the workspace with a bounded spin
- * (VC_ERR_TIMEOUT through the status word if it gives up); heads_per_pass is ignored there. */
+ * bytes become the status word). */
 vc_status vc_prep(const vc_params *p, const void *q, const void *k, const void *v,
                   const int32_t *perm, void *quant, void *workspace, void *stream);
 
@@ -244,7 +241,8 @@ int32_t vc_group_schedule(int32_t step, int32_t n_steps, int32_t reuse);
  *     without ordering between their streams) race on the array: serialize them.
  *   - The first call on each device looks up the array's device address
  *     (cudaGetSymbolAddress) with that device current; make that first call outside any
- *     stream capture.  Later calls only launch kernels and two small memsets on `stream`.
+ *     stream capture.  Later calls only set the kernels' shared-memory attribute (a host-side
+ *     call that allocates nothing), launch kernels and issue two small memsets on `stream`.
  * It calls no cudaMalloc / cudaFree and no allocating library routine.  The output is
  * the same bundle vc_prep writes. */
 #define VC_NOALLOC_SCRATCH_BYTES (4u << 20)

@@ -149,6 +149,24 @@ def emulate_head(bundle, cfg, p_format=None, softmax_scale=None, beta=C.EXPCAST_
     return C.bf16_round(o)
 
 
+def reference_scores(q, k, cfg, row, softmax_scale=None):
+    """Exact fp64 scores (natural-log domain) of one query row of the rotated Q against all rotated
+    keys: what the softmax of Sec. 3.1 sees (a diagnostic: effective keys 1 / sum p^2 of a row)."""
+    from .prep import rope_tables
+    q = np.asarray(q, dtype=np.float64)[row:row + 1]
+    k = np.asarray(k, dtype=np.float64)
+    if cfg.rope:
+        cos, sin = rope_tables(cfg)
+        def rot(x, c, s):
+            out = np.empty_like(x)
+            out[:, 0::2] = x[:, 0::2] * c - x[:, 1::2] * s
+            out[:, 1::2] = x[:, 0::2] * s + x[:, 1::2] * c
+            return out
+        q, k = rot(q, cos[row:row + 1], sin[row:row + 1]), rot(k, cos, sin)
+    scale = 1.0 / np.sqrt(q.shape[1]) if softmax_scale is None else softmax_scale
+    return (q @ k.T)[0] * scale
+
+
 def reference_head(q, k, v, cfg, rows=None, softmax_scale=None):
     """O0: exact fp64 attention of the rotated Q, K (no permutation, smoothing or
     Hadamard: each of them leaves the exact output unchanged)."""

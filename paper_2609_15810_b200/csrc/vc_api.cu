@@ -121,8 +121,6 @@ WorkLayout work_layout(const Problem& pr) {
   W.v_mu = place(BH * nb * d * 4);
   W.amax_bytes = BH * d * 4 + 2 * BH * 4;
   W.amax = place(W.amax_bytes);
-  W.sync_bytes = (2 * BH + 4) * 4;
-  W.sync = place(W.sync_bytes);
   W.perm_bits_bytes = (pr.flags & VC_FLAG_CHECK_PERM) ? BH * (((size_t)pr.N + 31) / 32) * 4 : 0;
   W.perm_bits = place(W.perm_bits_bytes);
   W.mu_mma = place(BH * nb * d * 32);

@@ -37,8 +37,9 @@ inline uint32_t attn_wait_limit() {
   const uint32_t lim = wait_limit_override();
   return lim ? lim : kWaitLimit2;
 }
-// with the test override a poll does not sleep, so that a tiny limit really is a short wait
-inline uint32_t attn_wait_hint_ns() { return wait_limit_override() ? 32u : 4000u; }
+// with the test override a poll never sleeps (hint 0 selects non-blocking tests of the barrier),
+// so that a tiny limit really is a short wait
+inline uint32_t attn_wait_hint_ns() { return wait_limit_override() ? 0u : 4000u; }
 
 struct FaSmem {
   uint64_t q_full, kv_full[kStages2], kv_empty[kStages2];
@@ -55,11 +56,18 @@ struct FaSmem {
 };
 
 __device__ __forceinline__ bool wait2(uint64_t* bar, uint32_t parity, FaSmem* sh, uint32_t* status, uint32_t code) {
-  if (mbar_try_wait(bar, parity)) return true;
-  const uint32_t limit = sh->wait_limit;
-  for (uint32_t i = 0; i < limit; ++i) {
-    if (mbar_try_wait_hint(bar, parity, sh->wait_hint_ns)) return true;
-    if ((i & 63u) == 63u && sh->abort) return false;
+  const uint32_t limit = sh->wait_limit, hint = sh->wait_hint_ns;
+  if (hint) {
+    if (mbar_try_wait(bar, parity)) return true;
+    for (uint32_t i = 0; i < limit; ++i) {
+      if (mbar_try_wait_hint(bar, parity, hint)) return true;
+      if ((i & 63u) == 63u && sh->abort) return false;
+    }
+  } else {                                     // test hook: polls that never sleep
+    for (uint32_t i = 0; i < limit; ++i) {
+      if (mbar_test_wait(bar, parity)) return true;
+      if ((i & 63u) == 63u && sh->abort) return false;
+    }
   }
   sh->abort = 1;
   atomicExch(status, kErrTimeout | code);

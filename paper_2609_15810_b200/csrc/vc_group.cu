@@ -46,6 +46,7 @@ struct GroupArgs {
   int32_t* perm;         // [BH][N]
   uint32_t* status;      // status word (first word of the workspace)
   uint32_t wait_limit;   // polls after which a wait gives up
+  uint32_t nonblocking;  // test hook: polls test the barrier without sleeping in hardware
 };
 
 template <int D>
@@ -79,16 +80,16 @@ struct GroupSmem {
   int count_acc[kGroupK];
   uint32_t tmem_base;
   int abort;
-  uint32_t wait_limit;
+  uint32_t wait_limit, nonblocking;
   uint32_t* status;
 };
 
 // Bounded wait.  When it gives up, the labels of this chunk are garbage (but in range) and the
 // status word says so: vc_poll_status on the workspace returns VC_ERR_TIMEOUT.
 __device__ __forceinline__ bool gwait(uint64_t* bar, uint32_t parity, GroupSmem* sh) {
-  if (mbar_try_wait(bar, parity)) return true;
+  if (!sh->nonblocking && mbar_try_wait(bar, parity)) return true;
   for (uint32_t i = 0; i < sh->wait_limit; ++i) {
-    if (mbar_try_wait(bar, parity)) return true;
+    if (sh->nonblocking ? mbar_test_wait(bar, parity) : mbar_try_wait(bar, parity)) return true;
     if ((i & 255u) == 255u && *reinterpret_cast<volatile int*>(&sh->abort)) return false;
   }
   *reinterpret_cast<volatile int*>(&sh->abort) = 1;
@@ -144,6 +145,7 @@ __global__ void __launch_bounds__(160, 1) group_assign_kernel(const __grid_const
     mbar_init(&sh->drain, 1);
     sh->abort = 0;
     sh->wait_limit = a.wait_limit;
+    sh->nonblocking = a.nonblocking;
     sh->status = a.status;
     mbar_fence_init();
     tma_prefetch_desc(&tm_v);
@@ -483,6 +485,7 @@ extern "C" vc_status vc_group(const vc_params* p, const void* v, int32_t k, int3
   a.status = (uint32_t*)(work + gl.status);
   const uint32_t lim = wait_limit_override();
   a.wait_limit = lim ? lim : kGroupWaitLimit;
+  a.nonblocking = lim ? 1u : 0u;
   if (cudaMemsetAsync(a.status, 0, 4, (cudaStream_t)stream) != cudaSuccess) return VC_ERR_CUDA;
   const cudaError_t e = pr.d == 128 ? run_group<128>(pr, a, iters, warm_start, (cudaStream_t)stream)
                                     : run_group<64>(pr, a, iters, warm_start, (cudaStream_t)stream);

@@ -45,8 +45,6 @@ struct WorkLayout {
   size_t v_mu;       // fp32 [BH][nb][d] block means of the gathered V
   size_t amax;       // uint32 [BH][d] residual amax bits (8-bit V) then [2][BH] Q/K head amax (4-bit)
   size_t amax_bytes;
-  size_t sync;       // uint32 [2 BH + 4]: per-head statistics counters, per-head ready flags, abort word (fused 8-bit pass)
-  size_t sync_bytes;
   size_t perm_bits;  // uint32 [BH][ceil(N / 32)]: bitmap of the permutation validator (VC_FLAG_CHECK_PERM)
   size_t perm_bits_bytes;
   size_t mu_mma;     // fp32 [BH][nb][d][8]: block means as the B operand of the mean-restoration MMA
@@ -74,11 +72,8 @@ cudaError_t launch_attn_fwd(const Problem& pr, const QuantLayout& ql, const Work
 cudaError_t launch_attn_fwd4(const Problem& pr, const QuantLayout& ql, const WorkLayout& wl,
                              const uint8_t* quant, void* o, uint8_t* work, cudaStream_t stream);
 
-// The fused 8-bit preprocessing pass (vc_prep8.cu): one persistent launch.
-struct PrepArgs;
 // Validator of the permutation (VC_FLAG_CHECK_PERM); the status word must have been cleared before.
 cudaError_t launch_perm_check(const Problem& pr, const int32_t* perm, const WorkLayout& wl, uint8_t* work, cudaStream_t stream);
-cudaError_t launch_prep8(const Problem& pr, const PrepArgs& a, const WorkLayout& wl, uint8_t* work, cudaStream_t stream);
 
 void count_launches(int n);
 

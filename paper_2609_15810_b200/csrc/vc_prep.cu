@@ -797,11 +797,14 @@ cudaError_t allow_smem(K kernel, size_t bytes) {
 }
 
 int persistent_grid(int n_items, int per_sm = 2) {
-  static int sms = 0;
-  if (!sms) {
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
-      sms = 148;
+  // SM count of the CURRENT device (cached per device: a process may drive GPUs of different sizes)
+  static int cache[64] = {};
+  int dev = 0, sms = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) dev = -1;
+  if (dev >= 0 && dev < 64 && cache[dev] > 0) sms = cache[dev];
+  else {
+    if (dev < 0 || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0) sms = 148;
+    if (dev >= 0 && dev < 64) cache[dev] = sms;
   }
   const int g = per_sm * sms;
   return n_items < g ? n_items : g;
@@ -903,9 +906,8 @@ cudaError_t launch_prep(const Problem& pr, const QuantLayout& ql, const WorkLayo
     count_launches(1);
   }
   if ((e = launch_perm_check(pr, perm, wl, work, stream)) != cudaSuccess) return e;
-  // 8 bits: one fused persistent launch; 4 bits: the pass-per-launch kernels of this file
-  if (pr.bits == 8) return launch_prep8(pr, a, wl, work, stream);
-  return pr.d == 128 ? run<128, 4>(pr, a, wl, work, stream) : run<64, 4>(pr, a, wl, work, stream);
+  if (pr.d == 128) return pr.bits == 8 ? run<128, 8>(pr, a, wl, work, stream) : run<128, 4>(pr, a, wl, work, stream);
+  return pr.bits == 8 ? run<64, 8>(pr, a, wl, work, stream) : run<64, 4>(pr, a, wl, work, stream);
 }
 
 }  // namespace vc

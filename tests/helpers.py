@@ -67,16 +67,27 @@ def gpu_sections(p, quant):
 
 
 def upload_bundle(p, quant, bundles):
-    """Writes the oracle's bundles (list over b*H+h) into the device bundle (8-bit)."""
-    assert p.bits == 8
+    """Writes the oracle's bundles (list over b*H+h) into the device bundle, in the layout the ABI
+    documents: bytes at 8 bits; at 4 bits nibbles two per byte (even index low), microscale bytes
+    beside them, the outer scales of Q and K in q_scale / k_scale."""
     view = vc.vc_quant_view(p, quant)
     put = lambda name, arr, dt=torch.uint8: section(view, name, quant, dt).copy_(
         torch.from_numpy(np.ascontiguousarray(arr)).view(dt).reshape(-1).to(quant.device))
-    put("q_codes", np.stack([b["q_codes"] for b in bundles]))
-    put("k_codes", np.stack([b["k_codes"] for b in bundles]))
-    put("v_codes", np.stack([b["v_codes"].T for b in bundles]))
-    put("q_scale", np.stack([b["q_scale"] for b in bundles]).astype(np.float32), torch.float32)
-    put("k_scale", np.stack([b["k_scale"] for b in bundles]).astype(np.float32), torch.float32)
+    if p.bits == 8:
+        put("q_codes", np.stack([b["q_codes"] for b in bundles]).view(np.uint8))
+        put("k_codes", np.stack([b["k_codes"] for b in bundles]).view(np.uint8))
+        put("v_codes", np.stack([b["v_codes"].T for b in bundles]))
+        put("q_scale", np.stack([b["q_scale"] for b in bundles]).astype(np.float32), torch.float32)
+        put("k_scale", np.stack([b["k_scale"] for b in bundles]).astype(np.float32), torch.float32)
+    else:
+        put("q_codes", np.stack([CMP.pack_nibbles(b["q_codes"]) for b in bundles]))
+        put("k_codes", np.stack([CMP.pack_nibbles(b["k_codes"]) for b in bundles]))
+        put("v_codes", np.stack([CMP.pack_nibbles(np.ascontiguousarray(b["v_codes"].T)) for b in bundles]))
+        put("q_micro", np.stack([b["q_micro"] for b in bundles]))
+        put("k_micro", np.stack([b["k_micro"] for b in bundles]))
+        put("v_micro", np.stack([np.ascontiguousarray(b["v_micro"].T) for b in bundles]))
+        put("q_scale", np.array([b["q_g"] for b in bundles], dtype=np.float32), torch.float32)
+        put("k_scale", np.array([b["k_g"] for b in bundles], dtype=np.float32), torch.float32)
     put("v_scale", np.stack([b["v_scale"] for b in bundles]).astype(np.float32), torch.float32)
     put("k_mean", np.stack([b["k_mean"] for b in bundles]).astype(np.float32), torch.float32)
     means = np.stack([OC.bf16_bits(b["v_means"]) for b in bundles]).view(np.int16)
@@ -88,7 +99,10 @@ def check_prep_head(p, got, bh, ref, what=""):
     mag = 7 if p.bits == 8 else 3
     rel = lambda a, b: float(np.max(np.abs(a - b) / np.maximum(np.abs(b), 1e-30)))
     stats = {}
-    assert rel(got["k_mean"][bh], ref["k_mean"]) < 1e-4 or np.abs(got["k_mean"][bh] - ref["k_mean"]).max() < 1e-5, what
+    # the channel mean of K as a VECTOR: 1e-5 of its largest component.  (An fp32 sum of N values
+    # of size A is off by about A 2^-24 sqrt(N), whatever the size of the mean itself, so a
+    # component that happens to lie near zero cannot be held to 1e-5 of its own value.)
+    assert np.abs(got["k_mean"][bh] - ref["k_mean"]).max() <= 1e-5 * max(np.abs(ref["k_mean"]).max(), 1e-30), what + " k_mean"
     if p.bits == 8:
         assert rel(got["q_scale"][bh], ref["q_scale"]) < 1e-5, what + " q_scale"
         assert rel(got["k_scale"][bh], ref["k_scale"]) < 1e-5, what + " k_scale"
@@ -107,13 +121,22 @@ def check_prep_head(p, got, bh, ref, what=""):
         elif p.bits == 8:
             stats[t] = CMP.assert_codes_close(got[t + "_codes"][bh], ref[t + "_codes"], mag, what=what + " " + t + "_codes")
         else:
-            # elements under a differing microscale are compared after decoding
-            same = np.repeat(got[t + "_micro"][bh] == ref[t + "_micro"], 32 if t == "v" and is_hybrid(p) else 16,
-                             axis=1 if t != "v" else 0)
+            # under the same microscale: codes identical except <= 0.1 % one step apart; under a
+            # differing microscale (itself one step apart, counted above): compared after decoding,
+            # within one element step of the larger microscale (the widest E2M1 gap is 2)
+            grp = 32 if t == "v" and is_hybrid(p) else 16
+            ax = 1 if t != "v" else 0
+            gm, rm = got[t + "_micro"][bh], ref[t + "_micro"]
+            same = np.repeat(gm == rm, grp, axis=ax)
             g, r = got[t + "_codes"][bh], ref[t + "_codes"]
             frac, dist = CMP.code_mismatch(g[same], r[same], 3)
             assert dist <= 1 and frac <= 1e-3, f"{what} {t}_codes: frac {frac:.2e} dist {dist}"
             stats[t] = frac
+            if not same.all():
+                dec = (lambda m: np.exp2(m.astype(np.float64) - 127.0)) if (t == "v" and is_hybrid(p)) else OC.e4m3_decode
+                sg, sr = np.repeat(dec(gm), grp, axis=ax), np.repeat(dec(rm), grp, axis=ax)
+                dg, dr = OC.e2m1_decode(g) * sg, OC.e2m1_decode(r) * sr
+                assert np.all(np.abs(dg - dr)[~same] <= 2.0 * np.maximum(sg, sr)[~same] * (1 + 1e-9)), f"{what} {t}_codes under differing microscales"
     # block means: at most one bf16 ulp
     gm, rm = got["v_means"][bh], ref["v_means"]
     ulp = np.maximum(np.abs(rm), 1e-30) * 2.0 ** -7

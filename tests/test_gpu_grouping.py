@@ -11,6 +11,7 @@ import torch
 
 import paper_2609_15810_b200 as vc
 import vc_inputs
+import vc_kmeans_harness
 from paper_2609_15810_b200.binding import Params, alloc_buffers
 from oracle import attention as OA
 from oracle import grouping as OG
@@ -117,7 +118,7 @@ def test_group_fullsize_config3_properties():
     same = sl[..., 1:] == sl[..., :-1]
     assert (perm[..., 1:][same] > perm[..., :-1][same]).all()          # stable inside a cluster
     for h in range(H):
-        ref_perm, ref_c = vc_inputs.kmeans_perm(v[0, h], k=64, iters=4)
+        ref_perm, ref_c = vc_kmeans_harness.kmeans_perm(v[0, h], k=64, iters=4)
         x = v[0, h].float()
         obj_g = ((x - cent[0, h][labels[0, h].long()]) ** 2).sum()
         d2 = (x * x).sum(1, keepdim=True) - 2.0 * (x @ ref_c.T) + (ref_c * ref_c).sum(1)[None, :]

@@ -12,6 +12,7 @@ import torch
 
 import paper_2609_15810_b200 as vc
 import vc_inputs
+import vc_kmeans_harness
 from paper_2609_15810_b200.binding import Params, alloc_buffers
 from oracle import attention as OA
 from oracle import compare as CMP
@@ -103,13 +104,45 @@ def test_attn_fwd_on_oracle_bundle(case, p_format):
         assert m["max_err_over_vmax"] < 1e-2, m
 
 
+@pytest.mark.parametrize("arrangement", ["nvfp4", "hybrid", "nvfp4_serial"])
+@pytest.mark.parametrize("case", SMALL, ids=[c[0] for c in SMALL])
+def test_attn_fwd_4bit_on_oracle_bundle(case, arrangement):
+    """Stage 2 at 4 bits: the attention kernels fed the ORACLE's bundle (nibbles, microscales or
+    power-of-two factors, outer scales uploaded through the ABI's layout), so that a difference
+    in the output cannot come from a code flip in vc_prep."""
+    _, B, H, N, d, grid = case
+    q, k, v = _inputs(B, H, N, d, grid, seed=61)
+    perm = vc_inputs.random_perm(B, H, N, 12).cuda()
+    hybrid = arrangement == "hybrid"
+    p = Params.make(B, H, N, d, grid, bits=4, p_format=vc.VC_P_EXPCAST_E4M3 if hybrid else vc.VC_P_DEFAULT,
+                    kernel_variant=1 if arrangement == "nvfp4_serial" else 0)
+    quant, work = alloc_buffers(p)
+    quant.zero_()
+    bundles, refs = [], []
+    for b in range(B):
+        for h in range(H):
+            bundle, cfg = Hh.oracle_prep(p, q, k, v, perm, b, h)
+            bundles.append(bundle)
+            refs.append(OA.emulate_head(bundle, cfg, p_format=OA.P_EXPCAST if hybrid else None))
+    Hh.upload_bundle(p, quant, bundles)
+    got = Hh.gpu_sections(p, quant)                      # the upload reads back as the oracle's bundle
+    assert np.array_equal(got["k_codes"][0], bundles[0]["k_codes"]) and np.array_equal(got["v_micro"][0], bundles[0]["v_micro"])
+    o = torch.empty(B, H, N, d, dtype=torch.bfloat16, device="cuda")
+    vc.vc_attn_fwd(p, quant, o, work)
+    vc.vc_poll_status(work)
+    vmax = float(v.float().abs().max())
+    for i, ref in enumerate(refs):
+        m = Hh.check_output(o.view(B * H, N, d)[i].float().cpu().numpy(), ref, vmax)
+        assert m["max_err_over_vmax"] < 1e-2, m
+
+
 @pytest.mark.parametrize("perm_kind", ["identity", "random", "kmeans"])
 def test_vc_attn_end_to_end_config1(perm_kind):
     """Stage 3 on the tiny correctness configuration (B=1, H=2, N=1024, d=128, 8-bit)."""
     w = vc_inputs.WORKLOADS["c1"]
     q, k, v = [t.cuda() for t in vc_inputs.make_qkv(w)]
     perm = {"identity": None, "random": vc_inputs.random_perm(w.B, w.H, w.N, 7).cuda(),
-            "kmeans": vc_inputs.kmeans_perm_all(v, k=8)}[perm_kind]
+            "kmeans": vc_kmeans_harness.kmeans_perm_all(v, k=8)}[perm_kind]
     p = Params.make(w.B, w.H, w.N, w.d, w.grid, bits=8)
     quant, work = alloc_buffers(p)
     o = torch.empty(w.B, w.H, w.N, w.d, dtype=torch.bfloat16, device="cuda")

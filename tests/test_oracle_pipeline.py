@@ -9,6 +9,7 @@ import pytest
 import torch
 
 import vc_inputs
+import vc_kmeans_harness
 from oracle import attention as A
 from oracle import codecs as C
 from oracle import prep as P
@@ -280,7 +281,7 @@ def test_inputs_are_reproducible_and_shaped():
     assert k.mean(0).std() > 1.5                                          # channel offsets ~ N(0, 9)
     p = vc_inputs.random_perm(1, 2, 1024, 3)
     assert sorted(p[0, 1].tolist()) == list(range(1024))
-    pk, _ = vc_inputs.kmeans_perm(a[2][0, 0], k=8)
+    pk, _ = vc_kmeans_harness.kmeans_perm(a[2][0, 0], k=8)
     assert sorted(pk.tolist()) == list(range(1024))
 
 

@@ -51,6 +51,26 @@ def test_noalloc_matches_vc_prep_on_two_calls_in_a_row(bits):
         assert torch.equal(got, want), f"{w.name}: {(got != want).sum().item()} bytes differ"
 
 
+def test_noalloc_takes_no_device_memory():
+    """The property the entry point is named for: once the first call on the device has looked
+    up the array's address, a call changes neither the driver's free-memory figure nor the
+    allocator's own count (PyTorch's, through which every other buffer here was obtained)."""
+    w = vc_inputs.Workload("m", 1, 2, 2048, 128, (8, 16, 16), (8,), 33, "gauss")
+    q, k, v = [t.cuda() for t in vc_inputs.make_qkv(w)]
+    p = Params.make(w.B, w.H, w.N, w.d, w.grid, bits=8)
+    quant = torch.zeros(vc.vc_quant_bytes(p), dtype=torch.uint8, device="cuda")
+    vc.vc_prep_noalloc(p, q, k, v, None, quant)          # warm call: address lookup, kernel images loaded
+    torch.cuda.synchronize()
+    free0, _ = torch.cuda.mem_get_info()
+    alloc0, reserved0 = torch.cuda.memory_allocated(), torch.cuda.memory_reserved()
+    for _ in range(3):
+        vc.vc_prep_noalloc(p, q, k, v, None, quant)
+    torch.cuda.synchronize()
+    free1, _ = torch.cuda.mem_get_info()
+    assert free1 == free0
+    assert torch.cuda.memory_allocated() == alloc0 and torch.cuda.memory_reserved() == reserved0
+
+
 def test_noalloc_refuses_what_does_not_fit_and_bad_arguments():
     big = Params.make(1, 40, 32760, 128, (21, 30, 52), bits=8)       # needs about 10 MB of scratch
     x = torch.zeros(16, dtype=torch.uint8, device="cuda")
