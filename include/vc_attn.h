@@ -159,6 +159,29 @@ size_t vc_workspace_bytes(const vc_params *p);
 vc_status vc_prep(const vc_params *p, const void *q, const void *k, const void *v,
                   const int32_t *perm, void *quant, void *workspace, void *stream);
 
+/* The statistics of the pass: what makes it read K and V twice.  App. B has the K pass fuse "the
+ * centering statistics" and the V pass "the block mean and scale reductions"; a caller whose
+ * producer of K and V (the projection in front of attention) already has them can hand them in,
+ * and the pass then runs without its statistics launches: K and V are read once.
+ *   k_mean        [B*H][d]      fp32  channel mean over all N tokens of K AFTER RoPE (Sec. 3.4)
+ *   v_block_mean  [B*H][nb][d]  fp32  mean of every 128-token block of the PERMUTED V (Eq. 4; the
+ *                                     ragged last block over its valid tokens; zeros with V smoothing off)
+ *   v_amax        [B*H][d]      fp32  max |V' - block mean| per channel over all tokens, >= 0
+ * All device pointers, 16-byte aligned.  8 bits only (VC_ERR_UNSUPPORTED at 4 bits, where the
+ * outer scales of Q and K are whole-head statistics as well).  The bundle is the one vc_prep
+ * writes when the statistics are the ones it would have computed; v_amax may be any upper
+ * bound of the true maximum at the price of coarser value codes. */
+typedef struct {
+  const float *k_mean, *v_block_mean, *v_amax;
+} vc_prep_stats;
+vc_status vc_prep_with_stats(const vc_params *p, const void *q, const void *k, const void *v,
+                             const int32_t *perm, const vc_prep_stats *stats, void *quant,
+                             void *workspace, void *stream);
+/* Where the last vc_prep call with this bundle and workspace left its own statistics (8 bits);
+ * valid until the workspace is used again. */
+vc_status vc_prep_stats_view(const vc_params *p, const void *quant, const void *workspace,
+                             vc_prep_stats *out);
+
 /* Quantized attention forward (Eq. 1, Eq. 6, Eq. 7) from a bundle in vc_prep's layout.
  * o: [B][H][N][d] bf16.  workspace as above.  `p` must describe the bundle: the same shape,
  * bits, p_format (it selects the value format at 4 bits) and flags as the vc_prep call that
@@ -265,6 +288,18 @@ vc_status vc_poll_status(void *workspace, void *stream);
  * the kernels then record VC_ERR_TIMEOUT, drain their own copies in flight, free their tensor
  * memory and return; outputs of such a call are invalid.  Process-wide; not for production. */
 void vc_test_set_wait_limit(uint32_t polls);
+
+/* Measurement aid (Sec. 3.1 "The softmax bottleneck" compares the softmax stage with the time of
+ * the two matrix products): the rate at which this GPU executes the products' MMAs with
+ * everything else taken away.  Every SM issues `groups` back-to-back 128 x 128 x 128 products of
+ * one kind on tiles resident in shared memory, accumulators in tensor memory:
+ *   kind 8   tcgen05.mma kind::f8f6f4, E4M3 x E4M3               (the 8-bit products)
+ *   kind 4   tcgen05.mma kind::mxf4nvf4.block_scale.block16      (the NVFP4 products)
+ * scratch: 8 bytes of device memory, 8-byte aligned.  tflops (host): 2 x MACs of all SMs / the
+ * launch's CUDA-event time; mac_per_clk_sm (host): MACs of one SM / its own cycle count.
+ * Synchronizes `stream`.  VC_ERR_TIMEOUT if the bounded wait for the MMAs gave up. */
+vc_status vc_mma_peak(int32_t kind, int32_t groups, void *scratch, double *tflops, double *mac_per_clk_sm,
+                      void *stream);
 
 /* Number of kernels this library has launched in this process (diagnostics). */
 uint64_t vc_launch_count(void);

@@ -57,6 +57,11 @@ class QuantView(ctypes.Structure):
                                                            "v_micro")])
 
 
+class PrepStats(ctypes.Structure):
+    """Mirror of vc_prep_stats (device pointers)."""
+    _fields_ = [("k_mean", ctypes.c_void_p), ("v_block_mean", ctypes.c_void_p), ("v_amax", ctypes.c_void_p)]
+
+
 _lib = None
 
 
@@ -75,6 +80,10 @@ def load_library():
     lib.vc_workspace_bytes.argtypes = [P]
     lib.vc_prep.restype = ctypes.c_int
     lib.vc_prep.argtypes = [P, vp, vp, vp, i32p, vp, vp, vp]
+    lib.vc_prep_with_stats.restype = ctypes.c_int
+    lib.vc_prep_with_stats.argtypes = [P, vp, vp, vp, i32p, ctypes.POINTER(PrepStats), vp, vp, vp]
+    lib.vc_prep_stats_view.restype = ctypes.c_int
+    lib.vc_prep_stats_view.argtypes = [P, vp, vp, ctypes.POINTER(PrepStats)]
     lib.vc_prep_noalloc.restype = ctypes.c_int
     lib.vc_prep_noalloc.argtypes = [P, vp, vp, vp, i32p, vp, vp]
     lib.vc_attn_fwd.restype = ctypes.c_int
@@ -95,6 +104,9 @@ def load_library():
     lib.vc_poll_status.argtypes = [vp, vp]
     lib.vc_test_set_wait_limit.restype = None
     lib.vc_test_set_wait_limit.argtypes = [ctypes.c_uint32]
+    lib.vc_mma_peak.restype = ctypes.c_int
+    lib.vc_mma_peak.argtypes = [ctypes.c_int32, ctypes.c_int32, vp, ctypes.POINTER(ctypes.c_double),
+                                ctypes.POINTER(ctypes.c_double), vp]
     lib.vc_launch_count.restype = ctypes.c_uint64
     lib.vc_launch_count.argtypes = []
     lib.vc_status_string.restype = ctypes.c_char_p
@@ -136,6 +148,25 @@ def vc_workspace_bytes(p):
 def vc_prep(p, q, k, v, perm, quant, workspace):
     _check(load_library().vc_prep(ctypes.byref(p), _ptr(q), _ptr(k), _ptr(v), _ptr(perm), _ptr(quant),
                                   _ptr(workspace), _stream()), "vc_prep")
+
+
+def vc_prep_with_stats(p, q, k, v, perm, k_mean, v_block_mean, v_amax, quant, workspace):
+    """vc_prep with the statistics supplied by the caller (fp32 device tensors): no statistics launches."""
+    st = PrepStats(_ptr(k_mean), _ptr(v_block_mean), _ptr(v_amax))
+    _check(load_library().vc_prep_with_stats(ctypes.byref(p), _ptr(q), _ptr(k), _ptr(v), _ptr(perm), ctypes.byref(st),
+                                             _ptr(quant), _ptr(workspace), _stream()), "vc_prep_with_stats")
+
+
+def vc_prep_stats_view(p, quant, workspace):
+    """(k_mean [BH, d], v_block_mean [BH, nb, d], v_amax [BH, d]) fp32 tensors aliasing where vc_prep left them."""
+    st = PrepStats()
+    _check(load_library().vc_prep_stats_view(ctypes.byref(p), _ptr(quant), _ptr(workspace), ctypes.byref(st)), "vc_prep_stats_view")
+    BH, d, nb = p.B * p.H, p.d, (p.N + 127) // 128
+    def alias(ptr, base, n):
+        off = ptr - base.data_ptr()
+        return base[off:off + 4 * n].view(torch.float32)
+    return (alias(st.k_mean, quant, BH * d).view(BH, d), alias(st.v_block_mean, workspace, BH * nb * d).view(BH, nb, d),
+            alias(st.v_amax, workspace, BH * d).view(BH, d))
 
 
 def vc_prep_noalloc(p, q, k, v, perm, quant):
@@ -192,6 +223,15 @@ def vc_poll_status(workspace):
 def vc_test_set_wait_limit(polls):
     """Test hook: polls after which a device-side wait gives up (0 = the default)."""
     load_library().vc_test_set_wait_limit(int(polls))
+
+
+def vc_mma_peak(kind, groups=4096):
+    """(TFLOP/s over the whole GPU, MAC per clock per SM) of back-to-back MMAs of one kind (8 or 4)."""
+    scratch = torch.zeros(1, dtype=torch.int64, device="cuda")
+    tf, mac = ctypes.c_double(0.0), ctypes.c_double(0.0)
+    _check(load_library().vc_mma_peak(int(kind), int(groups), _ptr(scratch), ctypes.byref(tf), ctypes.byref(mac), _stream()),
+           "vc_mma_peak")
+    return tf.value, mac.value
 
 
 def vc_launch_count():

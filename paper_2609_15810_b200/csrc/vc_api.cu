@@ -151,8 +151,8 @@ size_t vc_workspace_bytes(const vc_params* p) {
   return work_layout(pr).total;
 }
 
-vc_status vc_prep(const vc_params* p, const void* q, const void* k, const void* v,
-                  const int32_t* perm, void* quant, void* workspace, void* stream) {
+static vc_status prep_impl(const vc_params* p, const void* q, const void* k, const void* v, const int32_t* perm,
+                           const vc_prep_stats* stats, void* quant, void* workspace, void* stream) {
   Problem pr;
   vc_status st = resolve(p, &pr);
   if (st != VC_OK) return st;
@@ -162,9 +162,39 @@ vc_status vc_prep(const vc_params* p, const void* q, const void* k, const void* 
     return VC_ERR_INVALID_ARG;
   QuantLayout ql = quant_layout(pr);
   WorkLayout wl = work_layout(pr);
+  if (stats) {
+    if (pr.bits != 8) return VC_ERR_UNSUPPORTED;   // at 4 bits the outer scales of Q and K are statistics too
+    if (!stats->k_mean || !stats->v_block_mean || !stats->v_amax) return VC_ERR_INVALID_ARG;
+    if (misaligned(stats->k_mean) || misaligned(stats->v_block_mean) || misaligned(stats->v_amax)) return VC_ERR_INVALID_ARG;
+  }
   cudaError_t e = launch_prep(pr, ql, wl, q, k, v, perm, (uint8_t*)quant, (uint8_t*)workspace,
-                              (cudaStream_t)stream);
+                              (cudaStream_t)stream, stats);
   return e == cudaSuccess ? VC_OK : VC_ERR_CUDA;
+}
+
+vc_status vc_prep(const vc_params* p, const void* q, const void* k, const void* v,
+                  const int32_t* perm, void* quant, void* workspace, void* stream) {
+  return prep_impl(p, q, k, v, perm, nullptr, quant, workspace, stream);
+}
+
+vc_status vc_prep_with_stats(const vc_params* p, const void* q, const void* k, const void* v, const int32_t* perm,
+                             const vc_prep_stats* stats, void* quant, void* workspace, void* stream) {
+  if (!stats) return VC_ERR_INVALID_ARG;
+  return prep_impl(p, q, k, v, perm, stats, quant, workspace, stream);
+}
+
+vc_status vc_prep_stats_view(const vc_params* p, const void* quant, const void* workspace, vc_prep_stats* out) {
+  Problem pr;
+  vc_status st = resolve(p, &pr);
+  if (st != VC_OK) return st;
+  if (!quant || !workspace || !out) return VC_ERR_INVALID_ARG;
+  if (pr.bits != 8) return VC_ERR_UNSUPPORTED;
+  const QuantLayout ql = quant_layout(pr);
+  const WorkLayout wl = work_layout(pr);
+  out->k_mean = (const float*)((const uint8_t*)quant + ql.k_mean);
+  out->v_block_mean = (const float*)((const uint8_t*)workspace + wl.v_mu);
+  out->v_amax = (const float*)((const uint8_t*)workspace + wl.amax);
+  return VC_OK;
 }
 
 static vc_status attn_fwd_impl(const vc_params* p, const void* quant, void* o, void* workspace, void* stream, bool clear_status) {

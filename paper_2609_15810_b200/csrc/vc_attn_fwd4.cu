@@ -318,6 +318,7 @@ attn4_fwd_2q_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     const int p_xor = (row >> 1) & 3;
     uint32_t* sfp_row = reinterpret_cast<uint32_t*>(sSfp + t * kSfpBytes + (row & 31) * 16 + (row >> 5) * 4);
     const float cs = (a.q_g[bh] * a.k_g[bh]) * a.sl;       // code units -> log2 domain
+    const uint64_t k128x2 = pack_f32x2(128.0f, 128.0f), kMagicx2 = pack_f32x2(12582912.0f, 12582912.0f);
     float m_run = -INFINITY;
     for (int j = 0; j < nb; ++j) {
       const int ph = j & 1;
@@ -368,10 +369,10 @@ attn4_fwd_2q_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         if (j > 0 && !warp_wait2(&sh->o_done[t], (j - 1) & 1, sh, a.status, 31)) break;
         const float fa = cs * 0.0625f, fb = (a.code_off - 8.0f * m_new) * 0.0078125f;
         auto code4 = [&](const uint32_t (&sv)[32], int w) -> uint32_t {
-          const uint32_t r0 = __float_as_uint(fmaf(fma_sat(__uint_as_float(sv[4 * w]), fa, fb), 128.0f, 12582912.0f));
-          const uint32_t r1 = __float_as_uint(fmaf(fma_sat(__uint_as_float(sv[4 * w + 1]), fa, fb), 128.0f, 12582912.0f));
-          const uint32_t r2 = __float_as_uint(fmaf(fma_sat(__uint_as_float(sv[4 * w + 2]), fa, fb), 128.0f, 12582912.0f));
-          const uint32_t r3 = __float_as_uint(fmaf(fma_sat(__uint_as_float(sv[4 * w + 3]), fa, fb), 128.0f, 12582912.0f));
+          // (the second FMA runs two scores per instruction: the same fp32 operation per score)
+          uint32_t r0, r1, r2, r3;
+          fma_f32x2_bits(r0, r1, fma_sat(__uint_as_float(sv[4 * w]), fa, fb), fma_sat(__uint_as_float(sv[4 * w + 1]), fa, fb), k128x2, kMagicx2);
+          fma_f32x2_bits(r2, r3, fma_sat(__uint_as_float(sv[4 * w + 2]), fa, fb), fma_sat(__uint_as_float(sv[4 * w + 3]), fa, fb), k128x2, kMagicx2);
           return __byte_perm(__byte_perm(r0, r1, 0x0040), __byte_perm(r2, r3, 0x0040), 0x5410);
         };
         auto store16 = [&](const uint32_t (&sv)[32], int half, int chunk) {   // keys 16 chunk .. +15

@@ -63,7 +63,7 @@ WorkLayout work_layout(const Problem& pr);
 // Launchers (each returns the CUDA error of its launches; all asynchronous on `stream`).
 cudaError_t launch_prep(const Problem& pr, const QuantLayout& ql, const WorkLayout& wl,
                         const void* q, const void* k, const void* v, const int32_t* perm,
-                        uint8_t* quant, uint8_t* work, cudaStream_t stream);
+                        uint8_t* quant, uint8_t* work, cudaStream_t stream, const vc_prep_stats* stats);
 // clear_status: start with a zeroed status word (false inside vc_attn, where the word may already
 // hold what the preprocessing pass recorded)
 cudaError_t launch_attn_fwd(const Problem& pr, const QuantLayout& ql, const WorkLayout& wl,

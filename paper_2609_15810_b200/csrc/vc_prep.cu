@@ -691,12 +691,16 @@ __global__ void __launch_bounds__(kThreads, 2) prep_v_kernel(const PrepArgs a, i
 template <int D, int BITS>
 __global__ void prep_finalize_kernel(const PrepArgs a, int which) {
   const int bh = a.bh0 + blockIdx.x, c = threadIdx.x;
-  if (which == 0) {
+  if (which == 0 || which == 2) {
     if (c < D) {
-      double s = 0.0;
-      if (a.flags & VC_FLAG_K_SMOOTH)
-        for (int j = 0; j < a.nb; ++j) s += (double)a.k_part[((size_t)bh * a.nb + j) * D + c];
-      a.k_mean[(size_t)bh * D + c] = (float)(s / (double)a.N);
+      if (which == 2) {        // statistics from the caller: the mean as given (zero if K smoothing is off)
+        a.k_mean[(size_t)bh * D + c] = (a.flags & VC_FLAG_K_SMOOTH) ? a.ext_k_mean[(size_t)bh * D + c] : 0.f;
+      } else {
+        double s = 0.0;
+        if (a.flags & VC_FLAG_K_SMOOTH)
+          for (int j = 0; j < a.nb; ++j) s += (double)a.k_part[((size_t)bh * a.nb + j) * D + c];
+        a.k_mean[(size_t)bh * D + c] = (float)(s / (double)a.N);
+      }
       float vs = 1.0f;
       if (BITS == 8) {
         const float am = __uint_as_float(a.v_amax[(size_t)bh * D + c]);
@@ -834,14 +838,15 @@ cudaError_t run(const Problem& pr, PrepArgs a, const WorkLayout& wl, uint8_t* wo
     const int nh = pr.BH - bh0 < group ? pr.BH - bh0 : group;
     const int per = pr.nb * nh;
     a.bh0 = bh0;
-    if (a.flags & VC_FLAG_K_SMOOTH) {
+    const bool ext = a.ext_k_mean != nullptr;     // the caller supplied the statistics: no statistics launches
+    if ((a.flags & VC_FLAG_K_SMOOTH) && !ext) {
       prep_kcolsum_kernel<D><<<persistent_grid(per), kThreads, colsum_smem, s>>>(a, per, nh);
       count_launches(1);
     }
-    if (BITS == 8) prep_v_kernel<D, kVStats><<<persistent_grid(per), kThreads, v_smem, s>>>(a, per, nh);
+    if (BITS == 8 && !ext) { prep_v_kernel<D, kVStats><<<persistent_grid(per), kThreads, v_smem, s>>>(a, per, nh); count_launches(1); }
     if (BITS == 4) { prep_qk_kernel<D, kStageAmax, kTpr><<<persistent_grid(per), kRowThreads * kTpr, row_smem, s>>>(a, per, nh, 0); count_launches(1); }
-    prep_finalize_kernel<D, BITS><<<nh, D, 0, s>>>(a, 0);
-    count_launches(BITS == 8 ? 2 : 1);
+    prep_finalize_kernel<D, BITS><<<nh, D, 0, s>>>(a, ext ? 2 : 0);
+    count_launches(1);
     if (BITS == 4) {
       prep_qk_kernel<D, kStageAmax, kTpr><<<persistent_grid(per), kRowThreads * kTpr, row_smem, s>>>(a, per, nh, 1);
       prep_finalize_kernel<D, BITS><<<nh, 32, 0, s>>>(a, 1);
@@ -864,7 +869,7 @@ cudaError_t run(const Problem& pr, PrepArgs a, const WorkLayout& wl, uint8_t* wo
 
 cudaError_t launch_prep(const Problem& pr, const QuantLayout& ql, const WorkLayout& wl,
                         const void* q, const void* k, const void* v, const int32_t* perm,
-                        uint8_t* quant, uint8_t* work, cudaStream_t stream) {
+                        uint8_t* quant, uint8_t* work, cudaStream_t stream, const vc_prep_stats* stats) {
   PrepArgs a{};
   a.q = (const __nv_bfloat16*)q; a.k = (const __nv_bfloat16*)k; a.v = (const __nv_bfloat16*)v;
   a.perm = perm;
@@ -879,6 +884,12 @@ cudaError_t launch_prep(const Problem& pr, const QuantLayout& ql, const WorkLayo
   a.k_part = (float*)(work + wl.k_part); a.v_mu = (float*)(work + wl.v_mu);
   a.v_amax = (unsigned int*)(work + wl.amax);
   a.qk_amax = a.v_amax + (size_t)pr.BH * pr.d;
+  const bool ext = stats != nullptr;
+  if (ext) {   // K mean, V block means and residual maxima as the caller computed them
+    a.ext_k_mean = stats->k_mean;
+    a.v_mu = const_cast<float*>(stats->v_block_mean);
+    a.v_amax = reinterpret_cast<unsigned int*>(const_cast<float*>(stats->v_amax));
+  }
   const int len[3] = {pr.grid_t, pr.grid_h, pr.grid_w};
   int ps = 0;
   for (int ax = 0; ax < 3; ++ax) {
@@ -899,7 +910,7 @@ cudaError_t launch_prep(const Problem& pr, const QuantLayout& ql, const WorkLayo
   }
   cudaError_t e;
   if ((e = cudaMemsetAsync(work + wl.status, 0, 4, stream)) != cudaSuccess) return e;
-  if ((e = cudaMemsetAsync(work + wl.amax, 0, wl.amax_bytes, stream)) != cudaSuccess) return e;
+  if (!ext && (e = cudaMemsetAsync(work + wl.amax, 0, wl.amax_bytes, stream)) != cudaSuccess) return e;
   if (a.flags & VC_FLAG_ROPE) {
     rope_table_kernel<<<(a.rd.entries + 255) / 256, 256, 0, stream>>>(
         reinterpret_cast<float2*>(work + wl.rope), a.rd, (double)pr.rope_theta);
@@ -959,6 +970,6 @@ extern "C" vc_status vc_prep_noalloc(const vc_params* p, const void* q, const vo
   unsigned char* scratch = nullptr;
   if (scratch_address(&scratch) != cudaSuccess) return VC_ERR_CUDA;
   // launch_prep clears the words that must start at zero (status, amax) on the stream itself
-  cudaError_t e = vc::launch_prep(pr, ql, wl, q, k, v, perm, (uint8_t*)quant, scratch, (cudaStream_t)stream);
+  cudaError_t e = vc::launch_prep(pr, ql, wl, q, k, v, perm, (uint8_t*)quant, scratch, (cudaStream_t)stream, nullptr);
   return e == cudaSuccess ? VC_OK : VC_ERR_CUDA;
 }

@@ -33,6 +33,7 @@ struct PrepArgs {
   const float2* rope;
   float *k_part, *v_mu;
   unsigned int *v_amax, *qk_amax;   // qk_amax: [2][BH]
+  const float* ext_k_mean;          // caller-supplied statistics (vc_prep_with_stats), else null
   int BH;
   RopeDesc rd;
 };

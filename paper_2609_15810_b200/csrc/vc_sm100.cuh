@@ -183,6 +183,19 @@ __device__ __forceinline__ float fma_sat(float a, float b, float c) {
   asm("fma.rn.sat.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
   return d;
 }
+// Two FP32 lanes in one 64-bit register, and one fused multiply-add on both (fma.rn.f32x2): the
+// same IEEE operation per lane as fma.rn.f32, one issue slot for two results.
+__device__ __forceinline__ uint64_t pack_f32x2(float lo, float hi) {
+  uint64_t d;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(d) : "f"(lo), "f"(hi));
+  return d;
+}
+__device__ __forceinline__ void fma_f32x2_bits(uint32_t& d_lo, uint32_t& d_hi, float a_lo, float a_hi, uint64_t b, uint64_t c) {
+  uint64_t a, d;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(a) : "f"(a_lo), "f"(a_hi));
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  asm("mov.b64 {%0, %1}, %2;" : "=r"(d_lo), "=r"(d_hi) : "l"(d));
+}
 __device__ __forceinline__ float ex2_approx(float x) {
   float d;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(d) : "f"(x));

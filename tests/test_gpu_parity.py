@@ -210,6 +210,46 @@ def test_hybrid_4bit_arrangement(case, perm_kind):
             Hh.check_output(o[b, h].float().cpu().numpy(), ref, vmax)
 
 
+@pytest.mark.parametrize("perm_kind", ["identity", "random"])
+def test_prep_with_supplied_statistics(perm_kind):
+    """App. B: the statistics (K channel mean, V block means, residual maxima) can come from the
+    producer of K and V; the pass then reads K and V once.  Fed the statistics vc_prep itself
+    computed, the bundle is the same byte for byte; fed the ORACLE's, it matches the oracle's
+    bundle within the usual tolerance."""
+    B, H, N, d, grid = 2, 2, 300, 128, (3, 10, 10)
+    q, k, v = _inputs(B, H, N, d, grid, seed=71)
+    perm = None if perm_kind == "identity" else vc_inputs.random_perm(B, H, N, 13).cuda()
+    p = Params.make(B, H, N, d, grid, bits=8)
+    quant, work = Hh.run_prep(p, q, k, v, perm)
+    km, vmu, vam = [t.clone() for t in vc.vc_prep_stats_view(p, quant, work)]
+    quant2, work2 = alloc_buffers(p)
+    quant2.zero_()
+    n0 = vc.vc_launch_count()
+    vc.vc_prep_with_stats(p, q, k, v, perm, km, vmu, vam, quant2, work2)
+    torch.cuda.synchronize()
+    n1 = vc.vc_launch_count()
+    vc.vc_prep(p, q, k, v, perm, quant, work)
+    assert n1 - n0 == (vc.vc_launch_count() - n1) - 2          # the two statistics launches are gone
+    assert torch.equal(quant2, quant)
+    # the oracle's statistics
+    refs = [Hh.oracle_prep(p, q, k, v, perm, b, h)[0] for b in range(B) for h in range(H)]
+    f32 = lambda a: torch.from_numpy(np.ascontiguousarray(a, dtype=np.float32)).cuda()
+    km_o = f32(np.stack([r["k_mean"] for r in refs]))
+    vmu_o = f32(np.stack([r["v_mu"] for r in refs]))
+    vam_o = f32(np.stack([np.abs(r["v_pre"]).max(axis=0) for r in refs]))
+    quant2.zero_()
+    vc.vc_prep_with_stats(p, q, k, v, perm, km_o, vmu_o, vam_o, quant2, work2)
+    torch.cuda.synchronize()
+    got = Hh.gpu_sections(p, quant2)
+    for i, ref in enumerate(refs):
+        Hh.check_prep_head(p, got, i, ref, what=f"supplied statistics head {i}")
+    p4 = Params.make(B, H, N, d, grid, bits=4)
+    q4, w4 = alloc_buffers(p4)
+    with pytest.raises(vc.VcError) as e:
+        vc.vc_prep_with_stats(p4, q, k, v, perm, km, vmu, vam, q4, w4)
+    assert e.value.code == vc.VC_ERR_UNSUPPORTED
+
+
 def test_bad_arguments_are_rejected_on_the_host():
     p = Params.make(1, 1, 128, 128, (2, 8, 8))
     quant, work = alloc_buffers(p)

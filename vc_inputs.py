@@ -84,28 +84,52 @@ def make_head(w, tensor, b, h, call=0, device="cpu"):
            the offsets are not), same K offsets and V block shifts.
     outliers: each channel of Q and, drawn separately, of K is an outlier channel with
            probability 0.01 (at least one per head); there every token gets + 10 * t_3.
+    A list of calls returns the list of their tensors (the structure is drawn once).
     """
     tid = {"q": 0, "k": 1, "v": 2}[tensor]
+    calls = list(call) if isinstance(call, (list, tuple)) else [call]
     g_struct = _gen(device, w.seed, tid, b, h, 0)           # structure: same on every call
-    g_noise = _gen(device, w.seed, tid, b, h, 1, call)      # noise: redrawn per call
-    if w.kind == "gauss":
-        x = torch.randn(w.N, w.d, generator=g_noise, device=device)
-    else:
-        x = _field(w, g_struct, device) + 0.5 * torch.randn(w.N, w.d, generator=g_noise, device=device)
-    if tensor == "k":
-        x = x + 3.0 * torch.randn(1, w.d, generator=g_struct, device=device)
+    field = None if w.kind == "gauss" else _field(w, g_struct, device)
+    offset = 3.0 * torch.randn(1, w.d, generator=g_struct, device=device) if tensor == "k" else None
+    shift = None
     if tensor == "v":
         nb = (w.N + 127) // 128
-        shift = torch.randn(nb, w.d, generator=g_struct, device=device)
-        x = x + shift.repeat_interleave(128, dim=0)[: w.N]
+        shift = torch.randn(nb, w.d, generator=g_struct, device=device).repeat_interleave(128, dim=0)[: w.N]
+    mask = None
     if w.outliers and tensor in ("q", "k"):
         mask = torch.rand(w.d, generator=g_struct, device=device) < 0.01
         if not bool(mask.any()):
             mask[int(torch.randint(0, w.d, (1,), generator=g_struct, device=device))] = True
-        z = torch.randn(w.N, w.d, generator=g_noise, device=device)
-        chi = torch.randn(3, w.N, w.d, generator=g_noise, device=device).pow(2).sum(0) / 3.0
-        x = x + mask[None, :].float() * 10.0 * z / chi.sqrt()
-    return x.to(torch.bfloat16)
+    out = []
+    for c in calls:
+        g_noise = _gen(device, w.seed, tid, b, h, 1, c)     # noise: redrawn per call
+        x = torch.randn(w.N, w.d, generator=g_noise, device=device)
+        if field is not None:
+            x = field + 0.5 * x
+        if offset is not None:
+            x = x + offset
+        if shift is not None:
+            x = x + shift
+        if mask is not None:
+            z = torch.randn(w.N, w.d, generator=g_noise, device=device)
+            chi = torch.randn(3, w.N, w.d, generator=g_noise, device=device).pow(2).sum(0) / 3.0
+            x = x + mask[None, :].float() * 10.0 * z / chi.sqrt()
+        out.append(x.to(torch.bfloat16))
+    return out if isinstance(call, (list, tuple)) else out[0]
+
+
+def make_qkv_calls(w, n_calls, device="cpu"):
+    """[(Q, K, V)] for calls 0 .. n_calls-1 of the workload: what make_qkv(w, call) gives for each
+    call, with the per-head structure (field, offsets, shifts, outlier channels: the same on every
+    call) synthesised once instead of once per call."""
+    out = [[torch.empty(w.B, w.H, w.N, w.d, dtype=torch.bfloat16, device=device) for _ in range(3)] for _ in range(n_calls)]
+    for ti, tensor in enumerate(("q", "k", "v")):
+        for b in range(w.B):
+            for h in range(w.H):
+                heads = make_head(w, tensor, b, h, list(range(n_calls)), device)
+                for c in range(n_calls):
+                    out[c][ti][b, h] = heads[c]
+    return out
 
 
 def make_qkv(w, call=0, device="cpu", heads=None):
