@@ -225,7 +225,13 @@ def prep_v(v, perm, cfg):
               / n_valid[:, None]).astype(np.float32)              # mu_j  (Eq. 4)
     else:
         mu = np.zeros((nb, d), dtype=np.float32)
-    r = (x.astype(np.float64) - np.repeat(mu.astype(np.float64), BLOCK, axis=0)).astype(np.float32)
+    # Eq. 6 restores exactly what Eq. 4 subtracted only if the two means are the same number.  At 4
+    # bits the mean is stored as bf16 and added back unscaled (App. B), so the mean that is
+    # subtracted is that bf16 value.  (At 8 bits the stored mean is bf16(mu / s_V), restored as
+    # s_V times that: it differs from mu by at most 2^-9 |mu|, a constant offset per block that the
+    # probabilities, which sum to one, pass straight to the output; pinned in the tests.)
+    mu_sub = C.bf16_round(mu) if cfg.bits == 4 else mu
+    r = (x.astype(np.float64) - np.repeat(mu_sub.astype(np.float64), BLOCK, axis=0)).astype(np.float32)
     r = np.where(valid[:, None], r, np.float32(0.0))              # R_j  (Eq. 4)
     out = {"v_pre": r, "v_mu": mu}
     if cfg.bits == 8:

@@ -417,6 +417,12 @@ __device__ __forceinline__ void v_item(const PrepArgs& a, const unsigned char* s
       for (int g = 0; g < TG; ++g) { s0 += red[g * D + 2 * cp]; s1 += red[g * D + 2 * cp + 1]; }
       mu0 = s0 / (float)n_valid;
       mu1 = s1 / (float)n_valid;
+      if constexpr (kFusedMean) {
+        // at 4 bits the mean is stored as bf16 and added back unscaled (App. B): subtract exactly
+        // that number, so that Eq. 6 restores what Eq. 4 removed
+        mu0 = __bfloat162float(__float2bfloat16_rn(mu0));
+        mu1 = __bfloat162float(__float2bfloat16_rn(mu1));
+      }
       __syncthreads();
     }
   }

@@ -167,6 +167,30 @@ def test_mean_restoration_with_quantized_p_is_exact():
     assert np.linalg.norm(o_off - ref, axis=1).max() <= (0.0364 + 0.01) * diam
 
 
+def test_size_of_the_8bit_mean_rounding_offset():
+    """At 8 bits the block mean is stored as bf16(mu / s_V) and restored as s_V times that (App. B),
+    so what Eq. 6 adds back differs from what Eq. 4 subtracted by at most one bf16 rounding of the
+    mean: |s_V bf16(mu / s_V) - mu| <= 2^-8 |mu| (half an ulp of an 8-bit significand, plus the
+    fp32 roundings).  Because the probabilities of a row sum to one, that offset reaches the output
+    unchanged: with every other quantizer switched off, the output with stored means differs from
+    the output with exact means by no more than the largest offset."""
+    N, d = 384, 32
+    q, k, v = _tiny(N=N, d=d, grid=(6, 8, 8), seed=4, v_shift=3.0)
+    cfg8 = P.PrepConfig(N=N, d=d, grid=(6, 8, 8), bits=8)
+    b8 = P.prep_v(v, np.arange(N), cfg8)
+    mu = b8["v_mu"].astype(np.float64)
+    restored = b8["v_means"].astype(np.float64) * b8["v_scale"].astype(np.float64)[None, :]
+    off = np.abs(restored - mu)
+    assert np.all(off <= 2.0 ** -8 * np.abs(mu) * (1 + 1e-3) + 1e-12) and off.max() > 0
+    exact = P.prep_v(v, np.arange(N), P.PrepConfig(N=N, d=d, grid=(6, 8, 8), bits=0))
+    scale = np.float32(A.LOG2E / np.sqrt(d))
+    qd, kd = q.astype(np.float64), k.astype(np.float64)
+    o_exact = A.recurrence(qd, kd, exact["v_deq"], exact["v_means"], N, scale, A.P_EXPCAST, exact=True)
+    o_stored = A.recurrence(qd, kd, exact["v_deq"], restored, N, scale, A.P_EXPCAST, exact=True)
+    assert np.abs(o_stored - o_exact).max() <= off.max() * (1 + 1e-9)
+    assert np.abs(o_stored - o_exact).max() > 0.1 * off.max()          # and it is that offset, not something smaller
+
+
 def test_running_max_and_alpha_follow_eq1():
     """Trace the recurrence on one row by hand."""
     N, d = 256, 16

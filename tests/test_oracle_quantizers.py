@@ -163,7 +163,7 @@ def _v_case(N=300, d=16, seed=21):
     return v, perm, cfg
 
 
-def _v_residual_by_hand(v, perm, N, d):
+def _v_residual_by_hand(v, perm, N, d, mean_as_stored=False):
     n_pad = 128 * ((N + 127) // 128)
     x = [[0.0] * d for _ in range(n_pad)]
     for t in range(N):
@@ -172,6 +172,8 @@ def _v_residual_by_hand(v, perm, N, d):
     for j in range(n_pad // 128):
         n = min(128, N - 128 * j)
         m = [F(sum(x[128 * j + i][c] for i in range(n)) / n) for c in range(d)]   # Eq. 4, valid rows only
+        if mean_as_stored:        # 4 bits: the bf16 mean that Eq. 6 adds back is the one subtracted
+            m = [F(a) for a in C.bf16_round(np.array(m, dtype=F))]
         mu.append(m)
         for i in range(n):
             for c in range(d):
@@ -220,12 +222,15 @@ def test_prep_v_4bit_by_loops(fmt):
     N, d = 300, 16
     v, perm, cfg = _v_case(N, d)
     out = P.prep_v(v, perm, cfg(4, v_format=fmt))
-    mu, r, n_pad = _v_residual_by_hand(v, perm, N, d)
+    mu, r, n_pad = _v_residual_by_hand(v, perm, N, d, mean_as_stored=True)
     G = 16 if fmt == "nvfp4" else 32
     assert out["v_codes"].shape == (n_pad, d) and out["v_micro"].shape == (n_pad // G, d)
     assert np.all(out["v_scale"] == 1.0)
     for j in range(3):
-        assert np.array_equal(out["v_means"][j], C.bf16_round(np.array(mu[j], dtype=F)))
+        assert np.array_equal(out["v_means"][j], np.array(mu[j], dtype=F))
+    # Eq. 6 at 4 bits: residual plus STORED mean is the gathered value again, exactly
+    assert np.array_equal((out["v_pre"][:N].astype(np.float64) + np.repeat(out["v_means"].astype(np.float64), 128, 0)[:N]).astype(F),
+                          v[perm])
     for c in range(d):
         for g in range(n_pad // G):
             col = [r[G * g + i][c] for i in range(G)]
