@@ -17,7 +17,10 @@ Pins (tests/test_oracle_*.py): the codecs are pinned exhaustively and against an
 independent library cast; Hadamard, K smoothing, permutation, block demeaning and mean
 restoration are pinned by the identities the paper states for them; ExpCast-FP8 by the
 paper's worked example and printed constants; the recurrence by brute-force attention
-with quantization switched off.  The *end-to-end quantized* output has no printed value
+with quantization switched off; every block quantizer (8-bit Q/K blocks, NVFP4 groups under an
+outer scale, the NVFP4 probability format, the quantized branches of the V pass) by Python
+loops and a brute-force nearest-value search on inputs with planted maxima and ties
+(tests/test_oracle_quantizers.py).  The *end-to-end quantized* output has no printed value
 in the paper: "parity unpinned" for the granularity of the Q/K scales, the NVFP4
 second-level scales and the RoPE channel split, which are readings fixed by this build.
 Grouping is pinned by brute-force nearest-centroid search, cluster recovery on separated
