@@ -105,7 +105,7 @@ typedef struct {
   int32_t rope_dim_t, rope_dim_h, rope_dim_w; /* channels per axis, even, sum == d;
                                        all 0 => (d - 4*(d/6), 2*(d/6), 2*(d/6))         */
   float rope_theta;                 /* 0 => 10000                                       */
-  int64_t stride_b, stride_h, stride_n;       /* of Q, K and V, in elements; 0 => packed */
+  int64_t stride_b, stride_h, stride_n;       /* of Q, K and V, in elements; 0 => packed; stride_n < 2^30 */
   int32_t heads_per_pass;           /* heads preprocessed per launch group (L2 reuse of
                                        the second read of K and V); 0 => library default */
   int32_t kernel_variant;           /* attention kernel: 0 = pipelined, two query tiles per
@@ -199,8 +199,9 @@ vc_status vc_attn(const vc_params *p, const void *q, const void *k, const void *
  * stream.  The staging buffers are caller-allocated device memory of the same sizes.
  * Heads are independent, so the call works through groups of heads and overlaps the
  * input copy of the next group and the output copy of the previous one with the kernels of
- * the current one, on two helper streams that it creates and destroys itself (ordered after
- * the work already on `stream`; `stream` is complete when the call returns). */
+ * the current one, on two helper streams of its own (made on the first call on a device and kept;
+ * calls on one device take turns; ordered after the work already on `stream`; `stream` is
+ * complete when the call returns). */
 vc_status vc_attn_host(const vc_params *p, const void *q_host, const void *k_host,
                        const void *v_host, const int32_t *perm_host, void *o_host,
                        void *q_dev, void *k_dev, void *v_dev, int32_t *perm_dev, void *o_dev,

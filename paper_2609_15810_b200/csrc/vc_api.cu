@@ -1,5 +1,6 @@
 // C-ABI entry points of libvc: argument validation, buffer layouts, launch sequencing.
 #include <atomic>
+#include <mutex>
 #include <vector>
 #include <cstring>
 
@@ -61,6 +62,7 @@ vc_status resolve(const vc_params* p, Problem* out) {
   pr.stride_n = p->stride_n ? p->stride_n : pr.d;
   pr.stride_h = p->stride_h ? p->stride_h : (int64_t)pr.N * pr.d;
   pr.stride_b = p->stride_b ? p->stride_b : (int64_t)pr.H * pr.N * pr.d;
+  if (pr.stride_n >= (1ll << 30)) return VC_ERR_UNSUPPORTED;     // a row stride in bytes fits 32 bits
   if (pr.stride_n < pr.d || (pr.stride_n % 8) || (pr.stride_h % 8) || (pr.stride_b % 8))
     return VC_ERR_INVALID_ARG;   // rows are read with 16-byte vector loads
   pr.n_pad = kBlock * ((pr.N + kBlock - 1) / kBlock);
@@ -132,6 +134,15 @@ WorkLayout work_layout(const Problem& pr) {
 }
 
 static bool misaligned(const void* p) { return ((uintptr_t)p & 15) != 0; }
+
+// Helper streams and events of vc_attn_host, one set per device.
+constexpr int kMaxHostPipes = 64;
+struct HostPipe {
+  std::mutex mu;
+  cudaStream_t s_in = nullptr, s_out = nullptr;
+  std::vector<cudaEvent_t> ev;
+};
+static HostPipe g_host_pipes[kMaxHostPipes];
 
 }  // namespace vc
 
@@ -266,11 +277,23 @@ vc_status vc_attn_host(const vc_params* p, const void* q_host, const void* k_hos
   }
   const int groups = (int)sizes.size();
   const size_t head_elems = (size_t)pr.N * pr.d;
-  cudaStream_t s_in = nullptr, s_out = nullptr;
-  std::vector<cudaEvent_t> ev(2 * groups + 2, nullptr);
-  bool ok = cudaStreamCreateWithFlags(&s_in, cudaStreamNonBlocking) == cudaSuccess &&
-            cudaStreamCreateWithFlags(&s_out, cudaStreamNonBlocking) == cudaSuccess;
-  for (size_t i = 0; ok && i < ev.size(); ++i) ok = cudaEventCreateWithFlags(&ev[i], cudaEventDisableTiming) == cudaSuccess;
+  // The two helper streams and the events are made once per device and kept for the life of the
+  // process (a call used to create and destroy 2 streams and 2 * groups + 2 events); calls on one
+  // device take turns, which costs nothing: a call ends with the stream synchronized anyway.
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxHostPipes) return VC_ERR_CUDA;
+  HostPipe& hp = g_host_pipes[dev];
+  std::lock_guard<std::mutex> lock(hp.mu);
+  bool ok = true;
+  if (!hp.s_in) ok = cudaStreamCreateWithFlags(&hp.s_in, cudaStreamNonBlocking) == cudaSuccess;
+  if (ok && !hp.s_out) ok = cudaStreamCreateWithFlags(&hp.s_out, cudaStreamNonBlocking) == cudaSuccess;
+  while (ok && hp.ev.size() < (size_t)(2 * groups + 2)) {
+    cudaEvent_t e = nullptr;
+    ok = cudaEventCreateWithFlags(&e, cudaEventDisableTiming) == cudaSuccess;
+    if (ok) hp.ev.push_back(e);
+  }
+  cudaStream_t s_in = hp.s_in, s_out = hp.s_out;
+  std::vector<cudaEvent_t>& ev = hp.ev;
   vc_status result = VC_OK;
   if (ok) {
     cudaEvent_t e_begin = ev[2 * groups], e_end = ev[2 * groups + 1];
@@ -304,10 +327,7 @@ vc_status vc_attn_host(const vc_params* p, const void* q_host, const void* k_hos
     if (cudaStreamSynchronize(s_in) != cudaSuccess) ok = false;
     if (cudaStreamSynchronize(s) != cudaSuccess) ok = false;
   }
-  for (cudaEvent_t e : ev)
-    if (e) cudaEventDestroy(e);
-  if (s_in) cudaStreamDestroy(s_in);
-  if (s_out) cudaStreamDestroy(s_out);
+  if (cudaStreamSynchronize(s_out) != cudaSuccess) ok = false;   // the shared helpers are idle when the lock is released
   if (result != VC_OK) return result;
   return ok ? VC_OK : VC_ERR_CUDA;
 }

@@ -57,19 +57,64 @@ template <int D> struct Geo {
 struct Item {
   int z, bh, blk;
 };
-// items are numbered block-fastest, then head, then tensor
-__device__ __forceinline__ Item decode_item(int item, int nb, int nh, int bh0) {
-  Item it;
-  it.blk = item % nb;
+// Items are numbered block-fastest, then head, then tensor.  A CTA visits items blockIdx.x + k *
+// gridDim.x: the position is divided out once and then advanced by the grid stride with carries
+// (the divisions are not free at 64 elements per thread and item).
+struct Cursor {
+  int blk, hh, z;            // block, head within the launch's group, tensor
+};
+struct CursorStep {
+  int dblk, dhh;             // gridDim.x = dhh * nb + dblk
+};
+__device__ __forceinline__ Cursor cursor_at(int item, int nb, int nh) {
+  Cursor c;
+  c.blk = item % nb;
   const int r = item / nb;
-  it.bh = bh0 + r % nh;
-  it.z = r / nh;
+  c.hh = r % nh;
+  c.z = r / nh;
+  return c;
+}
+__device__ __forceinline__ CursorStep cursor_step(int nb) {
+  CursorStep s;
+  s.dhh = (int)gridDim.x / nb;
+  s.dblk = (int)gridDim.x - s.dhh * nb;
+  return s;
+}
+__device__ __forceinline__ void advance(Cursor& c, const CursorStep& s, int nb, int nh) {
+  c.blk += s.dblk;
+  c.hh += s.dhh;
+  if (c.blk >= nb) { c.blk -= nb; ++c.hh; }
+  while (c.hh >= nh) { c.hh -= nh; ++c.z; }      // at most once unless the launch is tiny
+}
+__device__ __forceinline__ Item item_of(const Cursor& c, int bh0) {
+  Item it;
+  it.z = c.z; it.bh = bh0 + c.hh; it.blk = c.blk;
   return it;
+}
+// Start of head bh in an input tensor, in bytes (bh = b * H + h, general strides).
+__device__ __forceinline__ int64_t head_offset_bytes(const PrepArgs& a, int bh) {
+  const int b = (int)div40((unsigned)bh, a.mul_H), h = bh - b * a.H;
+  return 2 * (b * a.stride_b + h * a.stride_h);
 }
 
 // ---------------------------------------------------------------------------------------
 // K column sums after RoPE (the channel mean of Sec. 3.4 is taken after the rotation).  A lane
 // owns 8 consecutive channels of D/16 rows, so a column's partial sums meet by xor-shuffles.
+// A RoPE table entry: from the copy in shared memory (address in the shared window) when there
+// is one, else from global memory.
+struct RopeTab {
+  uint32_t saddr;            // 0: no copy in shared memory
+  const float2* g;
+};
+__device__ __forceinline__ float2 rope_entry_s(uint32_t saddr, int e) {
+  float2 r;
+  asm("ld.shared.v2.f32 {%0, %1}, [%2];" : "=f"(r.x), "=f"(r.y) : "r"(saddr + 8u * (uint32_t)e));
+  return r;
+}
+__device__ __forceinline__ float2 rope_entry(const RopeTab& t, int e) {
+  return t.saddr ? rope_entry_s(t.saddr, e) : __ldg(t.g + e);
+}
+
 struct PairSlots {          // the 4 channel pairs a lane owns: axis and table slot of each
   int axis[4], idx[4], stride[4];
 };
@@ -87,7 +132,7 @@ __device__ __forceinline__ PairSlots pair_slots(const RopeDesc& rd, int first_pa
 }
 
 template <int D>
-__device__ __forceinline__ void k_colsum_item(const PrepArgs& a, const unsigned char* stage, float* red, const float2* tab,
+__device__ __forceinline__ void k_colsum_item(const PrepArgs& a, const unsigned char* stage, float* red, const RopeTab& tab,
                                               const PairSlots& ps, int bh, int blk) {
   constexpr int LPR = D / 8;         // lanes per row
   constexpr int RPL = LPR / 2;       // rows per lane (a warp covers 16 rows)
@@ -117,7 +162,7 @@ __device__ __forceinline__ void k_colsum_item(const PrepArgs& a, const unsigned 
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
         const int pos = ps.axis[j] == 0 ? tt : (ps.axis[j] == 1 ? ty : tx);
-        const float2 cs = tab[ps.idx[j] + pos * ps.stride[j]];
+        const float2 cs = rope_entry(tab, ps.idx[j] + pos * ps.stride[j]);
         const float x0 = x[2 * j], x1 = x[2 * j + 1];
         x[2 * j] = x0 * cs.x - x1 * cs.y;
         x[2 * j + 1] = x0 * cs.y + x1 * cs.x;
@@ -177,7 +222,7 @@ template <int D> __device__ __forceinline__ constexpr int rope_axis_of(int p) {
 
 template <int D, int STAGE, int TPR>
 __device__ __forceinline__ void qk_row_item(const PrepArgs& a, const int TENSOR /*0 = Q, 1 = K*/, const unsigned char* stage,
-                                            unsigned char* out_tile, float* red, float* kmean_s, const float2* tab, int bh,
+                                            unsigned char* out_tile, float* red, float* kmean_s, const RopeTab& tab, int bh,
                                             int blk, int iter, bool new_head, int src_row) {
   constexpr int C = D / TPR;                       // channels per thread
   constexpr int NT = kRowThreads * TPR;
@@ -188,12 +233,10 @@ __device__ __forceinline__ void qk_row_item(const PrepArgs& a, const int TENSOR 
   const bool center = TENSOR == 1 && (a.flags & VC_FLAG_K_SMOOTH);
   const bool valid = src_row >= 0;               // src_row: the input row behind this thread's row
   const int src = valid ? src_row : 0;           // (RoPE acts at the source position)
+  // (a row without a source reads what the stage holds and is zeroed below)
   uint4 raw[C / 8];
 #pragma unroll
-  for (int i = 0; i < C / 8; ++i) {
-    raw[i] = make_uint4(0, 0, 0, 0);
-    if (valid) raw[i] = *reinterpret_cast<const uint4*>(stage + row * Geo<D>::pitch + part * (2 * C) + 16 * i);
-  }
+  for (int i = 0; i < C / 8; ++i) raw[i] = *reinterpret_cast<const uint4*>(stage + row * Geo<D>::pitch + part * (2 * C) + 16 * i);
   if (center && new_head) {
     __syncthreads();                               // everyone is done with the previous head's mean
     for (int c = tid; c < D; c += NT) kmean_s[c] = a.k_mean[(size_t)bh * D + c];
@@ -210,6 +253,10 @@ __device__ __forceinline__ void qk_row_item(const PrepArgs& a, const int TENSOR 
       x[8 * i + 2 * j + 1] = __uint_as_float(w[j] & 0xffff0000u);
     }
   }
+  if (!valid) {
+#pragma unroll
+    for (int c = 0; c < C; ++c) x[c] = 0.f;
+  }
   if (do_rope && valid) {
     int tt, ty, tx;
     grid_pos(a.rd, src, tt, ty, tx);
@@ -218,7 +265,7 @@ __device__ __forceinline__ void qk_row_item(const PrepArgs& a, const int TENSOR 
                       a.rd.off[1] + ty * a.rd.pairs[1] - a.rd.pair_start[1],
                       a.rd.off[2] + tx * a.rd.pairs[2] - a.rd.pair_start[2]};
     const int p0 = part * (C / 2);               // first pair of this thread
-    if (a.rope_default) {
+    if (a.rope_default && tab.saddr) {
       // compile-time pair boundaries: the axis of local pair i is known for either part, so the
       // table base of each (axis in part 0, axis in part 1) combination is selected once per row
       int base[3][3];
@@ -228,7 +275,7 @@ __device__ __forceinline__ void qk_row_item(const PrepArgs& a, const int TENSOR 
         for (int a1 = 0; a1 < 3; ++a1) base[a0][a1] = (part ? e[a1] : e[a0]) + p0;
 #pragma unroll
       for (int i = 0; i < C / 2; ++i) {
-        const float2 cs = tab[base[rope_axis_of<D>(i)][rope_axis_of<D>(TPR == 1 ? i : C / 2 + i)] + i];
+        const float2 cs = rope_entry_s(tab.saddr, base[rope_axis_of<D>(i)][rope_axis_of<D>(TPR == 1 ? i : C / 2 + i)] + i);
         const float x0 = x[2 * i], x1 = x[2 * i + 1];
         x[2 * i] = x0 * cs.x - x1 * cs.y;
         x[2 * i + 1] = x0 * cs.y + x1 * cs.x;
@@ -238,7 +285,7 @@ __device__ __forceinline__ void qk_row_item(const PrepArgs& a, const int TENSOR 
       for (int i = 0; i < C / 2; ++i) {
         const int p = p0 + i;
         const int eb = p < a.rd.pair_start[1] ? e[0] : (p < a.rd.pair_start[2] ? e[1] : e[2]);
-        const float2 cs = tab[eb + p];
+        const float2 cs = rope_entry(tab, eb + p);
         const float x0 = x[2 * i], x1 = x[2 * i + 1];
         x[2 * i] = x0 * cs.x - x1 * cs.y;
         x[2 * i + 1] = x0 * cs.y + x1 * cs.x;
@@ -378,7 +425,8 @@ __device__ __forceinline__ void qk_row_item(const PrepArgs& a, const int TENSOR 
 // block, so block means and the channel-major (token-contiguous) code rows need no transposition.
 enum { kVStats = 0, kVQuant8 = 1, kVQuant4 = 2, kVQuant4M = 3 };   // 4M: E2M1 under power-of-two factors per 32 tokens
 
-template <int D, int STAGE>
+// FULL: all 128 rows of the block exist (every block but a head's ragged last one): no row tests.
+template <int D, int STAGE, bool FULL>
 __device__ __forceinline__ void v_item(const PrepArgs& a, const unsigned char* stage, float* red, int bh, int blk,
                                        float2 mu_in, float2 am_in) {
   constexpr int CP = D / 2;             // channel pairs
@@ -386,12 +434,12 @@ __device__ __forceinline__ void v_item(const PrepArgs& a, const unsigned char* s
   constexpr int TPG = kBlock / TG;      // tokens per thread
   const int tid = threadIdx.x;
   const int cp = tid % CP, tg = tid / CP;
-  const int n_valid = min(kBlock, a.N - blk * kBlock);
+  const int n_valid = FULL ? kBlock : min(kBlock, a.N - blk * kBlock);
   float v0[TPG], v1[TPG];
+  const unsigned char* mine = stage + tg * TPG * (2 * D) + 4 * cp;
 #pragma unroll
   for (int i = 0; i < TPG; ++i) {
-    const int row = tg * TPG + i;
-    const unsigned int w = row < n_valid ? *reinterpret_cast<const unsigned int*>(stage + row * (2 * D) + 4 * cp) : 0u;
+    const unsigned int w = (FULL || tg * TPG + i < n_valid) ? *reinterpret_cast<const unsigned int*>(mine + i * (2 * D)) : 0u;
     v0[i] = __uint_as_float(w << 16);
     v1[i] = __uint_as_float(w & 0xffff0000u);
   }
@@ -431,7 +479,7 @@ __device__ __forceinline__ void v_item(const PrepArgs& a, const unsigned char* s
     float m0 = 0.f, m1 = 0.f;
 #pragma unroll
     for (int i = 0; i < TPG; ++i) {
-      if (tg * TPG + i < n_valid) {
+      if (FULL || tg * TPG + i < n_valid) {
         m0 = fmaxf(m0, fabsf(v0[i] - mu0));
         m1 = fmaxf(m1, fabsf(v1[i] - mu1));
       }
@@ -455,7 +503,7 @@ __device__ __forceinline__ void v_item(const PrepArgs& a, const unsigned char* s
   float r0[TPG], r1[TPG];
 #pragma unroll
   for (int i = 0; i < TPG; ++i) {
-    const bool valid = tg * TPG + i < n_valid;
+    const bool valid = FULL || tg * TPG + i < n_valid;
     r0[i] = valid ? v0[i] - mu0 : 0.f;
     r1[i] = valid ? v1[i] - mu1 : 0.f;
   }
@@ -585,12 +633,12 @@ __device__ __forceinline__ void v_item(const PrepArgs& a, const unsigned char* s
 
 // ---------------------------------------------------------------------------------------
 // RoPE table -> shared memory (when it fits), once per CTA.
-__device__ __forceinline__ const float2* stage_rope_table(const PrepArgs& a, unsigned char* at) {
-  const float2* tab = a.rope;
+__device__ __forceinline__ RopeTab stage_rope_table(const PrepArgs& a, unsigned char* at) {
+  RopeTab tab{0u, a.rope};
   if ((a.flags & VC_FLAG_ROPE) && a.rope_in_smem) {
     float2* tab_s = reinterpret_cast<float2*>(at);
     for (int e = threadIdx.x; e < a.rd.entries; e += blockDim.x) tab_s[e] = __ldg(&a.rope[e]);
-    tab = tab_s;
+    tab.saddr = smem_u32(at);
   }
   __syncthreads();
   return tab;
@@ -603,93 +651,110 @@ __global__ void __launch_bounds__(kThreads, 2) prep_kcolsum_kernel(const PrepArg
   constexpr int LPR = D / 8, RPL = LPR / 2, kStage = kThreads * RPL * 16;
   extern __shared__ __align__(128) unsigned char smem[];
   float* red = reinterpret_cast<float*>(smem + 2 * kStage);
-  const float2* tab = stage_rope_table(a, smem + 2 * kStage + 8 * D * 4);
+  const RopeTab tab = stage_rope_table(a, smem + 2 * kStage + 8 * D * 4);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int lr = lane % LPR, hb = lane / LPR;
   const PairSlots ps = pair_slots(a.rd, 4 * lr);
-  auto issue = [&](int item, int st) {
+  const CursorStep step = cursor_step(a.nb);
+  auto issue = [&](int item, const Cursor& c, int st) {
     if (item < n_items) {
-      const Item w = decode_item(item, a.nb, nh, a.bh0);
-      const int b = w.bh / a.H, h = w.bh - b * a.H;
-      const __nv_bfloat16* base = a.k + b * a.stride_b + h * a.stride_h + 8 * lr;
+      const char* base = reinterpret_cast<const char*>(a.k) + head_offset_bytes(a, a.bh0 + c.hh) + 16 * lr;
+      const int t0 = c.blk * kBlock + 16 * warp + RPL * hb;
+      unsigned char* dst = smem + st * kStage + tid * 16;
 #pragma unroll
-      for (int i = 0; i < RPL; ++i) {
-        const int t = w.blk * kBlock + 16 * warp + RPL * hb + i;
-        if (t < a.N) cp_async16(smem + st * kStage + (i * kThreads + tid) * 16, base + (int64_t)t * a.stride_n);
-      }
+      for (int i = 0; i < RPL; ++i)
+        if (t0 + i < a.N) cp_async16(dst + i * kThreads * 16, base + (int64_t)(t0 + i) * a.stride_n_bytes);
     }
     cp_async_commit();
   };
-  issue(blockIdx.x, 0);
+  Cursor cur = cursor_at(blockIdx.x, a.nb, nh), nxt = cur;
+  advance(nxt, step, a.nb, nh);
+  issue(blockIdx.x, cur, 0);
   int i = 0;
   for (int item = blockIdx.x; item < n_items; item += gridDim.x, ++i) {
-    issue(item + gridDim.x, (i + 1) & 1);
+    issue(item + gridDim.x, nxt, (i + 1) & 1);
     cp_async_wait<1>();                       // this thread's chunks of item i have landed
-    const Item w = decode_item(item, a.nb, nh, a.bh0);
-    k_colsum_item<D>(a, smem + (i & 1) * kStage, red, tab, ps, w.bh, w.blk);
+    k_colsum_item<D>(a, smem + (i & 1) * kStage, red, tab, ps, a.bh0 + cur.hh, cur.blk);
+    cur = nxt;
+    advance(nxt, step, a.nb, nh);
   }
 }
 
 // V pass: STAGE = block means + residual amax (launch 1b) or quantization of the residual.
-// Shared memory: [3 stages x (128 x 2 D)][red: 8 D floats].
+// Shared memory: [3 stages x (128 x 2 D)][red: 8 D floats][source rows: 2 x 128].
 template <int D, int STAGE>
 __global__ void __launch_bounds__(kThreads, 2) prep_v_kernel(const PrepArgs a, int n_items, int nh) {
   constexpr int LPR = D / 8, kStage = kBlock * 2 * D, NL = kBlock * LPR / kThreads;
   extern __shared__ __align__(128) unsigned char smem[];
   float* red = reinterpret_cast<float*>(smem + 3 * kStage);
+  int* src_ring = reinterpret_cast<int*>(red + 8 * D);                 // [2][128]
   const int tid = threadIdx.x;
-  // items i .. i+3 of this CTA, decoded once each (the divisions are not free at 64 elements per thread)
-  Item q0 = decode_item(blockIdx.x, a.nb, nh, a.bh0), q1 = decode_item(blockIdx.x + gridDim.x, a.nb, nh, a.bh0),
-       q2 = decode_item(blockIdx.x + 2 * gridDim.x, a.nb, nh, a.bh0), q3 = decode_item(blockIdx.x + 3 * gridDim.x, a.nb, nh, a.bh0);
-  auto fetch = [&](int item, const Item& w, int (&src)[NL]) {          // source rows of the chunks this thread copies
-#pragma unroll
-    for (int c = 0; c < NL; ++c) src[c] = -1;
-    if (item >= n_items) return;
-    const int32_t* prow = a.perm + (size_t)w.bh * a.N;
-#pragma unroll
-    for (int c = 0; c < NL; ++c) {
-      const int t = w.blk * kBlock + (tid + c * kThreads) / LPR;
-      if (t < a.N) src[c] = a.perm ? min(max(__ldg(prow + t), 0), a.N - 1) : t;   // clamped: never a bad address
-    }
+  const CursorStep step = cursor_step(a.nb);
+  // source row of row `tid` of an item (the gather by pi), -1 if there is none
+  auto fetch = [&](int item, const Cursor& c) -> int {
+    if (item >= n_items || tid >= kBlock) return -1;
+    const int t = c.blk * kBlock + tid;
+    if (t >= a.N) return -1;
+    return a.perm ? min(max(__ldg(a.perm + (size_t)(a.bh0 + c.hh) * a.N + t), 0), a.N - 1) : t;   // clamped: never a bad address
   };
-  auto issue = [&](int item, const Item& w, int st, const int (&src)[NL]) {
+  auto issue = [&](int item, const Cursor& c, int st, const int* src) {
     if (item < n_items) {
-      const int b = w.bh / a.H, h = w.bh - b * a.H;
-      const __nv_bfloat16* base = a.v + b * a.stride_b + h * a.stride_h + 8 * (tid % LPR);
+      const char* base = reinterpret_cast<const char*>(a.v) + head_offset_bytes(a, a.bh0 + c.hh) + 16 * (tid % LPR);
+      unsigned char* dst = smem + st * kStage + tid * 16;
 #pragma unroll
-      for (int c = 0; c < NL; ++c)
-        if (src[c] >= 0) cp_async16(smem + st * kStage + (tid + c * kThreads) * 16, base + (int64_t)src[c] * a.stride_n);
+      for (int k = 0; k < NL; ++k) {
+        const int sr = src[tid / LPR + k * (kThreads / LPR)];
+        if (sr >= 0) cp_async16(dst + k * kThreads * 16, base + (int64_t)sr * a.stride_n_bytes);
+      }
     }
     cp_async_commit();
   };
   // per-item scalars of the quantizing stage, fetched one item ahead
   const int cp = tid % (D / 2);
-  auto fetch_mu = [&](int item, const Item& w) -> float2 {
+  auto fetch_mu = [&](int item, const Cursor& c) -> float2 {
     if (STAGE == kVStats || STAGE == kVQuant4 || STAGE == kVQuant4M || item >= n_items) return make_float2(0.f, 0.f);
-    return *reinterpret_cast<const float2*>(a.v_mu + ((size_t)w.bh * a.nb + w.blk) * D + 2 * cp);
+    return *reinterpret_cast<const float2*>(a.v_mu + ((size_t)(a.bh0 + c.hh) * a.nb + c.blk) * D + 2 * cp);
   };
-  int src[NL];
-  fetch(blockIdx.x, q0, src);
-  issue(blockIdx.x, q0, 0, src);
-  fetch(blockIdx.x + gridDim.x, q1, src);
-  issue(blockIdx.x + gridDim.x, q1, 1, src);
-  fetch(blockIdx.x + 2 * gridDim.x, q2, src);
-  float2 mu = fetch_mu(blockIdx.x, q0), am = make_float2(0.f, 0.f);
-  int i = 0, last_bh = -1;
-  for (int item = blockIdx.x; item < n_items; item += gridDim.x, ++i) {
+  // cursors of items i, i+1, i+2 and i+4 of this CTA
+  const int g = gridDim.x;
+  Cursor c0 = cursor_at(blockIdx.x, a.nb, nh), c1 = c0;
+  advance(c1, step, a.nb, nh);
+  Cursor c2 = c1;
+  advance(c2, step, a.nb, nh);
+  Cursor c4 = c2;
+  advance(c4, step, a.nb, nh);
+  if (tid < kBlock) {
+    src_ring[tid] = fetch(blockIdx.x, c0);
+    src_ring[kBlock + tid] = fetch(blockIdx.x + g, c1);
+  }
+  __syncthreads();
+  issue(blockIdx.x, c0, 0, src_ring);
+  issue(blockIdx.x + g, c1, 1, src_ring + kBlock);
+  __syncthreads();                            // the two slices have been read
+  if (tid < kBlock) src_ring[tid] = fetch(blockIdx.x + 2 * g, c2);
+  int nxt = fetch(blockIdx.x + 3 * g, c4);    // (c4 still stands at item 3 here)
+  advance(c4, step, a.nb, nh);
+  float2 mu = fetch_mu(blockIdx.x, c0), am = make_float2(0.f, 0.f);
+  int i = 0, last_hh = -1;
+  for (int item = blockIdx.x; item < n_items; item += g, ++i) {
     cp_async_wait<1>();                       // my chunks of item i have landed ...
     __syncthreads();                          // ... and everyone's; all are done with item i-1
-    issue(item + 2 * gridDim.x, q2, (i + 2) % 3, src);
-    fetch(item + 3 * gridDim.x, q3, src);
-    const float2 mu_next = fetch_mu(item + gridDim.x, q1);
-    if (STAGE == kVQuant8 && q0.bh != last_bh) {
-      am = make_float2(__uint_as_float(a.v_amax[(size_t)q0.bh * D + 2 * cp]), __uint_as_float(a.v_amax[(size_t)q0.bh * D + 2 * cp + 1]));
-      last_bh = q0.bh;
+    if (tid < kBlock) src_ring[((i + 1) & 1) * kBlock + tid] = nxt;     // source rows of item i+3
+    nxt = fetch(item + 4 * g, c4);
+    issue(item + 2 * g, c2, (i + 2) % 3, src_ring + (i & 1) * kBlock);
+    const float2 mu_next = fetch_mu(item + g, c1);
+    if (STAGE == kVQuant8 && c0.hh != last_hh) {
+      const size_t at = (size_t)(a.bh0 + c0.hh) * D + 2 * cp;
+      am = make_float2(__uint_as_float(a.v_amax[at]), __uint_as_float(a.v_amax[at + 1]));
+      last_hh = c0.hh;
     }
-    v_item<D, STAGE>(a, smem + (i % 3) * kStage, red, q0.bh, q0.blk, mu, am);
+    const unsigned char* stage = smem + (i % 3) * kStage;
+    if (a.N - c0.blk * kBlock >= kBlock) v_item<D, STAGE, true>(a, stage, red, a.bh0 + c0.hh, c0.blk, mu, am);
+    else v_item<D, STAGE, false>(a, stage, red, a.bh0 + c0.hh, c0.blk, mu, am);
     mu = mu_next;
-    q0 = q1; q1 = q2; q2 = q3;
-    q3 = decode_item(item + 4 * gridDim.x, a.nb, nh, a.bh0);
+    c0 = c1; c1 = c2;
+    advance(c2, step, a.nb, nh);
+    advance(c4, step, a.nb, nh);
   }
 }
 
@@ -740,64 +805,69 @@ __global__ void __launch_bounds__(kRowThreads * TPR, 2) prep_qk_kernel(const Pre
   int* src_ring = reinterpret_cast<int*>(out_tile + kBlock * D);     // [3][128]
   float* red = reinterpret_cast<float*>(src_ring + 3 * kBlock);      // [2][8]
   float* kmean_s = red + 16;                                         // [D]
-  const float2* tab = stage_rope_table(a, reinterpret_cast<unsigned char*>(kmean_s + D));
+  const RopeTab tab = stage_rope_table(a, reinterpret_cast<unsigned char*>(kmean_s + D));
   const int tid = threadIdx.x;
   const int my_row = qk_row_of<TPR>(tid);
-  auto fetch = [&](int item) -> int {        // input row behind row `tid` of the item, -1 if none
+  const CursorStep step = cursor_step(a.nb);
+  auto fetch = [&](int item, const Cursor& c) -> int {   // input row behind row `tid` of the item, -1 if none
     if (item >= n_items || tid >= kBlock) return -1;
-    const Item w = decode_item(item, a.nb, nh, a.bh0);
-    const int t = w.blk * kBlock + tid;
+    const int t = c.blk * kBlock + tid;
     if (t >= a.N) return -1;
     // the head amax is a maximum over all rows: that stage reads the rows in place
-    const bool gather = (w.z + z0) == 1 && a.perm != nullptr && STAGE != kStageAmax;
-    return gather ? min(max(__ldg(&a.perm[(size_t)w.bh * a.N + t]), 0), a.N - 1) : t;   // clamped: never a bad address
+    const bool gather = (c.z + z0) == 1 && a.perm != nullptr && STAGE != kStageAmax;
+    return gather ? min(max(__ldg(&a.perm[(size_t)(a.bh0 + c.hh) * a.N + t]), 0), a.N - 1) : t;   // clamped: never a bad address
   };
-  auto issue = [&](int item, int st, const int* src) {
+  auto issue = [&](int item, const Cursor& c, int st, const int* src) {
     if (item < n_items) {
-      const Item w = decode_item(item, a.nb, nh, a.bh0);
-      const int b = w.bh / a.H, h = w.bh - b * a.H;
-      const __nv_bfloat16* base = ((w.z + z0) == 0 ? a.q : a.k) + b * a.stride_b + h * a.stride_h + 8 * (tid % (D / 8));
-      unsigned char* dst = smem + st * Geo<D>::stage_bytes + 16 * (tid % (D / 8));
+      const char* base = reinterpret_cast<const char*>((c.z + z0) == 0 ? a.q : a.k) + head_offset_bytes(a, a.bh0 + c.hh) + 16 * (tid % (D / 8));
+      unsigned char* dst = smem + st * Geo<D>::stage_bytes + 16 * (tid % (D / 8)) + (tid / (D / 8)) * Geo<D>::pitch;
 #pragma unroll
-      for (int c = 0; c < kBlock * (D / 8) / NT; ++c) {
-        const int row = (c * NT + tid) / (D / 8);
-        const int sr = src[row];
-        if (sr >= 0) cp_async16(dst + row * Geo<D>::pitch, base + (int64_t)sr * a.stride_n);
+      for (int k = 0; k < kBlock * (D / 8) / NT; ++k) {
+        const int sr = src[tid / (D / 8) + k * (NT / (D / 8))];
+        if (sr >= 0) cp_async16(dst + k * (NT / (D / 8)) * Geo<D>::pitch, base + (int64_t)sr * a.stride_n_bytes);
       }
     }
     cp_async_commit();
   };
+  // cursors of items i, i+1 and i+3 of this CTA
+  const int g = gridDim.x;
+  Cursor c0 = cursor_at(blockIdx.x, a.nb, nh), c1 = c0;
+  advance(c1, step, a.nb, nh);
+  Cursor c3 = c1;
+  advance(c3, step, a.nb, nh);
   if (tid < kBlock) {
-    src_ring[tid] = fetch(blockIdx.x);
-    src_ring[kBlock + tid] = fetch(blockIdx.x + gridDim.x);
+    src_ring[tid] = fetch(blockIdx.x, c0);
+    src_ring[kBlock + tid] = fetch(blockIdx.x + g, c1);
   }
-  int nxt = fetch(blockIdx.x + 2 * gridDim.x);
+  int nxt = fetch(blockIdx.x + 2 * g, c3);    // (c3 still stands at item 2 here)
+  advance(c3, step, a.nb, nh);
   __syncthreads();
-  issue(blockIdx.x, 0, src_ring);
-  int i = 0, last_bh = -1;
-  for (int item = blockIdx.x; item < n_items; item += gridDim.x, ++i) {
+  issue(blockIdx.x, c0, 0, src_ring);
+  int i = 0, last_hh = -1;
+  for (int item = blockIdx.x; item < n_items; item += g, ++i) {
     cp_async_wait<0>();                       // my chunks of item i have landed ...
     __syncthreads();                          // ... and everyone's; item i-1 is finished everywhere
     if (tid < kBlock) src_ring[((i + 2) % 3) * kBlock + tid] = nxt;
-    nxt = fetch(item + 3 * gridDim.x);
-    issue(item + gridDim.x, (i + 1) & 1, src_ring + ((i + 1) % 3) * kBlock);
-    const Item w = decode_item(item, a.nb, nh, a.bh0);
+    nxt = fetch(item + 3 * g, c3);
+    issue(item + g, c1, (i + 1) & 1, src_ring + ((i + 1) % 3) * kBlock);
     const unsigned char* stage = smem + (i & 1) * Geo<D>::stage_bytes;
     const int s0 = src_ring[(i % 3) * kBlock + my_row];
-    const int tensor = w.z + z0;
-    qk_row_item<D, STAGE, TPR>(a, tensor, stage, out_tile, red, kmean_s, tab, w.bh, w.blk, i, tensor == 1 && w.bh != last_bh, s0);
-    if (tensor == 1) last_bh = w.bh;
+    const int tensor = c0.z + z0, bh = a.bh0 + c0.hh;
+    qk_row_item<D, STAGE, TPR>(a, tensor, stage, out_tile, red, kmean_s, tab, bh, c0.blk, i, tensor == 1 && c0.hh != last_hh, s0);
+    if (tensor == 1) last_hh = c0.hh;
     if constexpr (STAGE != kStageAmax) {
       __syncthreads();                        // the code tile is complete
-      uint8_t* gdst = (w.z + z0 == 0 ? a.q_codes : a.k_codes) + ((size_t)w.bh * a.n_pad + (size_t)w.blk * kBlock) * kRowBytes;
+      uint4* gdst = reinterpret_cast<uint4*>((tensor == 0 ? a.q_codes : a.k_codes) + ((size_t)bh * a.n_pad + (size_t)c0.blk * kBlock) * kRowBytes) + tid;
 #pragma unroll
-      for (int c = 0; c < CPR * kBlock / NT; ++c) {
-        const int idx = c * NT + tid, row = idx / CPR, chunk = idx % CPR;
+      for (int k = 0; k < CPR * kBlock / NT; ++k) {
+        const int idx = k * NT + tid, row = idx / CPR, chunk = idx % CPR;
         const int sw = (row / (8 / CPR)) & (CPR - 1);
-        const uint4 v = *reinterpret_cast<const uint4*>(out_tile + row * kRowBytes + ((chunk ^ sw) << 4));
-        *reinterpret_cast<uint4*>(gdst + (size_t)idx * 16) = v;
+        gdst[k * NT] = *reinterpret_cast<const uint4*>(out_tile + row * kRowBytes + ((chunk ^ sw) << 4));
       }
     }
+    c0 = c1;
+    advance(c1, step, a.nb, nh);
+    advance(c3, step, a.nb, nh);
   }
 }
 
@@ -825,7 +895,7 @@ cudaError_t run(const Problem& pr, PrepArgs a, const WorkLayout& wl, uint8_t* wo
   const size_t rope_bytes = ((a.flags & VC_FLAG_ROPE) && a.rope_in_smem) ? (size_t)a.rd.entries * 8 : 0;
   const size_t colsum_smem = 2 * (size_t)kThreads * (D / 16) * 16 + 8 * D * 4 + rope_bytes;
   const size_t row_smem = 2 * (size_t)Geo<D>::stage_bytes + (size_t)kBlock * D + 3 * kBlock * 4 + 64 + D * 4 + rope_bytes;
-  const size_t v_smem = 3 * (size_t)kBlock * 2 * D + 8 * D * 4;
+  const size_t v_smem = 3 * (size_t)kBlock * 2 * D + 8 * D * 4 + 2 * kBlock * 4;
   constexpr int kQuant = BITS == 8 ? kStageQuant8 : kStageQuant4;
   constexpr int kTpr = VC_PREP_TPR;            // threads per Q/K row
   constexpr int kVQuant = BITS == 8 ? kVQuant8 : kVQuant4;
@@ -880,6 +950,8 @@ cudaError_t launch_prep(const Problem& pr, const QuantLayout& ql, const WorkLayo
   a.q = (const __nv_bfloat16*)q; a.k = (const __nv_bfloat16*)k; a.v = (const __nv_bfloat16*)v;
   a.perm = perm;
   a.stride_b = pr.stride_b; a.stride_h = pr.stride_h; a.stride_n = pr.stride_n;
+  a.stride_n_bytes = (int)(2 * pr.stride_n);
+  a.mul_H = ((1ull << 40) + pr.H - 1) / pr.H;
   a.H = pr.H; a.N = pr.N; a.n_pad = pr.n_pad; a.nb = pr.nb; a.bh0 = 0; a.flags = pr.flags; a.BH = pr.BH;
   a.q_codes = quant + ql.q_codes; a.k_codes = quant + ql.k_codes; a.v_codes = quant + ql.v_codes;
   a.q_micro = quant + ql.q_micro; a.k_micro = quant + ql.k_micro; a.v_micro = quant + ql.v_micro;

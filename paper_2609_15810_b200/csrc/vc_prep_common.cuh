@@ -1,5 +1,4 @@
-// Declarations shared by the preprocessing kernels (vc_prep.cu: the 4-bit passes and the RoPE
-// table; vc_prep8.cu: the fused 8-bit pass).
+// Declarations shared by the preprocessing kernels.
 #pragma once
 #include <cuda_bf16.h>
 #include <cuda_fp4.h>
@@ -26,6 +25,8 @@ struct PrepArgs {
   const __nv_bfloat16 *q, *k, *v;
   const int32_t* perm;
   int64_t stride_b, stride_h, stride_n;
+  int stride_n_bytes;               // 2 * stride_n (a row stride fits 32 bits: checked when the call is resolved)
+  unsigned long long mul_H;         // ceil(2^40 / H): bh / H by one multiplication
   int H, N, n_pad, nb, bh0, flags, rope_in_smem, rope_default;
   uint8_t *q_codes, *k_codes, *v_codes, *q_micro, *k_micro, *v_micro;
   float *q_scale, *k_scale, *v_scale, *k_mean;
