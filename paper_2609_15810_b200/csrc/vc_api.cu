@@ -118,7 +118,7 @@ WorkLayout work_layout(const Problem& pr) {
   size_t off = 0;
   auto place = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 1024); return o; };
   W.status = place(256);
-  W.rope = place((size_t)e * 8);
+  W.rope = place((size_t)e * 16);   // (cos, sin) entries, then the same entries as (cos + sin, cos - sin)
   W.k_part = place(BH * nb * d * 4);
   W.v_mu = place(BH * nb * d * 4);
   W.amax_bytes = BH * d * 4 + 2 * BH * 4;

@@ -40,7 +40,7 @@ struct QuantLayout {
 // Byte offsets of the sections of the workspace.
 struct WorkLayout {
   size_t status;     // uint32 status word (+ padding)
-  size_t rope;       // float2 (cos, sin) compact per-axis tables
+  size_t rope;       // float2 (cos, sin) compact per-axis tables, then the same as (cos + sin, cos - sin)
   size_t k_part;     // fp32 [BH][nb][d] per-block column sums of RoPE(K)
   size_t v_mu;       // fp32 [BH][nb][d] block means of the gathered V
   size_t amax;       // uint32 [BH][d] residual amax bits (8-bit V) then [2][BH] Q/K head amax (4-bit)

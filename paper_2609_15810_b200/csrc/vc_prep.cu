@@ -30,7 +30,11 @@ __global__ void rope_table_kernel(float2* tab, RopeDesc rd, double theta) {
   int i = r - pos * rd.pairs[a];
   double freq = pow(theta, -2.0 * (double)i / (double)(2 * rd.pairs[a]));
   double phi = (double)pos * freq;
-  tab[e] = make_float2((float)cos(phi), (float)sin(phi));
+  const double c = cos(phi), sn = sin(phi);
+  tab[e] = make_float2((float)c, (float)sn);
+  // second table: the rotation folded into the first Hadamard level, u = x0 (c + s) + x1 (c - s),
+  // v = x0 (c - s) - x1 (c + s), each coefficient rounded once
+  tab[rd.entries + e] = make_float2((float)(c + sn), (float)(c - sn));
 }
 
 // ---------------------------------------------------------------------------------------
@@ -54,9 +58,6 @@ template <int D> struct Geo {
   static constexpr int stage_bytes = kBlock * pitch;
 };
 
-struct Item {
-  int z, bh, blk;
-};
 // Items are numbered block-fastest, then head, then tensor.  A CTA visits items blockIdx.x + k *
 // gridDim.x: the position is divided out once and then advanced by the grid stride with carries
 // (the divisions are not free at 64 elements per thread and item).
@@ -85,11 +86,6 @@ __device__ __forceinline__ void advance(Cursor& c, const CursorStep& s, int nb, 
   c.hh += s.dhh;
   if (c.blk >= nb) { c.blk -= nb; ++c.hh; }
   while (c.hh >= nh) { c.hh -= nh; ++c.z; }      // at most once unless the launch is tiny
-}
-__device__ __forceinline__ Item item_of(const Cursor& c, int bh0) {
-  Item it;
-  it.z = c.z; it.bh = bh0 + c.hh; it.blk = c.blk;
-  return it;
 }
 // Start of head bh in an input tensor, in bytes (bh = b * H + h, general strides).
 __device__ __forceinline__ int64_t head_offset_bytes(const PrepArgs& a, int bh) {
@@ -145,32 +141,81 @@ __device__ __forceinline__ void k_colsum_item(const PrepArgs& a, const unsigned 
   float s[8];
 #pragma unroll
   for (int c = 0; c < 8; ++c) s[c] = 0.f;
-#pragma unroll
-  for (int i = 0; i < RPL; ++i) {
-    const int row = 16 * warp + RPL * hb + i;
-    const int t = blk * kBlock + row;            // column sums need no gather: a sum over all rows
-    if (t >= a.N) break;                         // rows of a lane ascend: the rest is padding too
-    const uint4 raw = *reinterpret_cast<const uint4*>(stage + (i * kThreads + tid) * 16);   // the chunk this thread fetched
-    const unsigned int w[4] = {raw.x, raw.y, raw.z, raw.w};
-    float x[8];
-#pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      x[2 * j] = __uint_as_float(w[j] << 16);
-      x[2 * j + 1] = __uint_as_float(w[j] & 0xffff0000u);
-    }
-    if (do_rope) {
+  const int t0 = blk * kBlock + 16 * warp + RPL * hb;
+  const int n_rows = min(RPL, a.N - t0);           // rows of a lane ascend: the rest is padding
+  if (do_rope && tab.saddr) {
+    // The rotation is accumulated directly (four FMAs per channel pair and row).  The lane's four
+    // table addresses follow its rows: x advances by one per row, so the entries of the pairs on
+    // the x axis move by one table row and the others stay; a row that wraps x recomputes them.
+    // The coefficients of the pairs on the t and y axes are the same for all of a lane's rows
+    // unless x wraps, so they stay in registers; only lanes whose pairs lie on the x axis reload
+    // per row (a predicated load: the other lanes take no shared-memory bandwidth).
+    uint32_t ad[4], inc[4];
+    float cc[4], ss[4];
+    auto locate = [&]() {
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
         const int pos = ps.axis[j] == 0 ? tt : (ps.axis[j] == 1 ? ty : tx);
-        const float2 cs = rope_entry(tab, ps.idx[j] + pos * ps.stride[j]);
-        const float x0 = x[2 * j], x1 = x[2 * j + 1];
-        x[2 * j] = x0 * cs.x - x1 * cs.y;
-        x[2 * j + 1] = x0 * cs.y + x1 * cs.x;
+        ad[j] = tab.saddr + 8u * (uint32_t)(ps.idx[j] + pos * ps.stride[j]);
+        asm("ld.shared.v2.f32 {%0, %1}, [%2];" : "=f"(cc[j]), "=f"(ss[j]) : "r"(ad[j]));
       }
-      if (++tx == a.rd.grid_w) { tx = 0; if (++ty == a.rd.grid_h) { ty = 0; ++tt; } }
-    }
+    };
 #pragma unroll
-    for (int c = 0; c < 8; ++c) s[c] += x[c];
+    for (int j = 0; j < 4; ++j) inc[j] = ps.axis[j] == 2 ? 8u * (uint32_t)ps.stride[j] : 0u;
+    locate();
+#pragma unroll
+    for (int i = 0; i < RPL; ++i) {
+      if (i >= n_rows) break;
+      const uint4 raw = *reinterpret_cast<const uint4*>(stage + (i * kThreads + tid) * 16);   // the chunk this thread fetched
+      const unsigned int w[4] = {raw.x, raw.y, raw.z, raw.w};
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const float x0 = __uint_as_float(w[j] << 16), x1 = __uint_as_float(w[j] & 0xffff0000u);
+        s[2 * j] = fmaf(-x1, ss[j], fmaf(x0, cc[j], s[2 * j]));
+        s[2 * j + 1] = fmaf(x1, cc[j], fmaf(x0, ss[j], s[2 * j + 1]));
+      }
+      if (i + 1 < RPL) {
+        if (++tx == a.rd.grid_w) {
+          tx = 0;
+          if (++ty == a.rd.grid_h) { ty = 0; ++tt; }
+          locate();
+        } else {
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            if (inc[j]) {
+              ad[j] += inc[j];
+              asm("ld.shared.v2.f32 {%0, %1}, [%2];" : "=f"(cc[j]), "=f"(ss[j]) : "r"(ad[j]));
+            }
+          }
+        }
+      }
+    }
+  } else {
+#pragma unroll
+    for (int i = 0; i < RPL; ++i) {
+      if (i >= n_rows) break;
+      const uint4 raw = *reinterpret_cast<const uint4*>(stage + (i * kThreads + tid) * 16);   // the chunk this thread fetched
+      const unsigned int w[4] = {raw.x, raw.y, raw.z, raw.w};
+      float x[8];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        x[2 * j] = __uint_as_float(w[j] << 16);
+        x[2 * j + 1] = __uint_as_float(w[j] & 0xffff0000u);
+      }
+      if (do_rope) {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const int pos = ps.axis[j] == 0 ? tt : (ps.axis[j] == 1 ? ty : tx);
+          const float2 cs = rope_entry(tab, ps.idx[j] + pos * ps.stride[j]);
+          const float x0 = x[2 * j], x1 = x[2 * j + 1];
+          x[2 * j] = x0 * cs.x - x1 * cs.y;
+          x[2 * j + 1] = x0 * cs.y + x1 * cs.x;
+        }
+        if (++tx == a.rd.grid_w) { tx = 0; if (++ty == a.rd.grid_h) { ty = 0; ++tt; } }
+      }
+#pragma unroll
+      for (int c = 0; c < 8; ++c) s[c] += x[c];
+    }
   }
 #pragma unroll
   for (int c = 0; c < 8; ++c) {
@@ -421,9 +466,233 @@ __device__ __forceinline__ void qk_row_item(const PrepArgs& a, const int TENSOR 
 }
 
 // ---------------------------------------------------------------------------------------
+// The same row transform with fewer instructions, for the standard configuration (RoPE with the
+// default channel split and the table in shared memory, Hadamard on; K smoothing either way):
+//  * rotation, centering and the first Hadamard level are one step per channel pair: with
+//    (A, B) = (c + s, c - s) from the folded table and (m+, m-) = (m0 + m1, m0 - m1) of the mean,
+//    u = x0 A + x1 B - m+  and  v = x0 B - x1 A - m-  are the level-1 outputs (4 FMAs per pair);
+//  * a pair lives in one 64-bit register and the other levels, the cross-lane level and the scale
+//    multiply are packed two-lane FP32 instructions (add / sub / fma / mul .f32x2: the same FP32
+//    operation per lane, one instruction issued for two);
+//  * 1 / sqrt(D) and the quantization scale are one factor.
+// `kmean_pm` holds (m+, m-) per pair, zeros while Q rows or unsmoothed K rows are processed.
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
+  uint64_t d;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+__device__ __forceinline__ uint64_t sub2(uint64_t a, uint64_t b) {
+  uint64_t d;
+  asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+__device__ __forceinline__ uint64_t mul2(uint64_t a, uint64_t b) {
+  uint64_t d;
+  asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
+  uint64_t d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ void unpack2(uint64_t v, float& lo, float& hi) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+
+template <int D, int STAGE, int TPR>
+__device__ __forceinline__ void qk_row_item_fast(const PrepArgs& a, const int TENSOR, const unsigned char* stage,
+                                                 unsigned char* out_tile, float* red, float* kmean_pm, uint32_t tab_saddr,
+                                                 int bh, int blk, int iter, bool new_head, int src_row) {
+  static_assert(STAGE == kStageQuant8 || STAGE == kStageQuant8I, "the packed path covers the 8-bit stages");
+  constexpr int C = D / TPR, P = C / 2;            // channels and pairs per thread
+  constexpr int NT = kRowThreads * TPR;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int row = qk_row_of<TPR>(tid), part = qk_part_of<TPR>(tid);
+  const bool valid = src_row >= 0;
+  const int src = valid ? src_row : 0;
+  uint4 raw[C / 8];
+#pragma unroll
+  for (int i = 0; i < C / 8; ++i) raw[i] = *reinterpret_cast<const uint4*>(stage + row * Geo<D>::pitch + part * (2 * C) + 16 * i);
+  if (TENSOR == 1 && (a.flags & VC_FLAG_K_SMOOTH) && new_head) {
+    __syncthreads();                               // everyone is done with the previous head's mean
+    for (int pr = tid; pr < D / 2; pr += NT) {
+      const float2 m = *reinterpret_cast<const float2*>(a.k_mean + (size_t)bh * D + 2 * pr);
+      *reinterpret_cast<float2*>(kmean_pm + 2 * pr) = make_float2(m.x + m.y, m.x - m.y);
+    }
+    __syncthreads();
+  }
+  int tt, ty, tx;
+  grid_pos(a.rd, src, tt, ty, tx);
+  const int e[3] = {a.rd.off[0] + tt * a.rd.pairs[0] - a.rd.pair_start[0],
+                    a.rd.off[1] + ty * a.rd.pairs[1] - a.rd.pair_start[1],
+                    a.rd.off[2] + tx * a.rd.pairs[2] - a.rd.pair_start[2]};
+  const int p0 = part * P;
+  // byte address of pair i's entry = base of its axis + 8 i (the axis of local pair i is known at
+  // compile time for either part: one base per combination, selected once per row)
+  uint32_t base[3][3];
+#pragma unroll
+  for (int a0 = 0; a0 < 3; ++a0)
+#pragma unroll
+    for (int a1 = 0; a1 < 3; ++a1) base[a0][a1] = tab_saddr + 8u * (uint32_t)((part ? e[a1] : e[a0]) + p0);
+  const float4* km = reinterpret_cast<const float4*>(kmean_pm + part * C);
+
+  uint64_t X[P];
+#pragma unroll
+  for (int i = 0; i < P; i += 2) {
+    const float4 m = km[i / 2];                    // (m+, m-) of pairs i and i + 1
+#pragma unroll
+    for (int k = 0; k < 2; ++k) {
+      const int ii = i + k;
+      const unsigned int w = ii % 4 == 0 ? raw[ii / 4].x : (ii % 4 == 1 ? raw[ii / 4].y : (ii % 4 == 2 ? raw[ii / 4].z : raw[ii / 4].w));
+      const float x0 = __uint_as_float(w << 16), x1 = __uint_as_float(w & 0xffff0000u);
+      float A, B;
+      asm("ld.shared.v2.f32 {%0, %1}, [%2];" : "=f"(A), "=f"(B)
+          : "r"(base[rope_axis_of<D>(ii)][rope_axis_of<D>(TPR == 1 ? ii : P + ii)] + 8u * ii));
+      const float mp = k == 0 ? m.x : m.z, mm = k == 0 ? m.y : m.w;
+      const float u = fmaf(x0, A, fmaf(x1, B, -mp));
+      const float v = fmaf(x0, B, fmaf(-x1, A, -mm));
+      X[ii] = pack_f32x2(u, v);
+    }
+  }
+  if (!valid) {                                    // a padding row: zeros (codes 0, no part in the maximum)
+#pragma unroll
+    for (int i = 0; i < P; ++i) X[i] = 0ull;
+  }
+  // Hadamard levels 2 .. C/2 on whole pairs
+#pragma unroll
+  for (int h = 1; h < P; h <<= 1) {
+#pragma unroll
+    for (int i = 0; i < P; ++i) {
+      if (!(i & h)) {
+        const uint64_t U = X[i], V = X[i | h];
+        X[i] = add2(U, V);
+        X[i | h] = sub2(U, V);
+      }
+    }
+  }
+  if constexpr (TPR == 2) {
+    // the level that pairs channel c with c + D/2: lower half mine + theirs, upper half theirs - mine
+    const float sg = part ? -1.0f : 1.0f;
+    const uint64_t SG = pack_f32x2(sg, sg);
+#pragma unroll
+    for (int i = 0; i < P; ++i) {
+      float lo, hi;
+      unpack2(X[i], lo, hi);
+      const float olo = __shfl_xor_sync(0xffffffffu, lo, 16), ohi = __shfl_xor_sync(0xffffffffu, hi, 16);
+      X[i] = fma2(X[i], SG, pack_f32x2(olo, ohi));
+    }
+  }
+  constexpr float rs = D == 128 ? 0.08838834764831845f : 0.125f;   // 1/sqrt(D)
+
+  float m0 = 0.f, m1 = 0.f;
+#pragma unroll
+  for (int i = 0; i < P; i += 2) {
+    float a0, a1, b0, b1;
+    unpack2(X[i], a0, a1);
+    unpack2(X[i + 1], b0, b1);
+    m0 = max3(m0, fabsf(a0), fabsf(a1));
+    m1 = max3(m1, fabsf(b0), fabsf(b1));
+  }
+  float amax = warp_max(fmaxf(m0, m1) * rs);       // max and the (positive) scale commute exactly
+  float* rbuf = red + 8 * (iter & 1);              // alternate buffers: one barrier per item suffices
+  if (lane == 0) rbuf[warp] = amax;
+  __syncthreads();
+  amax = fmaxf(fmaxf(rbuf[0], rbuf[1]), fmaxf(rbuf[2], rbuf[3]));
+  if constexpr (TPR == 2) amax = fmaxf(amax, fmaxf(fmaxf(rbuf[4], rbuf[5]), fmaxf(rbuf[6], rbuf[7])));
+
+  constexpr bool int8 = STAGE == kStageQuant8I;
+  const float top = int8 ? 127.0f : 448.0f;
+  const float f = amax > 0.f ? rs * (top / amax) : 0.f;   // 1/sqrt(D) and 1/scale in one factor
+  if (tid == 0) (TENSOR == 0 ? a.q_scale : a.k_scale)[(size_t)bh * a.nb + blk] = amax > 0.f ? amax / top : 1.0f;
+  const uint64_t F = pack_f32x2(f, f);
+  constexpr int CPR = D / 16;
+  uint4* dst = reinterpret_cast<uint4*>(out_tile + row * D);
+  const int sw = (row / (8 / CPR)) & (CPR - 1);
+#pragma unroll
+  for (int i = 0; i < C / 16; ++i) {
+    unsigned int w[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int pi = 8 * i + 2 * j;                // pairs pi, pi + 1 = channels 16 i + 4 j .. + 3
+      if constexpr (int8) {
+        const uint64_t MG = pack_f32x2(12582912.0f, 12582912.0f);
+        const uint64_t ra = fma2(X[pi], F, MG), rb = fma2(X[pi + 1], F, MG);
+        w[j] = __byte_perm(__byte_perm((unsigned int)ra, (unsigned int)(ra >> 32), 0x0040),
+                           __byte_perm((unsigned int)rb, (unsigned int)(rb >> 32), 0x0040), 0x5410);
+      } else {
+        float y0, y1, y2, y3;
+        unpack2(mul2(X[pi], F), y0, y1);
+        unpack2(mul2(X[pi + 1], F), y2, y3);
+        const unsigned int lo = __nv_cvt_float2_to_fp8x2(make_float2(y0, y1), __NV_SATFINITE, __NV_E4M3);
+        const unsigned int hi = __nv_cvt_float2_to_fp8x2(make_float2(y2, y3), __NV_SATFINITE, __NV_E4M3);
+        w[j] = lo | (hi << 16);
+      }
+    }
+    dst[(part * (C / 16) + i) ^ sw] = make_uint4(w[0], w[1], w[2], w[3]);
+  }
+}
+
+// ---------------------------------------------------------------------------------------
 // V.  A thread owns one channel pair and 128 / (256 / (D/2)) consecutive tokens of the gathered
 // block, so block means and the channel-major (token-contiguous) code rows need no transposition.
 enum { kVStats = 0, kVQuant8 = 1, kVQuant4 = 2, kVQuant4M = 3 };   // 4M: E2M1 under power-of-two factors per 32 tokens
+
+// Statistics of a value block (launch 1b): block mean per channel (Eq. 4) and the block's
+// max |v - mu|, folded into the head's per-channel maximum.  One pass over the thread's tokens
+// collects the sum, the maximum and the minimum (the last two on the packed bf16 pairs as they
+// are: max/min.bf16x2), one exchange combines the token groups, and
+//     max_i |v_i - mu| = max(max_i v_i - mu, mu - min_i v_i)
+// bit for bit, because the FP32 subtraction is monotonic.
+template <int D, bool FULL>
+__device__ __forceinline__ void v_stats_item(const PrepArgs& a, const unsigned char* stage, float* red, int bh, int blk) {
+  constexpr int CP = D / 2, TG = kThreads / CP, TPG = kBlock / TG;
+  const int tid = threadIdx.x;
+  const int cp = tid % CP, tg = tid / CP;
+  const int n_valid = FULL ? kBlock : min(kBlock, a.N - blk * kBlock);
+  const unsigned char* mine = stage + tg * TPG * (2 * D) + 4 * cp;
+  float s0 = 0.f, s1 = 0.f;
+  __nv_bfloat162 mx = __halves2bfloat162(__ushort_as_bfloat16(0xff80), __ushort_as_bfloat16(0xff80));   // -inf
+  __nv_bfloat162 mn = __halves2bfloat162(__ushort_as_bfloat16(0x7f80), __ushort_as_bfloat16(0x7f80));   // +inf
+#pragma unroll
+  for (int i = 0; i < TPG; ++i) {
+    if (FULL || tg * TPG + i < n_valid) {
+      const unsigned int w = *reinterpret_cast<const unsigned int*>(mine + i * (2 * D));
+      s0 += __uint_as_float(w << 16);
+      s1 += __uint_as_float(w & 0xffff0000u);
+      const __nv_bfloat162 v = *reinterpret_cast<const __nv_bfloat162*>(&w);
+      mx = __hmax2(mx, v);
+      mn = __hmin2(mn, v);
+    }
+  }
+  // red: [TG][D] sums, then [TG][CP] packed maxima, then [TG][CP] packed minima
+  unsigned int* red_mx = reinterpret_cast<unsigned int*>(red + TG * D);
+  unsigned int* red_mn = red_mx + TG * CP;
+  *reinterpret_cast<float2*>(red + tg * D + 2 * cp) = make_float2(s0, s1);
+  red_mx[tg * CP + cp] = *reinterpret_cast<unsigned int*>(&mx);
+  red_mn[tg * CP + cp] = *reinterpret_cast<unsigned int*>(&mn);
+  __syncthreads();                           // (the barrier at the top of the next item covers these reads)
+  if (tg == 0) {
+    s0 = 0.f; s1 = 0.f;
+#pragma unroll
+    for (int g = 0; g < TG; ++g) {
+      const float2 p = *reinterpret_cast<const float2*>(red + g * D + 2 * cp);
+      s0 += p.x; s1 += p.y;
+      if (g > 0) {
+        mx = __hmax2(mx, *reinterpret_cast<const __nv_bfloat162*>(&red_mx[g * CP + cp]));
+        mn = __hmin2(mn, *reinterpret_cast<const __nv_bfloat162*>(&red_mn[g * CP + cp]));
+      }
+    }
+    const bool smooth = a.flags & VC_FLAG_V_SMOOTH;
+    const float mu0 = smooth ? s0 / (float)n_valid : 0.f, mu1 = smooth ? s1 / (float)n_valid : 0.f;
+    const size_t mu_at = ((size_t)bh * a.nb + blk) * D + 2 * cp;
+    *reinterpret_cast<float2*>(a.v_mu + mu_at) = make_float2(mu0, mu1);
+    const float2 hi = __bfloat1622float2(mx), lo = __bfloat1622float2(mn);
+    const float m0 = fmaxf(hi.x - mu0, mu0 - lo.x), m1 = fmaxf(hi.y - mu1, mu1 - lo.y);
+    atomicMax(&a.v_amax[(size_t)bh * D + 2 * cp], __float_as_uint(m0));
+    atomicMax(&a.v_amax[(size_t)bh * D + 2 * cp + 1], __float_as_uint(m1));
+  }
+}
 
 // FULL: all 128 rows of the block exist (every block but a head's ragged last one): no row tests.
 template <int D, int STAGE, bool FULL>
@@ -451,7 +720,8 @@ __device__ __forceinline__ void v_item(const PrepArgs& a, const unsigned char* s
   // other blocks: the block mean is formed here, in the quantizing pass, and the statistics
   // launch is not needed.
   constexpr bool kFusedMean = STAGE == kVQuant4 || STAGE == kVQuant4M;
-  if constexpr (STAGE == kVStats || kFusedMean) {
+  static_assert(STAGE != kVStats, "the statistics stage has its own item function");
+  if constexpr (kFusedMean) {
     __syncthreads();                         // the previous item's reads of `red` are done
     if (smooth) {
       float s0 = 0.f, s1 = 0.f;
@@ -474,28 +744,6 @@ __device__ __forceinline__ void v_item(const PrepArgs& a, const unsigned char* s
       __syncthreads();
     }
   }
-  if constexpr (STAGE == kVStats) {
-    if (tg == 0) { a.v_mu[mu_at] = mu0; a.v_mu[mu_at + 1] = mu1; }
-    float m0 = 0.f, m1 = 0.f;
-#pragma unroll
-    for (int i = 0; i < TPG; ++i) {
-      if (FULL || tg * TPG + i < n_valid) {
-        m0 = fmaxf(m0, fabsf(v0[i] - mu0));
-        m1 = fmaxf(m1, fabsf(v1[i] - mu1));
-      }
-    }
-    red[tg * D + 2 * cp] = m0;
-    red[tg * D + 2 * cp + 1] = m1;
-    __syncthreads();
-    if (tg == 0) {
-#pragma unroll
-      for (int g = 1; g < TG; ++g) { m0 = fmaxf(m0, red[g * D + 2 * cp]); m1 = fmaxf(m1, red[g * D + 2 * cp + 1]); }
-      atomicMax(&a.v_amax[(size_t)bh * D + 2 * cp], __float_as_uint(m0));
-      atomicMax(&a.v_amax[(size_t)bh * D + 2 * cp + 1], __float_as_uint(m1));
-    }
-    return;
-  }
-
   if constexpr (!kFusedMean) {
     mu0 = mu_in.x;
     mu1 = mu_in.y;
@@ -633,11 +881,12 @@ __device__ __forceinline__ void v_item(const PrepArgs& a, const unsigned char* s
 
 // ---------------------------------------------------------------------------------------
 // RoPE table -> shared memory (when it fits), once per CTA.
-__device__ __forceinline__ RopeTab stage_rope_table(const PrepArgs& a, unsigned char* at) {
-  RopeTab tab{0u, a.rope};
+__device__ __forceinline__ RopeTab stage_rope_table(const PrepArgs& a, unsigned char* at, bool folded = false) {
+  const float2* src = a.rope + (folded ? a.rd.entries : 0);
+  RopeTab tab{0u, src};
   if ((a.flags & VC_FLAG_ROPE) && a.rope_in_smem) {
     float2* tab_s = reinterpret_cast<float2*>(at);
-    for (int e = threadIdx.x; e < a.rd.entries; e += blockDim.x) tab_s[e] = __ldg(&a.rope[e]);
+    for (int e = threadIdx.x; e < a.rd.entries; e += blockDim.x) tab_s[e] = __ldg(&src[e]);
     tab.saddr = smem_u32(at);
   }
   __syncthreads();
@@ -681,13 +930,13 @@ __global__ void __launch_bounds__(kThreads, 2) prep_kcolsum_kernel(const PrepArg
 }
 
 // V pass: STAGE = block means + residual amax (launch 1b) or quantization of the residual.
-// Shared memory: [3 stages x (128 x 2 D)][red: 8 D floats][source rows: 2 x 128].
+// Shared memory: [3 stages x (128 x 2 D)][red: 16 D floats][source rows: 2 x 128].
 template <int D, int STAGE>
 __global__ void __launch_bounds__(kThreads, 2) prep_v_kernel(const PrepArgs a, int n_items, int nh) {
   constexpr int LPR = D / 8, kStage = kBlock * 2 * D, NL = kBlock * LPR / kThreads;
   extern __shared__ __align__(128) unsigned char smem[];
   float* red = reinterpret_cast<float*>(smem + 3 * kStage);
-  int* src_ring = reinterpret_cast<int*>(red + 8 * D);                 // [2][128]
+  int* src_ring = reinterpret_cast<int*>(red + 16 * D);                // [2][128]
   const int tid = threadIdx.x;
   const CursorStep step = cursor_step(a.nb);
   // source row of row `tid` of an item (the gather by pi), -1 if there is none
@@ -749,8 +998,14 @@ __global__ void __launch_bounds__(kThreads, 2) prep_v_kernel(const PrepArgs a, i
       last_hh = c0.hh;
     }
     const unsigned char* stage = smem + (i % 3) * kStage;
-    if (a.N - c0.blk * kBlock >= kBlock) v_item<D, STAGE, true>(a, stage, red, a.bh0 + c0.hh, c0.blk, mu, am);
-    else v_item<D, STAGE, false>(a, stage, red, a.bh0 + c0.hh, c0.blk, mu, am);
+    const bool full = a.N - c0.blk * kBlock >= kBlock;
+    if constexpr (STAGE == kVStats) {
+      if (full) v_stats_item<D, true>(a, stage, red, a.bh0 + c0.hh, c0.blk);
+      else v_stats_item<D, false>(a, stage, red, a.bh0 + c0.hh, c0.blk);
+    } else {
+      if (full) v_item<D, STAGE, true>(a, stage, red, a.bh0 + c0.hh, c0.blk, mu, am);
+      else v_item<D, STAGE, false>(a, stage, red, a.bh0 + c0.hh, c0.blk, mu, am);
+    }
     mu = mu_next;
     c0 = c1; c1 = c2;
     advance(c2, step, a.nb, nh);
@@ -761,15 +1016,24 @@ __global__ void __launch_bounds__(kThreads, 2) prep_v_kernel(const PrepArgs a, i
 // Launch 2: per-head finalization: K channel mean, V scale, g_Q.
 template <int D, int BITS>
 __global__ void prep_finalize_kernel(const PrepArgs a, int which) {
-  const int bh = a.bh0 + blockIdx.x, c = threadIdx.x;
+  // which 0 / 2: a block of 8 D threads per head; the block partial sums are added in double, in
+  // eight interleaved slices that are then added in a fixed order
+  __shared__ double part[8][D];
+  const int bh = a.bh0 + blockIdx.x, c = threadIdx.x % D, slice = threadIdx.x / D;
   if (which == 0 || which == 2) {
-    if (c < D) {
+    if (which == 0 && (a.flags & VC_FLAG_K_SMOOTH)) {
+      double s = 0.0;
+      for (int j = slice; j < a.nb; j += 8) s += (double)a.k_part[((size_t)bh * a.nb + j) * D + c];
+      part[slice][c] = s;
+      __syncthreads();
+    }
+    if (slice == 0) {
       if (which == 2) {        // statistics from the caller: the mean as given (zero if K smoothing is off)
         a.k_mean[(size_t)bh * D + c] = (a.flags & VC_FLAG_K_SMOOTH) ? a.ext_k_mean[(size_t)bh * D + c] : 0.f;
       } else {
         double s = 0.0;
         if (a.flags & VC_FLAG_K_SMOOTH)
-          for (int j = 0; j < a.nb; ++j) s += (double)a.k_part[((size_t)bh * a.nb + j) * D + c];
+          for (int k = 0; k < 8; ++k) s += part[k][c];
         a.k_mean[(size_t)bh * D + c] = (float)(s / (double)a.N);
       }
       float vs = 1.0f;
@@ -779,39 +1043,48 @@ __global__ void prep_finalize_kernel(const PrepArgs a, int which) {
       }
       a.v_scale[(size_t)bh * D + c] = vs;
     }
-    if (BITS == 4 && c == 0) {
+    if (BITS == 4 && threadIdx.x == 0) {
       const float am = __uint_as_float(a.qk_amax[bh]);
       a.q_scale[bh] = am > 0.f ? am / 2688.0f : 1.0f;
     }
-  } else if (BITS == 4 && c == 0) {
+  } else if (BITS == 4 && threadIdx.x == 0) {
     const float am = __uint_as_float(a.qk_amax[a.BH + bh]);
     a.k_scale[bh] = am > 0.f ? am / 2688.0f : 1.0f;
   }
 }
 
-// Q/K pass, one row per thread: STAGE = amax (4-bit head amax of tensor z0), or quantization
-// of Q (z = 0) and K (z = 1).  Loads and stores are coalesced: the CTA copies the next block in
-// with consecutive lanes on consecutive 16-byte chunks (two rows per warp instruction, the source
-// rows taken from a small ring of permutation slices in shared memory), a thread then reads its
-// row from the padded tile; codes leave through a swizzled tile in the same way.
+// Q/K pass: STAGE = amax (4-bit head amax of tensor z0), or quantization of Q (z = 0) and K
+// (z = 1).  A warp owns 32 / TPR rows of the block from end to end: it copies them in (consecutive
+// lanes on consecutive 16-byte chunks, the source rows taken from a small ring of permutation
+// entries in shared memory), its threads read their rows from the padded tile, and the rows'
+// codes leave through the warp's slice of a swizzled tile, again with full-line stores.  So the
+// data needs warp-level synchronization only; the one CTA-wide barrier per item is the exchange
+// of the block maximum.
 // Shared memory: [2 stages x 128 x pitch][out tile 128 x D][src ring 3 x 128][scratch][RoPE table].
-template <int D, int STAGE, int TPR>
+// FAST: the packed row transform (standard configuration, 8-bit stages), see qk_row_item_fast.
+template <int D, int STAGE, int TPR, bool FAST = false>
 __global__ void __launch_bounds__(kRowThreads * TPR, 2) prep_qk_kernel(const PrepArgs a, int n_items, int nh, int z0) {
   constexpr int NT = kRowThreads * TPR;
   constexpr int kRowBytes = STAGE == kStageQuant4 ? D / 2 : D;      // code bytes per row
   constexpr int CPR = kRowBytes / 16;                                // 16-byte chunks per code row
+  constexpr int RW = 32 / TPR;                                       // rows of a warp
+  constexpr int LPR = D / 8;                                         // lanes on one input row
+  constexpr int RPI = 32 / LPR;                                      // input rows per warp instruction
   extern __shared__ __align__(128) unsigned char smem[];
   unsigned char* out_tile = smem + 2 * Geo<D>::stage_bytes;
   int* src_ring = reinterpret_cast<int*>(out_tile + kBlock * D);     // [3][128]
   float* red = reinterpret_cast<float*>(src_ring + 3 * kBlock);      // [2][8]
   float* kmean_s = red + 16;                                         // [D]
-  const RopeTab tab = stage_rope_table(a, reinterpret_cast<unsigned char*>(kmean_s + D));
-  const int tid = threadIdx.x;
+  const int tid = threadIdx.x, lane = tid & 31, row0 = (tid >> 5) * RW;
+  if (FAST) {
+    for (int c = tid; c < D; c += NT) kmean_s[c] = 0.f;    // (m+, m-) pairs: zeros until a smoothed K head arrives
+  }
+  const RopeTab tab = stage_rope_table(a, reinterpret_cast<unsigned char*>(kmean_s + D), FAST);
   const int my_row = qk_row_of<TPR>(tid);
   const CursorStep step = cursor_step(a.nb);
-  auto fetch = [&](int item, const Cursor& c) -> int {   // input row behind row `tid` of the item, -1 if none
-    if (item >= n_items || tid >= kBlock) return -1;
-    const int t = c.blk * kBlock + tid;
+  auto fetch = [&](int item, const Cursor& c) -> int {   // input row behind row `row0 + lane` of the item, -1 if none
+    if (item >= n_items || lane >= RW) return -1;
+    const int t = c.blk * kBlock + row0 + lane;
     if (t >= a.N) return -1;
     // the head amax is a maximum over all rows: that stage reads the rows in place
     const bool gather = (c.z + z0) == 1 && a.perm != nullptr && STAGE != kStageAmax;
@@ -819,12 +1092,12 @@ __global__ void __launch_bounds__(kRowThreads * TPR, 2) prep_qk_kernel(const Pre
   };
   auto issue = [&](int item, const Cursor& c, int st, const int* src) {
     if (item < n_items) {
-      const char* base = reinterpret_cast<const char*>((c.z + z0) == 0 ? a.q : a.k) + head_offset_bytes(a, a.bh0 + c.hh) + 16 * (tid % (D / 8));
-      unsigned char* dst = smem + st * Geo<D>::stage_bytes + 16 * (tid % (D / 8)) + (tid / (D / 8)) * Geo<D>::pitch;
+      const char* base = reinterpret_cast<const char*>((c.z + z0) == 0 ? a.q : a.k) + head_offset_bytes(a, a.bh0 + c.hh) + 16 * (lane % LPR);
+      unsigned char* dst = smem + st * Geo<D>::stage_bytes + 16 * (lane % LPR) + (row0 + lane / LPR) * Geo<D>::pitch;
 #pragma unroll
-      for (int k = 0; k < kBlock * (D / 8) / NT; ++k) {
-        const int sr = src[tid / (D / 8) + k * (NT / (D / 8))];
-        if (sr >= 0) cp_async16(dst + k * (NT / (D / 8)) * Geo<D>::pitch, base + (int64_t)sr * a.stride_n_bytes);
+      for (int k = 0; k < RW / RPI; ++k) {
+        const int sr = src[row0 + lane / LPR + k * RPI];
+        if (sr >= 0) cp_async16(dst + k * RPI * Geo<D>::pitch, base + (int64_t)sr * a.stride_n_bytes);
       }
     }
     cp_async_commit();
@@ -835,34 +1108,37 @@ __global__ void __launch_bounds__(kRowThreads * TPR, 2) prep_qk_kernel(const Pre
   advance(c1, step, a.nb, nh);
   Cursor c3 = c1;
   advance(c3, step, a.nb, nh);
-  if (tid < kBlock) {
-    src_ring[tid] = fetch(blockIdx.x, c0);
-    src_ring[kBlock + tid] = fetch(blockIdx.x + g, c1);
+  if (lane < RW) {
+    src_ring[row0 + lane] = fetch(blockIdx.x, c0);
+    src_ring[kBlock + row0 + lane] = fetch(blockIdx.x + g, c1);
   }
   int nxt = fetch(blockIdx.x + 2 * g, c3);    // (c3 still stands at item 2 here)
   advance(c3, step, a.nb, nh);
-  __syncthreads();
+  __syncwarp();
   issue(blockIdx.x, c0, 0, src_ring);
   int i = 0, last_hh = -1;
   for (int item = blockIdx.x; item < n_items; item += g, ++i) {
     cp_async_wait<0>();                       // my chunks of item i have landed ...
-    __syncthreads();                          // ... and everyone's; item i-1 is finished everywhere
-    if (tid < kBlock) src_ring[((i + 2) % 3) * kBlock + tid] = nxt;
+    __syncwarp();                             // ... and the warp's; the warp is done with item i-1
+    if (lane < RW) src_ring[((i + 2) % 3) * kBlock + row0 + lane] = nxt;
     nxt = fetch(item + 3 * g, c3);
     issue(item + g, c1, (i + 1) & 1, src_ring + ((i + 1) % 3) * kBlock);
     const unsigned char* stage = smem + (i & 1) * Geo<D>::stage_bytes;
     const int s0 = src_ring[(i % 3) * kBlock + my_row];
     const int tensor = c0.z + z0, bh = a.bh0 + c0.hh;
-    qk_row_item<D, STAGE, TPR>(a, tensor, stage, out_tile, red, kmean_s, tab, bh, c0.blk, i, tensor == 1 && c0.hh != last_hh, s0);
+    if constexpr (FAST)
+      qk_row_item_fast<D, STAGE, TPR>(a, tensor, stage, out_tile, red, kmean_s, tab.saddr, bh, c0.blk, i, tensor == 1 && c0.hh != last_hh, s0);
+    else
+      qk_row_item<D, STAGE, TPR>(a, tensor, stage, out_tile, red, kmean_s, tab, bh, c0.blk, i, tensor == 1 && c0.hh != last_hh, s0);
     if (tensor == 1) last_hh = c0.hh;
     if constexpr (STAGE != kStageAmax) {
-      __syncthreads();                        // the code tile is complete
-      uint4* gdst = reinterpret_cast<uint4*>((tensor == 0 ? a.q_codes : a.k_codes) + ((size_t)bh * a.n_pad + (size_t)c0.blk * kBlock) * kRowBytes) + tid;
+      __syncwarp();                           // the warp's rows of the code tile are complete
+      uint4* gdst = reinterpret_cast<uint4*>((tensor == 0 ? a.q_codes : a.k_codes) + ((size_t)bh * a.n_pad + (size_t)c0.blk * kBlock + row0) * kRowBytes) + lane;
 #pragma unroll
-      for (int k = 0; k < CPR * kBlock / NT; ++k) {
-        const int idx = k * NT + tid, row = idx / CPR, chunk = idx % CPR;
+      for (int k = 0; k < CPR * RW / 32; ++k) {
+        const int idx = k * 32 + lane, row = row0 + idx / CPR, chunk = idx % CPR;
         const int sw = (row / (8 / CPR)) & (CPR - 1);
-        gdst[k * NT] = *reinterpret_cast<const uint4*>(out_tile + row * kRowBytes + ((chunk ^ sw) << 4));
+        gdst[k * 32] = *reinterpret_cast<const uint4*>(out_tile + row * kRowBytes + ((chunk ^ sw) << 4));
       }
     }
     c0 = c1;
@@ -895,7 +1171,7 @@ cudaError_t run(const Problem& pr, PrepArgs a, const WorkLayout& wl, uint8_t* wo
   const size_t rope_bytes = ((a.flags & VC_FLAG_ROPE) && a.rope_in_smem) ? (size_t)a.rd.entries * 8 : 0;
   const size_t colsum_smem = 2 * (size_t)kThreads * (D / 16) * 16 + 8 * D * 4 + rope_bytes;
   const size_t row_smem = 2 * (size_t)Geo<D>::stage_bytes + (size_t)kBlock * D + 3 * kBlock * 4 + 64 + D * 4 + rope_bytes;
-  const size_t v_smem = 3 * (size_t)kBlock * 2 * D + 8 * D * 4 + 2 * kBlock * 4;
+  const size_t v_smem = 3 * (size_t)kBlock * 2 * D + 16 * D * 4 + 2 * kBlock * 4;
   constexpr int kQuant = BITS == 8 ? kStageQuant8 : kStageQuant4;
   constexpr int kTpr = VC_PREP_TPR;            // threads per Q/K row
   constexpr int kVQuant = BITS == 8 ? kVQuant8 : kVQuant4;
@@ -907,6 +1183,10 @@ cudaError_t run(const Problem& pr, PrepArgs a, const WorkLayout& wl, uint8_t* wo
   const bool v_pow2 = hybrid4(pr);           // 4-bit values under power-of-two factors per 32 tokens
   if ((e = allow_smem(prep_qk_kernel<D, kQuant, kTpr>, row_smem)) != cudaSuccess) return e;
   if (BITS == 8 && (e = allow_smem(prep_qk_kernel<D, kStageQuant8I, kTpr>, row_smem)) != cudaSuccess) return e;
+  if (BITS == 8 && (e = allow_smem(prep_qk_kernel<D, kStageQuant8, kTpr, true>, row_smem)) != cudaSuccess) return e;
+  if (BITS == 8 && (e = allow_smem(prep_qk_kernel<D, kStageQuant8I, kTpr, true>, row_smem)) != cudaSuccess) return e;
+  // the packed row transform serves the standard configuration
+  const bool fast = BITS == 8 && (a.flags & VC_FLAG_ROPE) && (a.flags & VC_FLAG_HADAMARD) && a.rope_default && a.rope_in_smem;
   if (BITS == 4 && (e = allow_smem(prep_qk_kernel<D, kStageAmax, kTpr>, row_smem)) != cudaSuccess) return e;
   int group = pr.heads_per_pass > 0 ? pr.heads_per_pass : pr.BH;
   if (group > 32768) group = 32768;
@@ -921,17 +1201,25 @@ cudaError_t run(const Problem& pr, PrepArgs a, const WorkLayout& wl, uint8_t* wo
     }
     if (BITS == 8 && !ext) { prep_v_kernel<D, kVStats><<<persistent_grid(per), kThreads, v_smem, s>>>(a, per, nh); count_launches(1); }
     if (BITS == 4) { prep_qk_kernel<D, kStageAmax, kTpr><<<persistent_grid(per), kRowThreads * kTpr, row_smem, s>>>(a, per, nh, 0); count_launches(1); }
-    prep_finalize_kernel<D, BITS><<<nh, D, 0, s>>>(a, ext ? 2 : 0);
+    prep_finalize_kernel<D, BITS><<<nh, 8 * D, 0, s>>>(a, ext ? 2 : 0);
     count_launches(1);
     if (BITS == 4) {
       prep_qk_kernel<D, kStageAmax, kTpr><<<persistent_grid(per), kRowThreads * kTpr, row_smem, s>>>(a, per, nh, 1);
       prep_finalize_kernel<D, BITS><<<nh, 32, 0, s>>>(a, 1);
       count_launches(2);
     }
-    if (BITS == 8 && (a.flags & VC_FLAG_INT8_QK))
-      prep_qk_kernel<D, kStageQuant8I, kTpr><<<persistent_grid(2 * per), kRowThreads * kTpr, row_smem, s>>>(a, 2 * per, nh, 0);
-    else
+    if constexpr (BITS == 8) {
+      if (fast && (a.flags & VC_FLAG_INT8_QK))
+        prep_qk_kernel<D, kStageQuant8I, kTpr, true><<<persistent_grid(2 * per), kRowThreads * kTpr, row_smem, s>>>(a, 2 * per, nh, 0);
+      else if (fast)
+        prep_qk_kernel<D, kStageQuant8, kTpr, true><<<persistent_grid(2 * per), kRowThreads * kTpr, row_smem, s>>>(a, 2 * per, nh, 0);
+      else if (a.flags & VC_FLAG_INT8_QK)
+        prep_qk_kernel<D, kStageQuant8I, kTpr><<<persistent_grid(2 * per), kRowThreads * kTpr, row_smem, s>>>(a, 2 * per, nh, 0);
+      else
+        prep_qk_kernel<D, kStageQuant8, kTpr><<<persistent_grid(2 * per), kRowThreads * kTpr, row_smem, s>>>(a, 2 * per, nh, 0);
+    } else {
       prep_qk_kernel<D, kQuant, kTpr><<<persistent_grid(2 * per), kRowThreads * kTpr, row_smem, s>>>(a, 2 * per, nh, 0);
+    }
     if (BITS == 4 && v_pow2)
       prep_v_kernel<D, kVQuant4M><<<persistent_grid(per), kThreads, v_smem, s>>>(a, per, nh);
     else
