@@ -413,7 +413,6 @@ attn_fwd_2q_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
     // my row of the swizzled code tile: 16-byte chunk c sits at chunk position c ^ (row % 8)
     unsigned char* p_row = sP + t * kPBytes + (row >> 3) * 1024 + (row & 7) * 128;
     const float sq = qblk < nb ? a.q_scale[(size_t)bh * nb + qblk] : 1.0f;
-    const uint64_t k128x2 = pack_f32x2(128.0f, 128.0f), kMagicx2 = pack_f32x2(12582912.0f, 12582912.0f);
     float m_run = -INFINITY;
     float sk_next = __ldg(&a.k_scale[(size_t)bh * nb]);   // fetched one tile ahead: an L2 round trip
     for (int j = 0; j < nb; ++j) {
@@ -477,15 +476,12 @@ attn_fwd_2q_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
       if (j > 0 && !warp_wait2(&sh->o_done[t], (j - 1) & 1, sh, a.status, 31)) break;
 
       const float fa = cs * 0.0625f, fb = (a.code_off - 8.0f * m_new) * 0.0078125f, nm = 8.0f - m_new;
+      const uint64_t fa2 = pack_f32x2(fa, fa), fb2 = pack_f32x2(fb, fb);
       auto code4 = [&](const uint32_t (&sv)[32], int w) -> uint32_t {
         if constexpr (PF == kPfExpCast) {
-          // Eq. 7 in two FMAs: t = sat((8 u + 120 + beta) / 128) clips to [0, 1], then
-          // t * 128 + 1.5 * 2^23 rounds to the nearest even integer in the low mantissa bits.
-          // (the second FMA runs two scores per instruction: the same fp32 operation per score)
-          uint32_t r0, r1, r2, r3;
-          fma_f32x2_bits(r0, r1, fma_sat(__uint_as_float(sv[4 * w]), fa, fb), fma_sat(__uint_as_float(sv[4 * w + 1]), fa, fb), k128x2, kMagicx2);
-          fma_f32x2_bits(r2, r3, fma_sat(__uint_as_float(sv[4 * w + 2]), fa, fb), fma_sat(__uint_as_float(sv[4 * w + 3]), fa, fb), k128x2, kMagicx2);
-          return __byte_perm(__byte_perm(r0, r1, 0x0040), __byte_perm(r2, r3, 0x0040), 0x5410);
+          // Eq. 7: t = (8 u + 120 + beta) / 128, code = round-to-nearest-even(128 t) clipped at 0
+          // (two packed FP32 instructions and a saturating pack per two scores)
+          return expcast_codes4(sv[4 * w], sv[4 * w + 1], sv[4 * w + 2], sv[4 * w + 3], fa2, fb2);
         } else {
           // exponentiate, then cast (Fig. 4a upper box): on the special-function unit, on the
           // FMA pipe by a polynomial, or three and one per word

@@ -318,7 +318,6 @@ attn4_fwd_2q_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     const int p_xor = (row >> 1) & 3;
     uint32_t* sfp_row = reinterpret_cast<uint32_t*>(sSfp + t * kSfpBytes + (row & 31) * 16 + (row >> 5) * 4);
     const float cs = (a.q_g[bh] * a.k_g[bh]) * a.sl;       // code units -> log2 domain
-    const uint64_t k128x2 = pack_f32x2(128.0f, 128.0f), kMagicx2 = pack_f32x2(12582912.0f, 12582912.0f);
     float m_run = -INFINITY;
     for (int j = 0; j < nb; ++j) {
       const int ph = j & 1;
@@ -364,16 +363,13 @@ attn4_fwd_2q_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       mbar_arrive(&sh->a_full[t][j & 1]);
       m_run = m_new;
       if constexpr (HYB) {
-        // ExpCast-FP8 (Eq. 7) in two FMAs: t = sat((8 u + 120 + beta) / 128) clips to [0, 1], then
-        // t * 128 + 1.5 * 2^23 rounds to the nearest even integer in the low mantissa bits.
+        // ExpCast-FP8 (Eq. 7): t = (8 u + 120 + beta) / 128, code = round-to-nearest-even(128 t)
+        // clipped at 0 (two packed FP32 instructions and a saturating pack per two scores)
         if (j > 0 && !warp_wait2(&sh->o_done[t], (j - 1) & 1, sh, a.status, 31)) break;
         const float fa = cs * 0.0625f, fb = (a.code_off - 8.0f * m_new) * 0.0078125f;
+        const uint64_t fa2 = pack_f32x2(fa, fa), fb2 = pack_f32x2(fb, fb);
         auto code4 = [&](const uint32_t (&sv)[32], int w) -> uint32_t {
-          // (the second FMA runs two scores per instruction: the same fp32 operation per score)
-          uint32_t r0, r1, r2, r3;
-          fma_f32x2_bits(r0, r1, fma_sat(__uint_as_float(sv[4 * w]), fa, fb), fma_sat(__uint_as_float(sv[4 * w + 1]), fa, fb), k128x2, kMagicx2);
-          fma_f32x2_bits(r2, r3, fma_sat(__uint_as_float(sv[4 * w + 2]), fa, fb), fma_sat(__uint_as_float(sv[4 * w + 3]), fa, fb), k128x2, kMagicx2);
-          return __byte_perm(__byte_perm(r0, r1, 0x0040), __byte_perm(r2, r3, 0x0040), 0x5410);
+          return expcast_codes4(sv[4 * w], sv[4 * w + 1], sv[4 * w + 2], sv[4 * w + 3], fa2, fb2);
         };
         auto store16 = [&](const uint32_t (&sv)[32], int half, int chunk) {   // keys 16 chunk .. +15
           const uint4 v = make_uint4(code4(sv, 4 * half), code4(sv, 4 * half + 1), code4(sv, 4 * half + 2), code4(sv, 4 * half + 3));

@@ -476,30 +476,6 @@ __device__ __forceinline__ void qk_row_item(const PrepArgs& a, const int TENSOR 
 //    operation per lane, one instruction issued for two);
 //  * 1 / sqrt(D) and the quantization scale are one factor.
 // `kmean_pm` holds (m+, m-) per pair, zeros while Q rows or unsmoothed K rows are processed.
-__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
-  uint64_t d;
-  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
-  return d;
-}
-__device__ __forceinline__ uint64_t sub2(uint64_t a, uint64_t b) {
-  uint64_t d;
-  asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
-  return d;
-}
-__device__ __forceinline__ uint64_t mul2(uint64_t a, uint64_t b) {
-  uint64_t d;
-  asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
-  return d;
-}
-__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
-  uint64_t d;
-  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
-  return d;
-}
-__device__ __forceinline__ void unpack2(uint64_t v, float& lo, float& hi) {
-  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
-}
-
 template <int D, int STAGE, int TPR>
 __device__ __forceinline__ void qk_row_item_fast(const PrepArgs& a, const int TENSOR, const unsigned char* stage,
                                                  unsigned char* out_tile, float* red, float* kmean_pm, uint32_t tab_saddr,

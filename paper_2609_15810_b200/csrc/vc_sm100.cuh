@@ -196,6 +196,60 @@ __device__ __forceinline__ void fma_f32x2_bits(uint32_t& d_lo, uint32_t& d_hi, f
   asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
   asm("mov.b64 {%0, %1}, %2;" : "=r"(d_lo), "=r"(d_hi) : "l"(d));
 }
+// Packed two-lane FP32 arithmetic (add / sub / mul / fma .f32x2): per lane the IEEE operation of
+// the scalar instruction, subnormal results included.
+__device__ __forceinline__ uint64_t pack_b32x2(uint32_t lo, uint32_t hi) {
+  uint64_t d;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(d) : "r"(lo), "r"(hi));
+  return d;
+}
+__device__ __forceinline__ void unpack_b32x2(uint64_t v, uint32_t& lo, uint32_t& hi) {
+  asm("mov.b64 {%0, %1}, %2;" : "=r"(lo), "=r"(hi) : "l"(v));
+}
+__device__ __forceinline__ void unpack2(uint64_t v, float& lo, float& hi) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
+  uint64_t d;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+__device__ __forceinline__ uint64_t sub2(uint64_t a, uint64_t b) {
+  uint64_t d;
+  asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+__device__ __forceinline__ uint64_t mul2(uint64_t a, uint64_t b) {
+  uint64_t d;
+  asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
+  uint64_t d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+// { c[15:0], sat_u8(hi), sat_u8(lo) }: two signed words clamped to 0..255 and packed under 16 bits of c.
+__device__ __forceinline__ uint32_t pack_sat_u8(uint32_t lo, uint32_t hi, uint32_t c) {
+  uint32_t d;
+  asm("cvt.pack.sat.u8.s32.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(hi), "r"(lo), "r"(c));
+  return d;
+}
+// Four ExpCast codes (Eq. 7) from four scores, in five instructions: t = s * fa + fb on two
+// scores at a time; t * 2^-142 is subnormal, so the multiplication rounds 128 t to the nearest
+// even integer INTO THE LOW BITS of the result (the same rounding as adding 1.5 * 2^23), with the
+// sign bit set when t < 0; read as signed words, negative values clamp to code 0 in the packing
+// instruction, which replaces the saturating FMA and the byte permutes.  (t never exceeds
+// (120 + beta) / 128 < 1 because no score exceeds the running maximum.)
+__device__ __forceinline__ uint32_t expcast_codes4(uint32_t s0, uint32_t s1, uint32_t s2, uint32_t s3, uint64_t fa2, uint64_t fb2) {
+  const uint64_t k2 = 0x0000008000000080ull;              // (2^-142, 2^-142)
+  const uint64_t r01 = mul2(fma2(pack_b32x2(s0, s1), fa2, fb2), k2);
+  const uint64_t r23 = mul2(fma2(pack_b32x2(s2, s3), fa2, fb2), k2);
+  uint32_t c0, c1, c2, c3;
+  unpack_b32x2(r01, c0, c1);
+  unpack_b32x2(r23, c2, c3);
+  return pack_sat_u8(c0, c1, pack_sat_u8(c2, c3, 0u));
+}
 __device__ __forceinline__ float ex2_approx(float x) {
   float d;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(d) : "f"(x));
