@@ -474,13 +474,13 @@ __device__ __forceinline__ void qk_row_item(const PrepArgs& a, const int TENSOR 
 //  * a pair lives in one 64-bit register and the other levels, the cross-lane level and the scale
 //    multiply are packed two-lane FP32 instructions (add / sub / fma / mul .f32x2: the same FP32
 //    operation per lane, one instruction issued for two);
-//  * 1 / sqrt(D) and the quantization scale are one factor.
+//  * at 8 bits 1 / sqrt(D) and the quantization scale are one factor.
+// The 4-bit head-maximum and NVFP4 stages run on the same transform.
 // `kmean_pm` holds (m+, m-) per pair, zeros while Q rows or unsmoothed K rows are processed.
 template <int D, int STAGE, int TPR>
 __device__ __forceinline__ void qk_row_item_fast(const PrepArgs& a, const int TENSOR, const unsigned char* stage,
                                                  unsigned char* out_tile, float* red, float* kmean_pm, uint32_t tab_saddr,
                                                  int bh, int blk, int iter, bool new_head, int src_row) {
-  static_assert(STAGE == kStageQuant8 || STAGE == kStageQuant8I, "the packed path covers the 8-bit stages");
   constexpr int C = D / TPR, P = C / 2;            // channels and pairs per thread
   constexpr int NT = kRowThreads * TPR;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -561,21 +561,86 @@ __device__ __forceinline__ void qk_row_item_fast(const PrepArgs& a, const int TE
   }
   constexpr float rs = D == 128 ? 0.08838834764831845f : 0.125f;   // 1/sqrt(D)
 
-  float m0 = 0.f, m1 = 0.f;
+  float amax = 0.f;
+  if constexpr (STAGE != kStageQuant4) {
+    float m0 = 0.f, m1 = 0.f;
 #pragma unroll
-  for (int i = 0; i < P; i += 2) {
-    float a0, a1, b0, b1;
-    unpack2(X[i], a0, a1);
-    unpack2(X[i + 1], b0, b1);
-    m0 = max3(m0, fabsf(a0), fabsf(a1));
-    m1 = max3(m1, fabsf(b0), fabsf(b1));
+    for (int i = 0; i < P; i += 2) {
+      float a0, a1, b0, b1;
+      unpack2(X[i], a0, a1);
+      unpack2(X[i + 1], b0, b1);
+      m0 = max3(m0, fabsf(a0), fabsf(a1));
+      m1 = max3(m1, fabsf(b0), fabsf(b1));
+    }
+    amax = warp_max(fmaxf(m0, m1) * rs);           // max and the (positive) scale commute exactly
+    float* rbuf = red + 8 * (iter & 1);            // alternate buffers: one barrier per item suffices
+    if (lane == 0) rbuf[warp] = amax;
+    __syncthreads();
+    amax = fmaxf(fmaxf(rbuf[0], rbuf[1]), fmaxf(rbuf[2], rbuf[3]));
+    if constexpr (TPR == 2) amax = fmaxf(amax, fmaxf(fmaxf(rbuf[4], rbuf[5]), fmaxf(rbuf[6], rbuf[7])));
   }
-  float amax = warp_max(fmaxf(m0, m1) * rs);       // max and the (positive) scale commute exactly
-  float* rbuf = red + 8 * (iter & 1);              // alternate buffers: one barrier per item suffices
-  if (lane == 0) rbuf[warp] = amax;
-  __syncthreads();
-  amax = fmaxf(fmaxf(rbuf[0], rbuf[1]), fmaxf(rbuf[2], rbuf[3]));
-  if constexpr (TPR == 2) amax = fmaxf(amax, fmaxf(fmaxf(rbuf[4], rbuf[5]), fmaxf(rbuf[6], rbuf[7])));
+  if constexpr (STAGE == kStageAmax) {
+    if (tid == 0) atomicMax(&a.qk_amax[TENSOR * a.BH + bh], __float_as_uint(amax));
+    return;
+  }
+  if constexpr (STAGE == kStageQuant4) {
+    // NVFP4: outer scale g per (b, h), microscale per token per 16 channels (the arithmetic of the
+    // general row body: y = x / sqrt(D), then y / (g * microscale), each rounded once)
+    const float g = (TENSOR == 0 ? a.q_scale : a.k_scale)[bh];
+    const float inv6 = 1.0f / (6.0f * g);
+    const uint64_t RS = pack_f32x2(rs, rs);
+    constexpr int MB = C / 16;                     // microscale bytes of this thread
+    unsigned int codes[C / 8], micro[(MB + 3) / 4];
+#pragma unroll
+    for (int i = 0; i < (MB + 3) / 4; ++i) micro[i] = 0;
+#pragma unroll
+    for (int gq = 0; gq < C / 16; ++gq) {
+      float m0 = 0.f, m1 = 0.f;
+#pragma unroll
+      for (int i = 0; i < 8; i += 2) {
+        float a0, a1, b0, b1;
+        X[8 * gq + i] = mul2(X[8 * gq + i], RS);
+        X[8 * gq + i + 1] = mul2(X[8 * gq + i + 1], RS);
+        unpack2(X[8 * gq + i], a0, a1);
+        unpack2(X[8 * gq + i + 1], b0, b1);
+        m0 = max3(m0, fabsf(a0), fabsf(a1));
+        m1 = max3(m1, fabsf(b0), fabsf(b1));
+      }
+      const float m = fmaxf(m0, m1);
+      const unsigned int sb = __nv_cvt_float_to_fp8(m * inv6, __NV_SATFINITE, __NV_E4M3);
+      const float sdec = e4m3_to_float(sb);
+      const float rcp = sdec > 0.f ? 1.0f / (g * sdec) : 0.f;
+      const uint64_t RC = pack_f32x2(rcp, rcp);
+      micro[gq / 4] |= sb << (8 * (gq & 3));
+#pragma unroll
+      for (int wi = 0; wi < 2; ++wi) {
+        unsigned int word = 0;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          float y0, y1;
+          unpack2(mul2(X[8 * gq + 4 * wi + j], RC), y0, y1);
+          const unsigned int two = __nv_cvt_float2_to_fp4x2(make_float2(y0, y1), __NV_E2M1, cudaRoundNearest);
+          word |= (two & 0xffu) << (8 * j);
+        }
+        codes[2 * gq + wi] = sdec > 0.f ? word : 0u;
+      }
+    }
+    constexpr int CPR4 = D / 32;
+    uint4* dst4 = reinterpret_cast<uint4*>(out_tile + row * (D / 2));
+    const int sw4 = (row / (8 / CPR4)) & (CPR4 - 1);
+#pragma unroll
+    for (int i = 0; i < C / 32; ++i) dst4[(part * (C / 32) + i) ^ sw4] = make_uint4(codes[4 * i], codes[4 * i + 1], codes[4 * i + 2], codes[4 * i + 3]);
+    const size_t row_g = (size_t)bh * a.n_pad + (size_t)blk * kBlock + row;
+    uint8_t* mrow = (TENSOR == 0 ? a.q_micro : a.k_micro) + row_g * (D / 16) + part * MB;
+    if constexpr (MB % 4 == 0) {
+#pragma unroll
+      for (int i = 0; i < MB / 4; ++i) reinterpret_cast<unsigned int*>(mrow)[i] = micro[i];
+    } else {
+      static_assert(MB == 2, "microscale bytes per thread");
+      *reinterpret_cast<unsigned short*>(mrow) = (unsigned short)micro[0];
+    }
+    return;
+  }
 
   constexpr bool int8 = STAGE == kStageQuant8I;
   const float top = int8 ? 127.0f : 448.0f;
@@ -1037,7 +1102,7 @@ __global__ void prep_finalize_kernel(const PrepArgs a, int which) {
 // data needs warp-level synchronization only; the one CTA-wide barrier per item is the exchange
 // of the block maximum.
 // Shared memory: [2 stages x 128 x pitch][out tile 128 x D][src ring 3 x 128][scratch][RoPE table].
-// FAST: the packed row transform (standard configuration, 8-bit stages), see qk_row_item_fast.
+// FAST: the packed row transform (standard configuration), see qk_row_item_fast.
 template <int D, int STAGE, int TPR, bool FAST = false>
 __global__ void __launch_bounds__(kRowThreads * TPR, 2) prep_qk_kernel(const PrepArgs a, int n_items, int nh, int z0) {
   constexpr int NT = kRowThreads * TPR;
@@ -1162,8 +1227,10 @@ cudaError_t run(const Problem& pr, PrepArgs a, const WorkLayout& wl, uint8_t* wo
   if (BITS == 8 && (e = allow_smem(prep_qk_kernel<D, kStageQuant8, kTpr, true>, row_smem)) != cudaSuccess) return e;
   if (BITS == 8 && (e = allow_smem(prep_qk_kernel<D, kStageQuant8I, kTpr, true>, row_smem)) != cudaSuccess) return e;
   // the packed row transform serves the standard configuration
-  const bool fast = BITS == 8 && (a.flags & VC_FLAG_ROPE) && (a.flags & VC_FLAG_HADAMARD) && a.rope_default && a.rope_in_smem;
+  const bool fast = (a.flags & VC_FLAG_ROPE) && (a.flags & VC_FLAG_HADAMARD) && a.rope_default && a.rope_in_smem;
   if (BITS == 4 && (e = allow_smem(prep_qk_kernel<D, kStageAmax, kTpr>, row_smem)) != cudaSuccess) return e;
+  if (BITS == 4 && (e = allow_smem(prep_qk_kernel<D, kStageAmax, kTpr, true>, row_smem)) != cudaSuccess) return e;
+  if (BITS == 4 && (e = allow_smem(prep_qk_kernel<D, kStageQuant4, kTpr, true>, row_smem)) != cudaSuccess) return e;
   int group = pr.heads_per_pass > 0 ? pr.heads_per_pass : pr.BH;
   if (group > 32768) group = 32768;
   for (int bh0 = 0; bh0 < pr.BH; bh0 += group) {
@@ -1176,13 +1243,18 @@ cudaError_t run(const Problem& pr, PrepArgs a, const WorkLayout& wl, uint8_t* wo
       count_launches(1);
     }
     if (BITS == 8 && !ext) { prep_v_kernel<D, kVStats><<<persistent_grid(per), kThreads, v_smem, s>>>(a, per, nh); count_launches(1); }
-    if (BITS == 4) { prep_qk_kernel<D, kStageAmax, kTpr><<<persistent_grid(per), kRowThreads * kTpr, row_smem, s>>>(a, per, nh, 0); count_launches(1); }
+    auto amax_pass = [&](int z0) {
+      if (fast) prep_qk_kernel<D, kStageAmax, kTpr, true><<<persistent_grid(per), kRowThreads * kTpr, row_smem, s>>>(a, per, nh, z0);
+      else prep_qk_kernel<D, kStageAmax, kTpr><<<persistent_grid(per), kRowThreads * kTpr, row_smem, s>>>(a, per, nh, z0);
+      count_launches(1);
+    };
+    if (BITS == 4) amax_pass(0);
     prep_finalize_kernel<D, BITS><<<nh, 8 * D, 0, s>>>(a, ext ? 2 : 0);
     count_launches(1);
     if (BITS == 4) {
-      prep_qk_kernel<D, kStageAmax, kTpr><<<persistent_grid(per), kRowThreads * kTpr, row_smem, s>>>(a, per, nh, 1);
+      amax_pass(1);
       prep_finalize_kernel<D, BITS><<<nh, 32, 0, s>>>(a, 1);
-      count_launches(2);
+      count_launches(1);
     }
     if constexpr (BITS == 8) {
       if (fast && (a.flags & VC_FLAG_INT8_QK))
@@ -1194,7 +1266,8 @@ cudaError_t run(const Problem& pr, PrepArgs a, const WorkLayout& wl, uint8_t* wo
       else
         prep_qk_kernel<D, kStageQuant8, kTpr><<<persistent_grid(2 * per), kRowThreads * kTpr, row_smem, s>>>(a, 2 * per, nh, 0);
     } else {
-      prep_qk_kernel<D, kQuant, kTpr><<<persistent_grid(2 * per), kRowThreads * kTpr, row_smem, s>>>(a, 2 * per, nh, 0);
+      if (fast) prep_qk_kernel<D, kStageQuant4, kTpr, true><<<persistent_grid(2 * per), kRowThreads * kTpr, row_smem, s>>>(a, 2 * per, nh, 0);
+      else prep_qk_kernel<D, kStageQuant4, kTpr><<<persistent_grid(2 * per), kRowThreads * kTpr, row_smem, s>>>(a, 2 * per, nh, 0);
     }
     if (BITS == 4 && v_pow2)
       prep_v_kernel<D, kVQuant4M><<<persistent_grid(per), kThreads, v_smem, s>>>(a, per, nh);
