@@ -55,6 +55,10 @@ def test_sizes_and_argument_validation_without_a_gpu():
     assert lib.vc_prep(C.byref(pb), 16, 16, 16, None, 16, 16, None) == vc.VC_ERR_UNSUPPORTED      # refused before any launch
     pb = Params.make(1, 2, 1024, 128, (4, 16, 16), block_v=-1)
     assert lib.vc_prep(C.byref(pb), 16, 16, 16, None, 16, 16, None) == vc.VC_ERR_INVALID_ARG
+    # a row stride has to fit 32 bits in bytes (the kernels address rows with one 32 x 32 -> 64 multiply)
+    pb = Params.make(1, 2, 1024, 128, (4, 16, 16), stride_n=1 << 30, stride_h=1 << 41, stride_b=1 << 43)
+    assert lib.vc_prep(C.byref(pb), 16, 16, 16, None, 16, 16, None) == vc.VC_ERR_UNSUPPORTED
+    assert vc.vc_quant_bytes(Params.make(1, 2, 1024, 128, (4, 16, 16), stride_n=256, stride_h=1024 * 256, stride_b=2 * 1024 * 256)) == qb0
     # the validator's bitmap is part of the workspace only when it is asked for
     pc = Params.make(1, 2, 1024, 128, (4, 16, 16), flags=vc.VC_FLAG_ALL | vc.VC_FLAG_CHECK_PERM)
     assert vc.vc_workspace_bytes(pc) > vc.vc_workspace_bytes(Params.make(1, 2, 1024, 128, (4, 16, 16)))
