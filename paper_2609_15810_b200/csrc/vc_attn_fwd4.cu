@@ -398,10 +398,17 @@ attn4_fwd_2q_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       // the previous code tile must have been consumed before it is overwritten
       if (j > 0 && !warp_wait2(&sh->o_done[t], (j - 1) & 1, sh, a.status, 31)) break;
 
+      const uint64_t cs2 = pack_f32x2(cs, cs);
       auto quant16 = [&](const uint32_t (&sv)[32], int half, int g) -> uint2 {   // keys 16 g .. 16 g + 15
         float v[16];
+        const uint64_t off2 = pack_f32x2(off[g], off[g]);
 #pragma unroll
-        for (int i = 0; i < 16; ++i) v[i] = ex2_approx(fmaf(__uint_as_float(sv[16 * half + i]), cs, off[g]));
+        for (int i = 0; i < 16; i += 2) {                 // the exponent's FMA on two scores per instruction
+          float x0, x1;
+          unpack2(fma2(pack_b32x2(sv[16 * half + i], sv[16 * half + i + 1]), cs2, off2), x0, x1);
+          v[i] = ex2_approx(x0);
+          v[i + 1] = ex2_approx(x1);
+        }
         return make_uint2(cvt_e2m1x8(v[0], v[1], v[2], v[3], v[4], v[5], v[6], v[7]),
                           cvt_e2m1x8(v[8], v[9], v[10], v[11], v[12], v[13], v[14], v[15]));
       };
