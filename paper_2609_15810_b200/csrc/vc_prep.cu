@@ -42,9 +42,10 @@ __global__ void rope_table_kernel(float2* tab, RopeDesc rd, double theta) {
 // 128 rows); a CTA takes items blockIdx.x, blockIdx.x + gridDim.x, ...  The 16-byte chunks of
 // the NEXT items are already on their way into a ring of shared-memory stages (cp.async, no
 // registers held for bytes in flight) while the current item is transformed, so the load
-// latency of a block hides behind the arithmetic of the blocks before it.  For Q and K a
-// thread fetches exactly the chunks it will read itself, so those passes need no barrier for
-// the data at all; V is staged as a tile because its codes leave channel-major.
+// latency of a block hides behind the arithmetic of the blocks before it.  In the K column sums
+// a thread fetches exactly the chunks it will read itself and in the Q/K pass a warp fetches
+// exactly the rows it will transform, so those passes need no CTA-wide barrier for the data;
+// V is staged as a tile because its codes leave channel-major.
 // (One bulk-async copy per gathered row was tried instead of cp.async: 128 small copies per
 // block kept the copy engine, not HBM, busy.)
 constexpr int kThreads = 256;      // threads of the column-sum and V passes
