@@ -2,7 +2,7 @@
 // App. B): every operand is read as bf16 with 16-byte vector loads and leaves as low-bit
 // codes plus scales; no rotated / permuted / centered high-precision tensor reaches HBM.
 //
-//   Q : RoPE -> Hadamard (in registers, one row per thread) -> per-128-row scale -> codes
+//   Q : RoPE -> Hadamard (in registers, a row in two threads) -> per-128-row scale -> codes
 //   K : RoPE -> column sums (stats launch) ... gather by pi -> RoPE at the source position
 //       -> subtract channel mean -> Hadamard -> scale -> codes
 //   V : gather by pi -> block mean (Eq. 4) and residual amax (stats launch) ...
@@ -52,6 +52,9 @@ constexpr int kThreads = 256;      // threads of the column-sum and V passes
 constexpr int kRowThreads = 128;   // rows of a Q/K item (threads of the pass = rows x threads per row)
 #ifndef VC_PREP_TPR
 #define VC_PREP_TPR 2
+#endif
+#ifndef VC_PREP_TPR_FAST
+#define VC_PREP_TPR_FAST VC_PREP_TPR      // threads per row of the packed row transform
 #endif
 
 template <int D> struct Geo {
@@ -258,9 +261,11 @@ template <> struct RopeSplit<64> { static constexpr int p1 = 12, p2 = 22; };    
 // level crosses the two halves with one shuffle per value.  RoPE pairs and NVFP4 groups stay
 // thread-local either way.
 template <int TPR> __device__ __forceinline__ int qk_row_of(int tid) {
-  return TPR == 1 ? tid : 16 * (tid >> 5) + (tid & 15);
+  return TPR == 1 ? tid : (TPR == 2 ? 16 * (tid >> 5) + (tid & 15) : 8 * (tid >> 5) + (tid & 7));
 }
-template <int TPR> __device__ __forceinline__ int qk_part_of(int tid) { return TPR == 1 ? 0 : (tid >> 4) & 1; }
+template <int TPR> __device__ __forceinline__ int qk_part_of(int tid) {
+  return TPR == 1 ? 0 : (TPR == 2 ? (tid >> 4) & 1 : (tid >> 3) & 3);
+}
 
 template <int D> __device__ __forceinline__ constexpr int rope_axis_of(int p) {
   return p < RopeSplit<D>::p1 ? 0 : (p < RopeSplit<D>::p2 ? 1 : 2);
@@ -507,11 +512,14 @@ __device__ __forceinline__ void qk_row_item_fast(const PrepArgs& a, const int TE
   const int p0 = part * P;
   // byte address of pair i's entry = base of its axis + 8 i (the axis of local pair i is known at
   // compile time for either part: one base per combination, selected once per row)
-  uint32_t base[3][3];
-#pragma unroll
-  for (int a0 = 0; a0 < 3; ++a0)
-#pragma unroll
-    for (int a1 = 0; a1 < 3; ++a1) base[a0][a1] = tab_saddr + 8u * (uint32_t)((part ? e[a1] : e[a0]) + p0);
+  // (written as a selection per pair; identical selections fold into one value per combination)
+  auto base_of = [&](int i) -> uint32_t {          // i is a compile-time constant after unrolling
+    int ee;
+    if constexpr (TPR == 1) ee = e[rope_axis_of<D>(i)];
+    else if constexpr (TPR == 2) ee = part ? e[rope_axis_of<D>(P + i)] : e[rope_axis_of<D>(i)];
+    else ee = part == 0 ? e[rope_axis_of<D>(i)] : (part == 1 ? e[rope_axis_of<D>(P + i)] : (part == 2 ? e[rope_axis_of<D>(2 * P + i)] : e[rope_axis_of<D>(3 * P + i)]));
+    return tab_saddr + 8u * (uint32_t)(ee + p0);
+  };
   const float4* km = reinterpret_cast<const float4*>(kmean_pm + part * C);
 
   uint64_t X[P];
@@ -525,7 +533,7 @@ __device__ __forceinline__ void qk_row_item_fast(const PrepArgs& a, const int TE
       const float x0 = __uint_as_float(w << 16), x1 = __uint_as_float(w & 0xffff0000u);
       float A, B;
       asm("ld.shared.v2.f32 {%0, %1}, [%2];" : "=f"(A), "=f"(B)
-          : "r"(base[rope_axis_of<D>(ii)][rope_axis_of<D>(TPR == 1 ? ii : P + ii)] + 8u * ii));
+          : "r"(base_of(ii) + 8u * ii));
       const float mp = k == 0 ? m.x : m.z, mm = k == 0 ? m.y : m.w;
       const float u = fmaf(x0, A, fmaf(x1, B, -mp));
       const float v = fmaf(x0, B, fmaf(-x1, A, -mm));
@@ -548,16 +556,21 @@ __device__ __forceinline__ void qk_row_item_fast(const PrepArgs& a, const int TE
       }
     }
   }
-  if constexpr (TPR == 2) {
-    // the level that pairs channel c with c + D/2: lower half mine + theirs, upper half theirs - mine
-    const float sg = part ? -1.0f : 1.0f;
-    const uint64_t SG = pack_f32x2(sg, sg);
+  if constexpr (TPR >= 2) {
+    // the levels that pair channels across the threads of a row (distance C, then 2 C with four
+    // threads per row): the lower part takes mine + theirs, the upper part theirs - mine
 #pragma unroll
-    for (int i = 0; i < P; ++i) {
-      float lo, hi;
-      unpack2(X[i], lo, hi);
-      const float olo = __shfl_xor_sync(0xffffffffu, lo, 16), ohi = __shfl_xor_sync(0xffffffffu, hi, 16);
-      X[i] = fma2(X[i], SG, pack_f32x2(olo, ohi));
+    for (int lv = 0; lv < (TPR == 2 ? 1 : 2); ++lv) {
+      const int mask = TPR == 2 ? 16 : (lv == 0 ? 8 : 16);
+      const float sg = ((part >> lv) & 1) ? -1.0f : 1.0f;
+      const uint64_t SG = pack_f32x2(sg, sg);
+#pragma unroll
+      for (int i = 0; i < P; ++i) {
+        float lo, hi;
+        unpack2(X[i], lo, hi);
+        const float olo = __shfl_xor_sync(0xffffffffu, lo, mask), ohi = __shfl_xor_sync(0xffffffffu, hi, mask);
+        X[i] = fma2(X[i], SG, pack_f32x2(olo, ohi));
+      }
     }
   }
   constexpr float rs = D == 128 ? 0.08838834764831845f : 0.125f;   // 1/sqrt(D)
@@ -574,11 +587,15 @@ __device__ __forceinline__ void qk_row_item_fast(const PrepArgs& a, const int TE
       m1 = max3(m1, fabsf(b0), fabsf(b1));
     }
     amax = warp_max(fmaxf(m0, m1) * rs);           // max and the (positive) scale commute exactly
-    float* rbuf = red + 8 * (iter & 1);            // alternate buffers: one barrier per item suffices
+    float* rbuf = red + 16 * (iter & 1);           // alternate buffers: one barrier per item suffices
     if (lane == 0) rbuf[warp] = amax;
     __syncthreads();
     amax = fmaxf(fmaxf(rbuf[0], rbuf[1]), fmaxf(rbuf[2], rbuf[3]));
-    if constexpr (TPR == 2) amax = fmaxf(amax, fmaxf(fmaxf(rbuf[4], rbuf[5]), fmaxf(rbuf[6], rbuf[7])));
+    if constexpr (TPR >= 2) amax = fmaxf(amax, fmaxf(fmaxf(rbuf[4], rbuf[5]), fmaxf(rbuf[6], rbuf[7])));
+    if constexpr (TPR == 4) {
+      amax = fmaxf(amax, fmaxf(fmaxf(rbuf[8], rbuf[9]), fmaxf(rbuf[10], rbuf[11])));
+      amax = fmaxf(amax, fmaxf(fmaxf(rbuf[12], rbuf[13]), fmaxf(rbuf[14], rbuf[15])));
+    }
   }
   if constexpr (STAGE == kStageAmax) {
     if (tid == 0) atomicMax(&a.qk_amax[TENSOR * a.BH + bh], __float_as_uint(amax));
@@ -1115,8 +1132,8 @@ __global__ void __launch_bounds__(kRowThreads * TPR, 2) prep_qk_kernel(const Pre
   extern __shared__ __align__(128) unsigned char smem[];
   unsigned char* out_tile = smem + 2 * Geo<D>::stage_bytes;
   int* src_ring = reinterpret_cast<int*>(out_tile + kBlock * D);     // [3][128]
-  float* red = reinterpret_cast<float*>(src_ring + 3 * kBlock);      // [2][8]
-  float* kmean_s = red + 16;                                         // [D]
+  float* red = reinterpret_cast<float*>(src_ring + 3 * kBlock);      // [2][16]
+  float* kmean_s = red + 32;                                         // [D]
   const int tid = threadIdx.x, lane = tid & 31, row0 = (tid >> 5) * RW;
   if (FAST) {
     for (int c = tid; c < D; c += NT) kmean_s[c] = 0.f;    // (m+, m-) pairs: zeros until a smoothed K head arrives
@@ -1212,10 +1229,11 @@ template <int D, int BITS>
 cudaError_t run(const Problem& pr, PrepArgs a, const WorkLayout& wl, uint8_t* work, cudaStream_t s) {
   const size_t rope_bytes = ((a.flags & VC_FLAG_ROPE) && a.rope_in_smem) ? (size_t)a.rd.entries * 8 : 0;
   const size_t colsum_smem = 2 * (size_t)kThreads * (D / 16) * 16 + 8 * D * 4 + rope_bytes;
-  const size_t row_smem = 2 * (size_t)Geo<D>::stage_bytes + (size_t)kBlock * D + 3 * kBlock * 4 + 64 + D * 4 + rope_bytes;
+  const size_t row_smem = 2 * (size_t)Geo<D>::stage_bytes + (size_t)kBlock * D + 3 * kBlock * 4 + 128 + D * 4 + rope_bytes;
   const size_t v_smem = 3 * (size_t)kBlock * 2 * D + 16 * D * 4 + 2 * kBlock * 4;
   constexpr int kQuant = BITS == 8 ? kStageQuant8 : kStageQuant4;
   constexpr int kTpr = VC_PREP_TPR;            // threads per Q/K row
+  constexpr int kTprF = D == 128 ? VC_PREP_TPR_FAST : VC_PREP_TPR;   // ... of the packed row transform
   constexpr int kVQuant = BITS == 8 ? kVQuant8 : kVQuant4;
   cudaError_t e;
   if ((e = allow_smem(prep_kcolsum_kernel<D>, colsum_smem)) != cudaSuccess) return e;
@@ -1225,13 +1243,13 @@ cudaError_t run(const Problem& pr, PrepArgs a, const WorkLayout& wl, uint8_t* wo
   const bool v_pow2 = hybrid4(pr);           // 4-bit values under power-of-two factors per 32 tokens
   if ((e = allow_smem(prep_qk_kernel<D, kQuant, kTpr>, row_smem)) != cudaSuccess) return e;
   if (BITS == 8 && (e = allow_smem(prep_qk_kernel<D, kStageQuant8I, kTpr>, row_smem)) != cudaSuccess) return e;
-  if (BITS == 8 && (e = allow_smem(prep_qk_kernel<D, kStageQuant8, kTpr, true>, row_smem)) != cudaSuccess) return e;
-  if (BITS == 8 && (e = allow_smem(prep_qk_kernel<D, kStageQuant8I, kTpr, true>, row_smem)) != cudaSuccess) return e;
+  if (BITS == 8 && (e = allow_smem(prep_qk_kernel<D, kStageQuant8, kTprF, true>, row_smem)) != cudaSuccess) return e;
+  if (BITS == 8 && (e = allow_smem(prep_qk_kernel<D, kStageQuant8I, kTprF, true>, row_smem)) != cudaSuccess) return e;
   // the packed row transform serves the standard configuration
   const bool fast = (a.flags & VC_FLAG_ROPE) && (a.flags & VC_FLAG_HADAMARD) && a.rope_default && a.rope_in_smem;
   if (BITS == 4 && (e = allow_smem(prep_qk_kernel<D, kStageAmax, kTpr>, row_smem)) != cudaSuccess) return e;
-  if (BITS == 4 && (e = allow_smem(prep_qk_kernel<D, kStageAmax, kTpr, true>, row_smem)) != cudaSuccess) return e;
-  if (BITS == 4 && (e = allow_smem(prep_qk_kernel<D, kStageQuant4, kTpr, true>, row_smem)) != cudaSuccess) return e;
+  if (BITS == 4 && (e = allow_smem(prep_qk_kernel<D, kStageAmax, kTprF, true>, row_smem)) != cudaSuccess) return e;
+  if (BITS == 4 && (e = allow_smem(prep_qk_kernel<D, kStageQuant4, kTprF, true>, row_smem)) != cudaSuccess) return e;
   int group = pr.heads_per_pass > 0 ? pr.heads_per_pass : pr.BH;
   if (group > 32768) group = 32768;
   for (int bh0 = 0; bh0 < pr.BH; bh0 += group) {
@@ -1245,7 +1263,7 @@ cudaError_t run(const Problem& pr, PrepArgs a, const WorkLayout& wl, uint8_t* wo
     }
     if (BITS == 8 && !ext) { prep_v_kernel<D, kVStats><<<persistent_grid(per), kThreads, v_smem, s>>>(a, per, nh); count_launches(1); }
     auto amax_pass = [&](int z0) {
-      if (fast) prep_qk_kernel<D, kStageAmax, kTpr, true><<<persistent_grid(per), kRowThreads * kTpr, row_smem, s>>>(a, per, nh, z0);
+      if (fast) prep_qk_kernel<D, kStageAmax, kTprF, true><<<persistent_grid(per), kRowThreads * kTprF, row_smem, s>>>(a, per, nh, z0);
       else prep_qk_kernel<D, kStageAmax, kTpr><<<persistent_grid(per), kRowThreads * kTpr, row_smem, s>>>(a, per, nh, z0);
       count_launches(1);
     };
@@ -1259,15 +1277,15 @@ cudaError_t run(const Problem& pr, PrepArgs a, const WorkLayout& wl, uint8_t* wo
     }
     if constexpr (BITS == 8) {
       if (fast && (a.flags & VC_FLAG_INT8_QK))
-        prep_qk_kernel<D, kStageQuant8I, kTpr, true><<<persistent_grid(2 * per), kRowThreads * kTpr, row_smem, s>>>(a, 2 * per, nh, 0);
+        prep_qk_kernel<D, kStageQuant8I, kTprF, true><<<persistent_grid(2 * per), kRowThreads * kTprF, row_smem, s>>>(a, 2 * per, nh, 0);
       else if (fast)
-        prep_qk_kernel<D, kStageQuant8, kTpr, true><<<persistent_grid(2 * per), kRowThreads * kTpr, row_smem, s>>>(a, 2 * per, nh, 0);
+        prep_qk_kernel<D, kStageQuant8, kTprF, true><<<persistent_grid(2 * per), kRowThreads * kTprF, row_smem, s>>>(a, 2 * per, nh, 0);
       else if (a.flags & VC_FLAG_INT8_QK)
         prep_qk_kernel<D, kStageQuant8I, kTpr><<<persistent_grid(2 * per), kRowThreads * kTpr, row_smem, s>>>(a, 2 * per, nh, 0);
       else
         prep_qk_kernel<D, kStageQuant8, kTpr><<<persistent_grid(2 * per), kRowThreads * kTpr, row_smem, s>>>(a, 2 * per, nh, 0);
     } else {
-      if (fast) prep_qk_kernel<D, kStageQuant4, kTpr, true><<<persistent_grid(2 * per), kRowThreads * kTpr, row_smem, s>>>(a, 2 * per, nh, 0);
+      if (fast) prep_qk_kernel<D, kStageQuant4, kTprF, true><<<persistent_grid(2 * per), kRowThreads * kTprF, row_smem, s>>>(a, 2 * per, nh, 0);
       else prep_qk_kernel<D, kStageQuant4, kTpr><<<persistent_grid(2 * per), kRowThreads * kTpr, row_smem, s>>>(a, 2 * per, nh, 0);
     }
     if (BITS == 4 && v_pow2)
