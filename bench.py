@@ -481,7 +481,7 @@ def main():
     # DRAM traffic of one attention launch: measured once under ncu on a smaller case of the same
     # kernel (the headline launch is too long to capture) and proportional to B*H*N (codes in,
     # bf16 out; key/value re-reads are L2 hits)
-    per_ht = {8: 323.9e6, 4: 220.6e6}[args.bits] / (32 * 16384) * (w.d / 128.0)
+    per_ht = {8: 322.2e6, 4: 219.2e6}[args.bits] / (32 * 16384) * (w.d / 128.0)
     traffic = per_ht * w.B * w.H * w.N
     n_pad = 128 * ((w.N + 127) // 128)
     prep_bytes = w.B * w.H * (3 * w.N * w.d * 2 + 2 * w.N * 4 + 3 * n_pad * w.d * (1 if args.bits == 8 else 0.5625)
