@@ -290,6 +290,16 @@ vc_status vc_poll_status(void *workspace, void *stream);
  * memory and return; outputs of such a call are invalid.  Process-wide; not for production. */
 void vc_test_set_wait_limit(uint32_t polls);
 
+/* Test hook: the ExpCast-FP8 probability code (Eq. 7) formed exactly as the softmax stage of the
+ * attention kernels forms it, on its own.  codes[i] is the E4M3 byte of score s[i] (FP32, in units
+ * of the integer-like score product) under the factor `cs` that takes such units to the log2
+ * domain (> 0) and the running row maximum `m` (log2 domain; s[i] * cs <= m is the caller's
+ * business): round-to-nearest-even(8 (s cs - m) + 120 + beta), clipped at 0.  beta 0 => -0.35.
+ * `s` and `codes` are device pointers, 16-byte aligned; n is a multiple of 4.  Asynchronous on
+ * `stream`; VC_ERR_INVALID_ARG for a bad argument.  Not for production. */
+vc_status vc_test_expcast_codes(const float *s, int64_t n, float cs, float m, float beta,
+                                uint8_t *codes, void *stream);
+
 /* Measurement aid (Sec. 3.1 "The softmax bottleneck" compares the softmax stage with the time of
  * the two matrix products): the rate at which this GPU executes the products' MMAs with
  * everything else taken away.  Every SM issues `groups` back-to-back 128 x 128 x 128 products of

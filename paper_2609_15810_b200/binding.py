@@ -104,6 +104,8 @@ def load_library():
     lib.vc_poll_status.argtypes = [vp, vp]
     lib.vc_test_set_wait_limit.restype = None
     lib.vc_test_set_wait_limit.argtypes = [ctypes.c_uint32]
+    lib.vc_test_expcast_codes.restype = ctypes.c_int
+    lib.vc_test_expcast_codes.argtypes = [vp, ctypes.c_int64, ctypes.c_float, ctypes.c_float, ctypes.c_float, vp, vp]
     lib.vc_mma_peak.restype = ctypes.c_int
     lib.vc_mma_peak.argtypes = [ctypes.c_int32, ctypes.c_int32, vp, ctypes.POINTER(ctypes.c_double),
                                 ctypes.POINTER(ctypes.c_double), vp]
@@ -223,6 +225,16 @@ def vc_poll_status(workspace):
 def vc_test_set_wait_limit(polls):
     """Test hook: polls after which a device-side wait gives up (0 = the default)."""
     load_library().vc_test_set_wait_limit(int(polls))
+
+
+def vc_test_expcast_codes(s, cs, m, beta=0.0):
+    """Test hook: the ExpCast-FP8 codes of the fp32 scores `s` (CUDA tensor, numel a multiple of 4)
+    under the factor cs and the running maximum m, as the attention kernels form them (uint8 tensor)."""
+    assert s.dtype == torch.float32 and s.is_cuda and s.is_contiguous()
+    out = torch.empty(s.numel(), dtype=torch.uint8, device=s.device)
+    _check(load_library().vc_test_expcast_codes(_ptr(s), s.numel(), float(cs), float(m), float(beta), _ptr(out), _stream()),
+           "vc_test_expcast_codes")
+    return out.view(s.shape)
 
 
 def vc_mma_peak(kind, groups=4096):

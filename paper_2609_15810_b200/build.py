@@ -14,7 +14,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libvc.so")
-SOURCES = ["vc_api.cu", "vc_prep.cu", "vc_perm_check.cu", "vc_attn_fwd.cu", "vc_attn_fwd4.cu", "vc_group.cu", "vc_mma_peak.cu"]
+SOURCES = ["vc_api.cu", "vc_prep.cu", "vc_perm_check.cu", "vc_attn_fwd.cu", "vc_attn_fwd4.cu", "vc_group.cu", "vc_mma_peak.cu", "vc_test_hooks.cu"]
 NVCC = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
 FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
          "-Xcompiler", "-fPIC", "-I", os.path.join(ROOT, "include"), "-I", CSRC]
